@@ -1,0 +1,96 @@
+"""Workload descriptions for the FreqFormer heterogeneous attention forward.
+
+Pure data: grid sizes, band cut-offs and operator parameters in the paper's
+notation (Method, "Setup and notation" .. "Cross-band residual exchange").
+No arithmetic of the method lives here; both the CUDA path and the test
+oracle read these records.
+
+Notation
+  T, H, W     token grid (temporal, height, width); N = T*H*W
+  heads, d    number of heads n_h and per-head width d_k
+  low_cut     per-axis cut-off L_a: coefficient k is LOW iff k_a < L_a on all axes
+  mid_cut     per-axis cut-off M_a: MID iff not LOW and k_a < M_a on all axes
+  r           low-band compression ratio (N_low -> ceil(N_low / r))
+  b, s        mid-band block size and block stride
+  R           high-band window radius (w = 2R+1 keys before clipping)
+  m           summary tokens per band
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, replace
+from typing import Tuple
+
+
+@dataclass(frozen=True)
+class FFConfig:
+    name: str
+    batch: int
+    T: int
+    H: int
+    W: int
+    heads: int
+    head_dim: int
+    dtype: str                      # "bf16" or "fp32": storage type of Q, K, V and out
+    low_cut: Tuple[int, int, int]
+    mid_cut: Tuple[int, int, int]
+    r: int
+    b: int
+    s: int
+    R: int
+    m: int
+    router_hidden: int = 64
+    t_embed_dim: int = 64
+    seed: int = 0
+    timesteps: Tuple[float, ...] = (500.0,)
+    smooth_cosines: int = 0         # number of separable cosines added to every tensor
+    smooth_amplitude: float = 0.0
+
+    @property
+    def N(self) -> int:
+        return self.T * self.H * self.W
+
+    @property
+    def grid(self) -> Tuple[int, int, int]:
+        return (self.T, self.H, self.W)
+
+    def scaled(self, name: str, **kw) -> "FFConfig":
+        return replace(self, name=name, **kw)
+
+
+def _cuts(grid, c_low_num, c_low_den):
+    """L_a = n_a * c_low, M_a = n_a * (c_low + 1/2), both exact integers here."""
+    low = tuple(n * c_low_num // c_low_den for n in grid)
+    mid = tuple(n * c_low_num // c_low_den + n // 2 for n in grid)
+    return low, mid
+
+
+def _make(name, batch, grid, heads, d, dtype, c_low, r, b, s, R, m, seed, timesteps, **kw):
+    low, mid = _cuts(grid, *c_low)
+    return FFConfig(name=name, batch=batch, T=grid[0], H=grid[1], W=grid[2], heads=heads,
+                    head_dim=d, dtype=dtype, low_cut=low, mid_cut=mid, r=r, b=b, s=s, R=R, m=m,
+                    seed=seed, timesteps=tuple(float(t) for t in timesteps), **kw)
+
+
+# The five workloads of the benchmark definition, in its order.
+TINY = _make("tiny_fp32", 1, (4, 8, 8), 2, 32, "fp32", (1, 4), 4, 16, 4, 8, 4, 0, (500,))
+G64K = _make("64k", 1, (16, 64, 64), 24, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 1, (800,))
+G256K = _make("256k", 1, (64, 64, 64), 24, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 2, (200,),
+              smooth_cosines=8, smooth_amplitude=3.0)
+G1M = _make("1m", 1, (64, 128, 128), 16, 128, "bf16", (1, 16), 16, 128, 16, 512, 32, 3, (500,))
+G128K = _make("128k_sweep", 2, (32, 64, 64), 24, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 4,
+              (999, 750, 500, 250, 1))
+
+CONFIGS = (TINY, G64K, G256K, G1M, G128K)
+BY_NAME = {c.name: c for c in CONFIGS}
+
+# Scaled-down replicas (same operator parameters, grids of 4K-16K tokens, fewer heads) on which
+# the fp64 oracle can run every stage in full within seconds.
+R64K = _make("64k_replica", 1, (8, 32, 32), 6, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 11, (800,))
+R256K = _make("256k_replica", 1, (8, 32, 32), 6, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 12, (200,),
+              smooth_cosines=8, smooth_amplitude=3.0)
+R1M = _make("1m_replica", 1, (16, 32, 32), 4, 128, "bf16", (1, 16), 16, 128, 16, 512, 32, 13, (500,))
+R128K = _make("128k_replica", 2, (8, 32, 16), 6, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 14,
+              (999, 750, 500, 250, 1))
+
+REPLICAS = (R64K, R256K, R1M, R128K)
+BY_NAME.update({c.name: c for c in REPLICAS})

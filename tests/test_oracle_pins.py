@@ -1,0 +1,436 @@
+"""Pins for the fp64 oracle: each test checks it against something the paper or the
+mathematics fixes independently of the oracle's own code (closed forms, library
+routines, brute force written separately here, special cases that reduce to dense
+softmax attention, the values the paper prints)."""
+import itertools
+import math
+import os
+from types import SimpleNamespace
+
+import numpy as np
+import pytest
+import scipy.fft
+
+from oracle import freqformer_oracle as O
+from paper_2604_22808_b200 import configs as C
+from paper_2604_22808_b200 import inputs as I
+
+
+def _golden(golden_dir):
+    vals = {}
+    with open(os.path.join(golden_dir, "paper_constants.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                k, v = line.split()
+                vals[k] = float(v) if "." in v else int(v)
+    return vals
+
+
+def _cfg(T, H, W, d, low_cut, mid_cut, r=1, b=4, s=2, R=2, m=0, heads=1, d_t=8):
+    return SimpleNamespace(T=T, H=H, W=W, heads=heads, head_dim=d, low_cut=low_cut, mid_cut=mid_cut,
+                           r=r, b=b, s=s, R=R, m=m, t_embed_dim=d_t)
+
+
+def _loop_attention(Q, K, V, allowed):
+    """Dense-reference softmax attention written out with scalar loops (separate from the oracle)."""
+    n, d = Q.shape
+    out = np.zeros((n, d))
+    for i in range(n):
+        keys = [j for j in range(K.shape[0]) if allowed(i, j)]
+        sc = [sum(Q[i, c] * K[j, c] for c in range(d)) / math.sqrt(d) for j in keys]
+        mx = max(sc)
+        w = [math.exp(x - mx) for x in sc]
+        tot = sum(w)
+        for wj, j in zip(w, keys):
+            out[i] += (wj / tot) * V[j]
+    return out
+
+
+# ------------------------------------------------------------------ transform
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 8, 16, 64, 128])
+def test_dct_matrix_orthonormal(n):
+    Cn = O.dct_matrix(n)
+    assert np.abs(Cn @ Cn.T - np.eye(n)).max() < 1e-13
+    assert np.abs(Cn.T @ Cn - np.eye(n)).max() < 1e-13
+
+
+def test_dct_matrix_matches_library_dct2_ortho():
+    rng = np.random.default_rng(0)
+    for n in (4, 7, 16):
+        x = rng.standard_normal(n)
+        assert np.allclose(O.dct_matrix(n) @ x, scipy.fft.dct(x, type=2, norm="ortho"), atol=1e-13)
+
+
+def test_transform_matches_library_dctn_and_roundtrip_and_parseval():
+    rng = np.random.default_rng(1)
+    X = rng.standard_normal((4, 6, 5, 3))
+    Xt = O.forward_transform(X)
+    ref = scipy.fft.dctn(X, type=2, norm="ortho", axes=(0, 1, 2))
+    assert np.abs(Xt - ref).max() < 1e-12
+    assert np.abs(O.inverse_transform(Xt) - X).max() < 1e-12
+    # Parseval per channel ("Approximation Perspective").
+    assert np.allclose((Xt ** 2).sum(axis=(0, 1, 2)), (X ** 2).sum(axis=(0, 1, 2)), rtol=1e-12)
+
+
+def test_transform_brute_force_triple_sum():
+    rng = np.random.default_rng(2)
+    T, H, W, d = 2, 3, 4, 2
+    X = rng.standard_normal((T, H, W, d))
+    Xt = O.forward_transform(X)
+
+    def a(k, n):
+        return math.sqrt(1.0 / n) if k == 0 else math.sqrt(2.0 / n)
+
+    for kt, kh, kw, c in itertools.product(range(T), range(H), range(W), range(d)):
+        acc = 0.0
+        for t, h, w in itertools.product(range(T), range(H), range(W)):
+            acc += (a(kt, T) * math.cos(math.pi * (2 * t + 1) * kt / (2 * T))
+                    * a(kh, H) * math.cos(math.pi * (2 * h + 1) * kh / (2 * H))
+                    * a(kw, W) * math.cos(math.pi * (2 * w + 1) * kw / (2 * W)) * X[t, h, w, c])
+        assert abs(acc - Xt[kt, kh, kw, c]) < 1e-12
+
+
+def test_transform_closed_forms():
+    T, H, W = 4, 8, 8
+    N = T * H * W
+    Xt = O.forward_transform(np.full((T, H, W, 1), 2.5))
+    assert abs(Xt[0, 0, 0, 0] - 2.5 * math.sqrt(N)) < 1e-12
+    Xt[0, 0, 0, 0] = 0
+    assert np.abs(Xt).max() < 1e-12
+    # One DCT-aligned separable cosine -> one coefficient of known size.
+    a_, b_, c_ = 1, 3, 0
+    t = np.arange(T)[:, None, None]; h = np.arange(H)[None, :, None]; w = np.arange(W)[None, None, :]
+    X = (np.cos(np.pi * (2 * t + 1) * a_ / (2 * T)) * np.cos(np.pi * (2 * h + 1) * b_ / (2 * H))
+         * np.cos(np.pi * (2 * w + 1) * c_ / (2 * W)))[..., None]
+    Xt = O.forward_transform(X)
+    expect = math.sqrt(T / 2) * math.sqrt(H / 2) * math.sqrt(W)
+    assert abs(Xt[a_, b_, c_, 0] - expect) < 1e-12
+    Xt[a_, b_, c_, 0] = 0
+    assert np.abs(Xt).max() < 1e-12
+
+
+def test_smooth_component_of_inputs_lands_in_low_box_only():
+    cfg = C.R256K
+    x = I.qkv_head(cfg, I.TENSOR_V, 0, 1).astype(np.float64)
+    noise = C.R256K.scaled("n", smooth_cosines=0, smooth_amplitude=0.0)
+    # the smooth part is what remains after removing the same seed's pure-noise draw, up to bf16 rounding
+    comp = O.forward_transform(x - I.qkv_head(noise, I.TENSOR_V, 0, 1).astype(np.float64))
+    lab = O.band_labels(cfg.grid, cfg.low_cut, cfg.mid_cut)
+    assert np.abs(comp[lab == 0]).max() > 50.0
+    assert np.abs(comp[lab != 0]).max() < 1.0
+
+
+# ------------------------------------------------------------------ bands
+@pytest.mark.parametrize("cfg", C.CONFIGS + C.REPLICAS, ids=lambda c: c.name)
+def test_band_partition_sizes(cfg):
+    mem = O.band_members(cfg.grid, cfg.low_cut, cfg.mid_cut)
+    allidx = np.concatenate(mem)
+    assert len(allidx) == cfg.N and len(np.unique(allidx)) == cfg.N       # disjoint cover, sizes sum to N
+    L, M = cfg.low_cut, cfg.mid_cut
+    assert len(mem[0]) == L[0] * L[1] * L[2]
+    assert len(mem[1]) == M[0] * M[1] * M[2] - L[0] * L[1] * L[2]
+    assert len(mem[2]) == cfg.N - M[0] * M[1] * M[2]
+    for ix in mem:
+        assert np.all(np.diff(ix) > 0)
+
+
+def test_band_sizes_of_the_benchmark_workloads():
+    expect = {"tiny_fp32": (4, 104, 148), "64k": (128, 15872, 49536), "256k": (512, 63488, 198144),
+              "1m": (256, 186368, 861952), "128k_sweep": (256, 31744, 99072)}
+    for cfg in C.CONFIGS:
+        mem = O.band_members(cfg.grid, cfg.low_cut, cfg.mid_cut)
+        assert tuple(len(x) for x in mem) == expect[cfg.name]
+
+
+def test_band_labels_brute_force_nondivisible():
+    grid, L, M = (3, 5, 7), (1, 2, 3), (2, 4, 5)
+    lab = O.band_labels(grid, L, M)
+    for kt, kh, kw in itertools.product(*(range(n) for n in grid)):
+        k = (kt, kh, kw)
+        if all(k[a] < L[a] for a in range(3)):
+            e = 0
+        elif all(k[a] < M[a] for a in range(3)):
+            e = 1
+        else:
+            e = 2
+        assert lab[kt, kh, kw] == e
+
+
+# ------------------------------------------------------------------ low band
+def test_low_compression_group_means_and_broadcast():
+    x = np.arange(14, dtype=np.float64).reshape(7, 2)
+    c = O.compress_low(x, 3)
+    assert c.shape == (3, 2)
+    assert np.allclose(c[0], x[0:3].mean(0)) and np.allclose(c[2], x[6])
+    assert np.array_equal(O.compress_low(x, 1), x)
+    back = O.decompress_low(c, 3, 7)
+    assert np.allclose(back[[0, 1, 2]], c[0]) and np.allclose(back[6], c[2])
+
+
+def test_low_band_everything_r1_is_dense_attention_in_dct_domain():
+    rng = np.random.default_rng(3)
+    T, H, W, d = 2, 3, 2, 4
+    cfg = _cfg(T, H, W, d, (T, H, W), (T, H, W), r=1, m=0)
+    Q, K, V = (rng.standard_normal((1, T, H, W, d)) for _ in range(3))
+    res = O.forward_sample(cfg, Q, K, V, None, None, 0.0, alloc=[O.BAND_LOW])
+    qs, ks, vs = (scipy.fft.dctn(x[0], type=2, norm="ortho", axes=(0, 1, 2)).reshape(-1, d) for x in (Q, K, V))
+    y = _loop_attention(qs, ks, vs, lambda i, j: True)
+    ref = scipy.fft.idctn(y.reshape(T, H, W, d), type=2, norm="ortho", axes=(0, 1, 2))
+    assert np.abs(res["out"][0] - ref).max() < 1e-12
+    assert res["counters"]["pairs_low"] == (T * H * W) ** 2
+
+
+def test_low_band_single_compressed_token_returns_mean_value():
+    rng = np.random.default_rng(4)
+    cfg = _cfg(2, 4, 4, 3, (1, 2, 2), (2, 3, 3), r=4, m=0)
+    Q, K, V = (rng.standard_normal((1, 2, 4, 4, 3)) for _ in range(3))
+    res = O.forward_sample(cfg, Q, K, V, None, None, 0.0, alloc=[O.BAND_LOW], want_taps=True)
+    vlow = res["taps"]["Vb"][0][0]
+    assert res["taps"]["Y"][0][0].shape == (1, 3)
+    assert np.allclose(res["taps"]["Y"][0][0][0], vlow.mean(axis=0))
+
+
+# ------------------------------------------------------------------ mid band
+def test_mid_key_sets_brute_force():
+    for n, b, s in [(23, 4, 3), (16, 4, 2), (9, 16, 4), (30, 1, 5), (104, 16, 4)]:
+        nb = -(-n // b)
+        total = 0
+        for p in range(n):
+            expect = [q for q in range(n) if ((q // b) - (p // b)) % s == 0]
+            got = O.mid_keys(p, n, b, s)
+            assert list(got) == expect
+            assert all(q in expect for q in range((p // b) * b, min(n, (p // b + 1) * b)))  # own block
+            total += len(expect)
+        assert total == O.mid_interactions(n, b, s)
+        assert nb >= 1
+
+
+def test_mid_reduces_to_dense():
+    rng = np.random.default_rng(5)
+    n, d = 21, 5
+    Q, K, V = (rng.standard_normal((n, d)) for _ in range(3))
+    dense = _loop_attention(Q, K, V, lambda i, j: True)
+    y1, pairs = O.mid_operator(Q, K, V, b=4, s=1)             # stride 1: every block kept
+    assert np.abs(y1 - dense).max() < 1e-12 and pairs == n * n
+    y2, _ = O.mid_operator(Q, K, V, b=32, s=4)                # one block holds the whole band
+    assert np.abs(y2 - dense).max() < 1e-12
+    assert np.abs(O.dense_attention(Q, K, V) - dense).max() < 1e-12
+
+
+def test_mid_sparse_matches_loop_reference():
+    rng = np.random.default_rng(6)
+    n, d, b, s = 19, 3, 3, 2
+    Q, K, V = (rng.standard_normal((n, d)) for _ in range(3))
+    ref = _loop_attention(Q, K, V, lambda i, j: ((j // b) - (i // b)) % s == 0)
+    y, _ = O.mid_operator(Q, K, V, b, s)
+    assert np.abs(y - ref).max() < 1e-12
+    rows = np.array([0, 7, 18])
+    ysub, _ = O.mid_operator(Q, K, V, b, s, rows=rows)
+    assert np.abs(ysub - ref[rows]).max() < 1e-12
+
+
+# ------------------------------------------------------------------ high band
+def test_high_reduces_to_dense_and_identity():
+    rng = np.random.default_rng(7)
+    n, d = 17, 4
+    Q, K, V = (rng.standard_normal((n, d)) for _ in range(3))
+    dense = _loop_attention(Q, K, V, lambda i, j: True)
+    y, pairs = O.high_operator(Q, K, V, R=n)
+    assert np.abs(y - dense).max() < 1e-12 and pairs == n * n
+    y0, pairs0 = O.high_operator(Q, K, V, R=0)
+    assert np.abs(y0 - V).max() < 1e-14 and pairs0 == n
+    ref = _loop_attention(Q, K, V, lambda i, j: abs(i - j) <= 3)
+    y3, pairs3 = O.high_operator(Q, K, V, R=3)
+    assert np.abs(y3 - ref).max() < 1e-12
+    assert pairs3 == n * 7 - 3 * 4 == O.high_interactions(n, 3)
+
+
+def test_interaction_closed_forms():
+    for n, R in [(148, 8), (49536, 256), (1000, 0)]:
+        assert O.high_interactions(n, R) == n * (2 * R + 1) - R * (R + 1)
+    # blocks divide evenly -> every query sees exactly N_mid / s keys: I = N_mid * k_mid
+    assert O.mid_interactions(15872, 64, 8) == 15872 * 1984
+    assert O.mid_interactions(63488, 64, 8) == 63488 * 7936
+
+
+# ------------------------------------------------------------------ exchange / summaries
+def test_summary_segments_cover_and_repeat():
+    assert O.summary_segments(8, 4) == [(0, 2), (2, 4), (4, 6), (6, 8)]
+    assert O.summary_segments(1, 4) == [(0, 1)] * 4
+    segs = O.summary_segments(10, 4)
+    assert segs[0][0] == 0 and segs[-1][1] == 10
+    assert all(segs[i][1] == segs[i + 1][0] for i in range(3))
+
+
+def test_summary_tokens_and_exchange_properties():
+    rng = np.random.default_rng(8)
+    d, m = 4, 2
+    Y = rng.standard_normal((6, d))
+    S = O.summary_tokens(Y, np.eye(d), m)
+    assert np.allclose(S[0], Y[:3].mean(0)) and np.allclose(S[1], Y[3:].mean(0))
+    U = rng.standard_normal((d, d))
+    assert np.allclose(O.summary_tokens(Y, U, m)[1], U @ Y[3:].mean(0))
+    Z = rng.standard_normal((4, d))
+    dY = O.exchange(Y, Z) - Y
+    assert np.all(dY <= Z.max(0) + 1e-12) and np.all(dY >= Z.min(0) - 1e-12)   # convex combination of Z
+    assert np.abs(O.exchange(Y, np.zeros((4, d))) - Y).max() == 0                # U = 0 -> no change
+
+
+def test_hand_worked_three_token_layer():
+    """Grid 1x1x3, d=1, one coefficient per band, m=1, U=1: every band operator sees one key
+    (Y = V~), and the exchange of band l is a two-key softmax that can be written by hand."""
+    cfg = _cfg(1, 1, 3, 1, (1, 1, 1), (1, 1, 2), r=1, b=1, s=1, R=0, m=1)
+    v = np.array([1.0, -2.0, 0.5])
+    q = np.array([0.3, 0.1, -0.7]); k = np.array([0.2, -0.4, 0.9])
+    as6 = lambda x: x.reshape(1, 1, 1, 3, 1)
+    U = np.ones((3, 1, 1))
+    res = O.forward_sample(cfg, as6(q), as6(k), as6(v), None, U, 0.0, alloc=[7])
+    # hand DCT-II of three samples
+    c0 = (v[0] + v[1] + v[2]) / math.sqrt(3)
+    c1 = math.sqrt(2 / 3) * (math.cos(math.pi / 6) * v[0] + math.cos(3 * math.pi / 6) * v[1] + math.cos(5 * math.pi / 6) * v[2])
+    c2 = math.sqrt(2 / 3) * (math.cos(2 * math.pi / 6) * v[0] + math.cos(6 * math.pi / 6) * v[1] + math.cos(10 * math.pi / 6) * v[2])
+    y = [c0, c1, c2]
+    yh = []
+    for l in range(3):
+        a, b_ = [y[o] for o in range(3) if o != l]
+        wa, wb = math.exp(y[l] * a), math.exp(y[l] * b_)
+        yh.append(y[l] + (wa * a + wb * b_) / (wa + wb))
+    out = [sum((math.sqrt(1 / 3) if kk == 0 else math.sqrt(2 / 3)) * math.cos(math.pi * (2 * i + 1) * kk / 6) * yh[kk]
+               for kk in range(3)) for i in range(3)]
+    assert np.allclose(res["out"].reshape(-1), out, atol=1e-13)
+    assert res["counters"]["pairs_exchange"] == 6
+
+
+# ------------------------------------------------------------------ whole pipeline
+def test_empty_mask_no_exchange_returns_v():
+    rng = np.random.default_rng(9)
+    cfg = C.TINY.scaled("t", m=0)
+    Q, K, V = (rng.standard_normal((2, 4, 8, 8, 32)) for _ in range(3))
+    res = O.forward_sample(cfg, Q, K, V, None, None, 0.0, alloc=[0, 0])
+    assert np.abs(res["out"] - V).max() < 1e-12
+
+
+def test_outputs_stay_in_value_hull_and_heads_are_independent():
+    rng = np.random.default_rng(10)
+    cfg = C.TINY.scaled("t", m=0)
+    Q, K, V = (rng.standard_normal((2, 4, 8, 8, 32)) for _ in range(3))
+    res = O.forward_sample(cfg, Q, K, V, None, None, 0.0, alloc=[7, 7], want_taps=True)
+    for h in range(2):
+        for l in range(3):
+            vb = res["taps"]["Vb"][h][l]
+            if l == 0:
+                vb = O.compress_low(vb, cfg.r)
+            y = res["taps"]["Y"][h][l]
+            assert np.all(y <= vb.max(0) + 1e-12) and np.all(y >= vb.min(0) - 1e-12)
+    swapped = O.forward_sample(cfg, Q[::-1], K[::-1], V[::-1], None, None, 0.0, alloc=[7, 7])
+    assert np.abs(swapped["out"][::-1] - res["out"]).max() < 1e-13
+
+
+def test_error_decomposition_over_bands():
+    """||Y_full - Y_freq||^2 = sum over bands of ||P_band F(Y_full - Y_freq)||^2."""
+    rng = np.random.default_rng(11)
+    cfg = C.TINY
+    Q, K, V = (rng.standard_normal((1, 4, 8, 8, 32)) for _ in range(3))
+    U = I.summary_projection(cfg)
+    yfreq = O.forward_sample(cfg, Q, K, V, None, U, 0.0, alloc=[7])["out"][0]
+    flat = lambda x: x.reshape(-1, 32)
+    yfull = O.dense_attention(flat(Q[0]), flat(K[0]), flat(V[0])).reshape(4, 8, 8, 32)
+    diff = yfull - yfreq
+    mem = O.band_members(cfg.grid, cfg.low_cut, cfg.mid_cut)
+    parts = [np.sum(x ** 2) for x in O.split_bands(O.forward_transform(diff), mem)]
+    assert math.isclose(sum(parts), np.sum(diff ** 2), rel_tol=1e-12)
+
+
+# ------------------------------------------------------------------ router
+def test_router_counts_from_paper(golden_dir):
+    g = _golden(golden_dir)
+    assert O.router_parameter_count(256, 128, 3) == g["router_params_256_128_3"]
+    assert O.router_flops(256, 128, 3) == g["router_flops_256_128_3"]
+
+
+def test_timestep_embedding_closed_forms():
+    e = O.timestep_embedding(0.0, 8)
+    assert np.allclose(e[:4], 0) and np.allclose(e[4:], 1)
+    e = O.timestep_embedding(500.0, 64)
+    assert math.isclose(e[0], math.sin(500.0)) and math.isclose(e[32], math.cos(500.0))
+    assert math.isclose(e[16], math.sin(500.0 * 10000 ** -0.5))
+    assert np.allclose(e[:32] ** 2 + e[32:] ** 2, 1.0)
+
+
+def test_router_hand_example():
+    # two hidden units, inputs g=[1,2,3] (d_r = 1) and e=[0.5, -1]
+    W1 = np.array([[1.0, 0, 0, 1, 0], [0, -1.0, 0, 0, 1]]); b1 = np.array([0.5, 0.0])
+    W2 = np.array([[1.0, 0], [0, 1.0], [1.0, 1.0]]); b2 = np.array([0.0, 0.1, -0.1])
+    pi, z = O.router_probabilities(np.array([1.0, 2, 3]), np.array([0.5, -1.0]), W1, b1, W2, b2)
+    h = [max(0.0, 1 + 0.5 + 0.5), max(0.0, -2 - 1)]                  # [2.0, 0.0]
+    ze = [h[0], h[1] + 0.1, h[0] + h[1] - 0.1]
+    den = sum(math.exp(v) for v in ze)
+    assert np.allclose(z, ze) and np.allclose(pi, [math.exp(v) / den for v in ze])
+    assert math.isclose(pi.sum(), 1.0)
+
+
+def test_pooled_statistics_definition():
+    es = np.array([[2.0, 4.0], [6.0, 0.0], [1.0, 1.0]])
+    g = O.pooled_statistics(es, [2, 3, 1])
+    assert np.allclose(g, [math.log(2), math.log(3), math.log(3), 0.0, math.log(2), math.log(2)])
+
+
+def test_head_quota_largest_remainder():
+    counts, _ = O.head_quota(np.array([0.5, 0.3, 0.2]), 24)
+    assert list(counts) == [12, 7, 5] and counts.sum() == 24
+    counts, _ = O.head_quota(np.array([0.26, 0.26, 0.48]), 2)      # q = .52 .52 .96 -> high, then tie -> low
+    assert list(counts) == [1, 0, 1]
+    counts, _ = O.head_quota(np.array([1.0, 0.0, 0.0]), 16)
+    assert list(counts) == [16, 0, 0]
+    rng = np.random.default_rng(12)
+    for _ in range(200):
+        p = rng.dirichlet([1, 1, 1])
+        n = int(rng.integers(1, 40))
+        c, _ = O.head_quota(p, n)
+        assert c.sum() == n and np.all(np.abs(c - p * n) < 1.0 + 1e-6)
+    assert list(O.head_allocation([2, 1, 3])) == [1, 1, 2, 4, 4, 4]
+
+
+# ------------------------------------------------------------------ cost model
+def test_cost_model_against_paper(golden_dir):
+    g = _golden(golden_dir)
+    for N in (65536, 131072, 262144, 524288, 1048576):
+        assert O.dense_attention_flops(N, 64) == g[f"dense_flops_{N}"]
+        closed = g["closed_form_quadratic_coeff"] * N * N * 64 + g["closed_form_linear_coeff"] * N * 64
+        assert math.isclose(O.paper_attention_cost_reference(N, 64), closed, rel_tol=1e-15)
+    assert 2 * 65536 ** 2 == g["dense_traffic_65536"] and 2 * 1048576 ** 2 == g["dense_traffic_1048576"]
+
+
+def test_counters_match_cost_formula():
+    """The pairs the oracle actually scores equal N_low_bar^2 + N_mid k_mid + N_high w with the
+    boundary-clipped window (w exact for interior rows), and transform MACs are N(T+H+W)d per tensor."""
+    rng = np.random.default_rng(13)
+    cfg = C.TINY
+    Q, K, V = (rng.standard_normal((2, 4, 8, 8, 32)) for _ in range(3))
+    res = O.forward_sample(cfg, Q, K, V, None, I.summary_projection(cfg), 0.0, alloc=[7, 7])
+    c = res["counters"]
+    n_low, n_mid, n_high = res["sizes"]
+    n_low_bar = -(-n_low // cfg.r)
+    assert c["pairs_low"] == 2 * n_low_bar ** 2
+    assert c["pairs_mid"] == 2 * O.mid_interactions(n_mid, cfg.b, cfg.s)
+    assert c["pairs_high"] == 2 * (n_high * (2 * cfg.R + 1) - cfg.R * (cfg.R + 1))
+    assert c["pairs_exchange"] == 2 * (2 * cfg.m) * (n_low_bar + n_mid + n_high)
+    assert c["transform_macs"] == 2 * 4 * cfg.N * (4 + 8 + 8) * 32
+    total = c["pairs_low"] + c["pairs_mid"] + c["pairs_high"]
+    k_mid = O.mid_interactions(n_mid, cfg.b, cfg.s) / n_mid
+    w_bar = O.high_interactions(n_high, cfg.R) / n_high
+    assert math.isclose(total, 2 * O.paper_interactions(n_low_bar, n_mid, k_mid, n_high, w_bar), rel_tol=1e-12)
+
+
+def test_router_allocation_path_runs_and_is_consistent():
+    cfg = C.TINY
+    Q, K, V = (np.stack([I.qkv_head(cfg, t, 0, h) for h in range(cfg.heads)]) for t in range(3))
+    res = O.forward_sample(cfg, Q, K, V, I.router_weights(cfg), I.summary_projection(cfg), cfg.timesteps[0])
+    assert math.isclose(res["pi"].sum(), 1.0, rel_tol=1e-12)
+    assert len(res["alloc"]) == cfg.heads and set(res["alloc"]) <= {1, 2, 4}
+    # statistics: by Parseval the three band energies add up to the token-domain energy
+    E = np.expm1(res["g"]).reshape(3, -1)
+    sizes = np.array(res["sizes"])[:, None]
+    tok = sum((x.astype(np.float64) ** 2).sum(axis=(0, 1, 2, 3)) for x in (Q, K, V))
+    assert np.allclose((E * sizes * 3 * cfg.heads).sum(0), tok, rtol=1e-10)
