@@ -1,0 +1,337 @@
+"""Benchmark of the FreqFormer attention forward on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 64k|256k|1m|128k_sweep]
+  python bench.py --impl reference ...        # the fp64 oracle timed on the host cores
+
+A step is one ff_forward (transform, band split, router, three band operators, summary
+exchange, recombination, inverse transform) over one batch of the synthetic workload.  With
+N > 1 (torchrun) every rank runs its own replica of the batch: samples are independent problems,
+so there is no data-path collective and the scaling is weak.  One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2604_22808_b200 import configs as C          # noqa: E402
+from paper_2604_22808_b200 import inputs as I           # noqa: E402
+
+METRIC = "freqformer_attn_layer_tokens_per_s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------------------------
+# Work model of one layer (per workload, given the head allocation)
+# ---------------------------------------------------------------------------------------------
+def band_sizes(cfg):
+    L, M = cfg.low_cut, cfg.mid_cut
+    n_low = L[0] * L[1] * L[2]
+    n_mid = M[0] * M[1] * M[2] - n_low
+    return n_low, -(-n_low // cfg.r), n_mid, cfg.N - M[0] * M[1] * M[2]
+
+
+def interactions(cfg):
+    """Scored (query, key) pairs of one head per band operator, and of the exchange."""
+    n_low, n_bar, n_mid, n_high = band_sizes(cfg)
+    nb = -(-n_mid // cfg.b)
+    i_mid = 0
+    for c in range(min(cfg.s, nb)):
+        n_c = sum(min(cfg.b, n_mid - J * cfg.b) for J in range(c, nb, cfg.s))
+        i_mid += n_c * n_c
+    R = min(cfg.R, n_high - 1)
+    i_high = n_high * (2 * R + 1) - R * (R + 1)
+    return n_bar * n_bar, i_mid, i_high
+
+
+def layer_work(cfg, alloc):
+    """Useful attention FLOPs (4 d per pair: QK^T and PV) and algorithmic HBM bytes of one forward."""
+    d, e = cfg.head_dim, (4 if cfg.dtype == "fp32" else 2)
+    n_low, n_bar, n_mid, n_high = band_sizes(cfg)
+    pairs = interactions(cfg)
+    u = cfg.N * d * e
+    flops = 0
+    bytes_attn = 0
+    for mask in alloc:
+        for l, (p, n_l) in enumerate(zip(pairs, (n_bar, n_mid, n_high))):
+            if mask >> l & 1:
+                flops += 4 * d * p
+                bytes_attn += 4 * n_l * d * e
+    heads = len(alloc)
+    exch_pairs = heads * 2 * cfg.m * cfg.N
+    return {
+        "attn_flops": flops,
+        "exchange_flops": 4 * d * exch_pairs,
+        "transform_flops": heads * 4 * 2 * cfg.N * (cfg.T + cfg.H + cfg.W) * d,
+        # forward transform: read Q,K,V, write Q~,K~,V~; inverse: read Y^, write out
+        "bytes_transform": heads * 6 * u,
+        "bytes_inverse": heads * 2 * u,
+        "bytes_attention": bytes_attn,
+    }
+
+
+# ---------------------------------------------------------------------------------------------
+# Clock sampling during the timed region
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _loop(self):
+        while not self._stop.is_set():
+            try:
+                self.samples.append(self._nv.nvmlDeviceGetClockInfo(self._h, self._nv.NVML_CLOCK_SM))
+                mask = self._nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.05)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU baseline: the oracle, as it stands, on a bounded sample
+# ---------------------------------------------------------------------------------------------
+def oracle_sample_time(cfg, alloc):
+    """Times the oracle's whole layer for one head per band type present in `alloc` on the full
+    grid (transform of Q,K,V, that band's operator over every row, summaries, exchange, inverse)
+    and extrapolates to all heads by the allocation.  Returns (tokens/s, seconds, cores, text)."""
+    from threadpoolctl import threadpool_info
+    from oracle import freqformer_oracle as O
+    weights = I.router_weights(cfg)
+    U = I.summary_projection(cfg)
+    per_band = {}
+    spent = 0.0
+    for l, bit in enumerate((1, 2, 4)):
+        heads_l = [h for h, mk in enumerate(alloc) if mk == bit]
+        if not heads_l:
+            continue
+        h = heads_l[0]
+        Q, K, V = (I.qkv_head(cfg, t, 0, h)[None] for t in range(3))
+        t0 = time.perf_counter()
+        O.forward_sample(cfg, Q, K, V, weights, U, cfg.timesteps[0], alloc=[bit])
+        per_band[bit] = time.perf_counter() - t0
+        spent += per_band[bit]
+    total = sum(per_band.get(mk, max(per_band.values())) for mk in alloc) * (cfg.batch)
+    cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    text = (f"one head per allocated band type ({len(per_band)} of {len(alloc)} heads) on the full {cfg.name} grid, "
+            f"whole layer each, extrapolated by the head allocation")
+    return cfg.batch * cfg.N / total, spent, cores, text
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n = cfg.heads
+    alloc = [1] * (n // 3) + [2] * (n // 3) + [4] * (n - 2 * (n // 3))
+    vals = []
+    t_all = time.perf_counter()
+    for i in range(args.warmup + args.steps):
+        if i > 0 and time.perf_counter() - t_all > 240:
+            break
+        v, spent, cores, text = oracle_sample_time(cfg, alloc)
+        if i >= args.warmup or i == args.warmup + args.steps - 1:
+            vals.append(v)
+    value = float(np.mean(vals))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": len(vals), "warmup": args.warmup, "ms_per_step": 1e3 * cfg.batch * cfg.N / value,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "grid": list(cfg.grid), "heads": cfg.heads, "head_dim": cfg.head_dim,
+                       "allocation": "even split low/mid/high"},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": text},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+# The CUDA arm
+# ---------------------------------------------------------------------------------------------
+def run_cuda(args, cfg):
+    import torch
+    import torch.distributed as dist
+    from paper_2604_22808_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    dt = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
+    cfg_r = cfg.scaled(cfg.name, seed=cfg.seed + 1000 * rank) if rank else cfg       # each rank its own replica
+    host = [torch.from_numpy(I.qkv_full(cfg_r, t)).to(dt).pin_memory() for t in range(3)]
+    q, k, v = (x.to(dev, non_blocking=True) for x in host)
+    out = torch.empty_like(q)
+    out_host = torch.empty_like(host[0]).pin_memory()
+    weights = I.router_weights(cfg)
+    plan = B.Plan(cfg, weights, host_staging=True, device=dev)
+    plan.set_profiling(True)
+    ts = [cfg.timesteps[args.timestep_index]] * cfg.batch
+    torch.cuda.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def reduce_max(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # device-resident timing
+    for _ in range(args.warmup):
+        plan.forward(q, k, v, out, timesteps=ts)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    stage_ms = {name: 0.0 for name in B.STAGES}
+    stage_launches = {}
+    ev[0].record()
+    for i in range(args.steps):
+        plan.forward(q, k, v, out, timesteps=ts)
+        ev[i + 1].record()
+        for name, (ms, n) in plan.stage_times().items():       # waits for this step's last event
+            stage_ms[name] += ms / args.steps
+            stage_launches[name] = n
+    barrier()
+    clocks = sampler.stop()
+    ms_step = reduce_max(ev[0].elapsed_time(ev[-1]) / args.steps)
+    launches = plan.last_launches()
+    assert plan.device_status() == 0
+    alloc = plan.tap(B.TAP_ALLOC).cpu().numpy().tolist()
+    pi = plan.tap(B.TAP_PI).cpu().numpy().tolist()
+
+    # end to end through the host-buffer entry point (pinned host memory, copies inside the call)
+    for _ in range(min(2, args.warmup)):
+        plan.forward_host(host[0], host[1], host[2], out_host, timesteps=ts)
+    barrier()
+    e2e_steps = max(1, min(args.steps, 5))
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        plan.forward_host(host[0], host[1], host[2], out_host, timesteps=ts)      # synchronises the stream
+    e2e_ms = reduce_max((time.perf_counter() - t0) * 1e3 / e2e_steps)
+    barrier()
+
+    if rank == 0:
+        peaks = measured_peaks()
+        tokens = cfg.batch * cfg.N * world
+        work = layer_work(cfg, alloc)
+        # roofline of the dominant stage
+        top = max(stage_ms, key=stage_ms.get)
+        if top == "attention":
+            achieved = work["attn_flops"] / (stage_ms[top] * 1e-3) / 1e12
+            roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                    "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None}
+        else:
+            nbytes = work["bytes_transform"] if top == "transform" else work["bytes_inverse"]
+            achieved = nbytes / (stage_ms[top] * 1e-3) / 1e9
+            roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": None}
+        roof.update({"kernel": top, "launches_per_step": stage_launches.get(top), "ms_per_step": stage_ms[top],
+                     "peak_source": peaks["source"]})
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            v_cpu, spent, cores, text = oracle_sample_time(cfg, alloc)
+            cpu = {"value": v_cpu, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": text,
+                   "seconds": spent}
+        io_bytes = q.numel() * q.element_size()
+        line = {
+            "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": cfg.name, "grid": list(cfg.grid), "batch": cfg.batch, "heads": cfg.heads,
+                       "head_dim": cfg.head_dim, "timestep": ts[0], "allocation": "router",
+                       "heads_per_band": [alloc.count(1), alloc.count(2), alloc.count(4)], "pi": pi[0],
+                       "l2": "inputs (%.0f MB) larger than L2" % (3 * io_bytes / 1e6)},
+            "roofline": roof,
+            "cpu_baseline": cpu,
+            "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 3 * io_bytes,
+                    "d2h_bytes_per_step": io_bytes, "ms_per_step": e2e_ms},
+            "gpu_launches": launches * args.steps,
+            "clocks": clocks,
+            "stages_ms": stage_ms,
+            "useful_attention_tflops": work["attn_flops"] / (ms_step * 1e-3) / 1e12,
+            "attention_stage_tflops": work["attn_flops"] / (max(stage_ms["attention"], 1e-9) * 1e-3) / 1e12,
+            "transform_stage_gbs": work["bytes_transform"] / (max(stage_ms["transform"], 1e-9) * 1e-3) / 1e9,
+            "inverse_stage_gbs": work["bytes_inverse"] / (max(stage_ms["inverse"], 1e-9) * 1e-3) / 1e9,
+            "paper_context": "simulated estimates only: 9.3-27.3x attention-FLOP and 8.8-20.9x score-traffic reduction vs dense",
+        }
+        print(json.dumps(line))
+    plan.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="64k")
+    ap.add_argument("--timestep-index", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    cfg = C.BY_NAME[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        args.warmup = max(args.warmup, 3)
+        run_cuda(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

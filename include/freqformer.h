@@ -1,0 +1,208 @@
+/*
+ * freqformer.h -- C ABI of the B200 (sm_100a) FreqFormer heterogeneous attention forward.
+ *
+ * One layer's attention forward over a T x H x W token grid, per head
+ * (paper: Method, "Setup and notation" .. "Reconstruction"):
+ *
+ *   Q,K,V --separable orthonormal DCT-II along t/h/w--> spectral coefficients
+ *         --split into low / mid / high bands (band-major token lists)
+ *         --router: pooled band statistics + timestep embedding -> pi -> heads per band
+ *         --low: dense attention on r:1 pooled tokens; mid: strided block-sparse attention;
+ *           high: sliding-window attention; bands a head is not allocated to pass V~ through
+ *         --m summary tokens per band, cross-band exchange (every token attends the 2m
+ *           summaries of the other two bands, residual add)
+ *         --recombination in the spectral domain, inverse transform --> out
+ *
+ * Conventions
+ *   - All functions return an ff_status_t (int32_t); none throws, aborts or exits.
+ *   - "device" pointers are CUDA device pointers on the device that was current at
+ *     ff_plan_create; "host" pointers are ordinary host memory.
+ *   - Q, K, V, out: device, contiguous [batch][heads][T][H][W][head_dim], element type
+ *     cfg.dtype (bf16 or fp32).  out has the layout and type of the inputs.  The caller owns
+ *     them; the library neither keeps nor frees them.
+ *   - The caller also owns the workspace (ff_plan_set_workspace); the plan owns only small
+ *     device tables (transform matrices, router weights, summary projections), freed by
+ *     ff_destroy.
+ *   - Calls are asynchronous on the given CUDA stream (a cudaStream_t passed as void*; NULL =
+ *     the legacy default stream) unless a host output pointer is requested, which makes the
+ *     call synchronise the stream before it returns.
+ *   - A plan is not thread-safe; distinct plans are independent.
+ */
+#ifndef FREQFORMER_H_
+#define FREQFORMER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ff_plan ff_plan_t; /* opaque */
+
+typedef int32_t ff_status_t;
+enum {
+  FF_OK = 0,
+  FF_ERR_INVALID_ARG = 1, /* NULL pointer, non-positive size, cut-offs out of order, bad mask ... */
+  FF_ERR_UNSUPPORTED = 2, /* head_dim / axis length / parameter outside what the kernels cover */
+  FF_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small */
+  FF_ERR_CUDA = 4,        /* a CUDA runtime call failed; ff_last_error has its message */
+  FF_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (read back at the next sync) */
+  FF_ERR_EMPTY_BAND = 6,  /* the cut-offs leave a band without coefficients */
+  FF_ERR_NOT_ROUTED = 7   /* ff_forward without allocation and without timestep */
+};
+
+enum { FF_BF16 = 0, FF_FP32 = 1 };
+
+/* Band-mask bits of one head.  The router emits one-hot masks; callers may pass any subset,
+ * LOW|MID|HIGH being the paper's formal per-head definition (every head runs all three
+ * operators, "Reconstruction" / "Per-layer complexity"). */
+enum { FF_BAND_LOW = 1, FF_BAND_MID = 2, FF_BAND_HIGH = 4 };
+
+/* Problem statement ("Setup and notation", "Frequency band partitioning",
+ * "Hierarchical frequency-domain attention", "Cross-band residual exchange"). */
+typedef struct {
+  int32_t batch, T, H, W, heads, head_dim; /* head_dim: multiple of 32, <= 128; axes <= 128 */
+  int32_t dtype;                           /* FF_BF16 or FF_FP32: Q, K, V and out */
+  int32_t low_cut[3];      /* L_a (t,h,w): coefficient k is LOW iff k_a < L_a on all axes */
+  int32_t mid_cut[3];      /* M_a: MID iff not LOW and k_a < M_a on all axes; L_a <= M_a <= n_a */
+  int32_t low_compress;    /* r >= 1: low-band tokens are mean-pooled r:1 before attention */
+  int32_t mid_block;       /* b >= 1: mid-band block size (consecutive band ranks) */
+  int32_t mid_stride;      /* s >= 1: a query block sees key blocks at block distance = 0 mod s */
+  int32_t high_radius;     /* R >= 0: high-band window |p - p'| <= R in band order */
+  int32_t n_summary;       /* m >= 0 summary tokens per band; 0 disables the exchange */
+  int32_t router_hidden;   /* hidden width of the two-layer router MLP */
+  int32_t t_embed_dim;     /* d_t, even: width of the sinusoidal timestep embedding */
+} ff_config_t;
+
+/* Host arrays, copied at ff_plan_create.  Router input is [g_low; g_mid; g_high; e(t)]
+ * (3*head_dim + t_embed_dim values).  NULL router pointers => ff_route / internal routing
+ * return FF_ERR_NOT_ROUTED.  U == NULL => identity summary projections. */
+typedef struct {
+  const float *W1; /* [router_hidden][3*head_dim + t_embed_dim], row-major */
+  const float *b1; /* [router_hidden] */
+  const float *W2; /* [3][router_hidden] */
+  const float *b2; /* [3] */
+  const float *U;  /* [3][head_dim][head_dim]: S = U_l * Pool(Y^(l)) */
+} ff_weights_t;
+
+/* ---- host-only helpers (no GPU needed) --------------------------------------------------- */
+
+/* Validate a configuration.  FF_OK, FF_ERR_INVALID_ARG, FF_ERR_UNSUPPORTED or FF_ERR_EMPTY_BAND. */
+ff_status_t ff_config_validate(const ff_config_t *cfg);
+
+/* Band sizes: sizes[0..3] = N_low, ceil(N_low / r), N_mid, N_high
+ * ("Frequency band partitioning": N_low + N_mid + N_high = N). */
+ff_status_t ff_band_sizes(const ff_config_t *cfg, int64_t sizes[4]);
+
+/* Band (0 low, 1 mid, 2 high) and band-local rank of coefficient (k_t, k_h, k_w); the rank is
+ * the coefficient's position in its band when the band is listed in increasing flat index
+ * (k_t*H + k_h)*W + k_w.  This closed form is what the kernels evaluate in registers. */
+ff_status_t ff_band_rank(const ff_config_t *cfg, int32_t kt, int32_t kh, int32_t kw,
+                         int32_t *band, int64_t *rank);
+
+/* Workspace size a plan of this configuration needs (device bytes, 256-byte aligned base). */
+ff_status_t ff_workspace_bytes(const ff_config_t *cfg, size_t *bytes);
+
+/* ---- plan lifetime ------------------------------------------------------------------------ */
+
+/* Build a plan on the current CUDA device: validates cfg, computes the DCT-II matrices
+ * ("Separable spectral decomposition") in double precision on the host and uploads them with
+ * the weights.  No kernel runs.  *out_plan is NULL on failure. */
+ff_status_t ff_plan_create(const ff_config_t *cfg, const ff_weights_t *weights, ff_plan_t **out_plan);
+
+ff_status_t ff_plan_workspace_bytes(const ff_plan_t *plan, size_t *bytes);
+
+/* Hand the plan its workspace (device memory owned by the caller, >= the size above, base
+ * aligned to 256 bytes).  Must precede ff_route / ff_forward; may be called again. */
+ff_status_t ff_plan_set_workspace(ff_plan_t *plan, void *dev_ptr, size_t bytes);
+
+/* Frees the plan's device tables and the plan.  NULL is allowed. */
+ff_status_t ff_destroy(ff_plan_t *plan);
+
+/* Message of the last failing call on this plan ("" if none); with plan == NULL, of the last
+ * failing plan-less call of the calling thread.  Owned by the library. */
+const char *ff_last_error(const ff_plan_t *plan);
+
+/* ---- the path -------------------------------------------------------------------------------- */
+
+/* Spectral routing network ("Spectral routing network"): forward transform of Q, K, V, pooled
+ * band statistics g, timestep embedding e(t), z = MLP([g; e(t)]), pi = softmax(z), largest-
+ * remainder head quota, heads [0,n_low) -> LOW, next n_mid -> MID, rest -> HIGH.
+ *   timestep    host, [batch]: raw diffusion step per sample
+ *   alloc_dev   device, [batch*heads] band masks written by the router; may be NULL
+ *   alloc_host  host,   [batch*heads]; non-NULL forces a stream synchronisation
+ *   pi_host     host,   [batch*3]; non-NULL forces a stream synchronisation
+ * The transformed Q~, K~, V~ stay in the workspace; an ff_forward on the same inputs recomputes
+ * them (the two calls are independent). */
+ff_status_t ff_route(ff_plan_t *plan, const void *Q, const void *K, const void *V,
+                     const float *timestep, uint8_t *alloc_dev, uint8_t *alloc_host,
+                     float *pi_host, void *cuda_stream);
+
+/* The attention forward ("Separable spectral decomposition" .. "Reconstruction").
+ *   alloc_dev   device, [batch*heads] band masks (any subset of LOW|MID|HIGH per head), or
+ *               NULL to route internally from `timestep` (host, [batch]) as ff_route does
+ *   out         device, same shape and type as Q
+ * Errors found on the host are returned at once; a device-side FF_ERR_TIMEOUT is reported by
+ * ff_plan_device_status after a synchronisation. */
+ff_status_t ff_forward(ff_plan_t *plan, const void *Q, const void *K, const void *V,
+                       const uint8_t *alloc_dev, const float *timestep, void *out,
+                       void *cuda_stream);
+
+/* Same computation with HOST buffers: copies Q, K, V host->device into staging space inside the
+ * workspace, runs ff_forward, copies out device->host, all on `cuda_stream`, then synchronises.
+ * The workspace must have been sized with ff_workspace_bytes_host.  alloc_host may be NULL
+ * (route internally); pinned host memory makes the copies asynchronous. */
+ff_status_t ff_forward_host(ff_plan_t *plan, const void *Q_host, const void *K_host,
+                            const void *V_host, const uint8_t *alloc_host, const float *timestep,
+                            void *out_host, void *cuda_stream);
+ff_status_t ff_workspace_bytes_host(const ff_config_t *cfg, size_t *bytes);
+
+/* Synchronises the stream and returns the device status word (FF_OK or FF_ERR_TIMEOUT), then
+ * clears it. */
+ff_status_t ff_plan_device_status(ff_plan_t *plan, void *cuda_stream);
+
+/* Number of kernel launches the last ff_forward / ff_route on this plan issued. */
+ff_status_t ff_plan_last_launches(const ff_plan_t *plan, int64_t *launches);
+
+/* Stage timing for benchmarks.  With profiling enabled, ff_forward records CUDA events on its
+ * stream at the stage boundaries; ff_plan_stage_times waits for the last one and returns the
+ * device time (ms) and the number of kernel launches of each stage of the last ff_forward:
+ *   TRANSFORM  forward transform + band split          ROUTER   band statistics + router MLP
+ *   ATTENTION  low pooling + the three band operators  SUMMARY  summary tokens
+ *   INVERSE    exchange + recombination + inverse transform */
+enum { FF_STAGE_TRANSFORM = 0, FF_STAGE_ROUTER = 1, FF_STAGE_ATTENTION = 2, FF_STAGE_SUMMARY = 3,
+       FF_STAGE_INVERSE = 4, FF_STAGE_COUNT = 5 };
+ff_status_t ff_plan_set_profiling(ff_plan_t *plan, int32_t enable);
+ff_status_t ff_plan_stage_times(ff_plan_t *plan, float ms[FF_STAGE_COUNT], int64_t launches[FF_STAGE_COUNT]);
+
+/* ---- inspection (tests) --------------------------------------------------------------------- */
+
+/* Intermediate buffers inside the workspace after the last call.  st = cfg.dtype, BH = batch*heads.
+ *   FF_TAP_SPEC_LOW   float  [3 (Q,K,V)][BH][N_low][d]      low-band coefficients
+ *   FF_TAP_SPEC_MID   st     [3][BH][N_mid][d]
+ *   FF_TAP_SPEC_HIGH  st     [3][BH][N_high][d]
+ *   FF_TAP_POOLED_LOW float  [3][BH][ceil(N_low/r)][d]      pooled low-band tokens
+ *   FF_TAP_Y_LOW      float  [BH][ceil(N_low/r)][d]         low operator output (executed heads)
+ *   FF_TAP_Y_MID      st     [BH][N_mid][d]                 mid operator output (executed heads)
+ *   FF_TAP_Y_HIGH     st     [BH][N_high][d]
+ *   FF_TAP_SUMMARY    float  [BH][3][m][d]                  summary tokens S
+ *   FF_TAP_ENERGY     double [batch][3][d]                  pooled sums of squared coefficients
+ *   FF_TAP_ALLOC      uint8  [BH]                           masks used by the last forward
+ *   FF_TAP_PI         float  [batch][3]
+ */
+enum {
+  FF_TAP_SPEC_LOW = 0, FF_TAP_SPEC_MID = 1, FF_TAP_SPEC_HIGH = 2, FF_TAP_POOLED_LOW = 3,
+  FF_TAP_Y_LOW = 4, FF_TAP_Y_MID = 5, FF_TAP_Y_HIGH = 6, FF_TAP_SUMMARY = 7, FF_TAP_ENERGY = 8,
+  FF_TAP_ALLOC = 9, FF_TAP_PI = 10, FF_TAP_COUNT = 11
+};
+ff_status_t ff_get_tap(const ff_plan_t *plan, int32_t which, const void **dev_ptr, size_t *bytes);
+
+/* Selects the attention implementation: 0 = automatic (tensor-core kernel where it applies),
+ * 1 = force the generic SIMT kernel.  For tests. */
+ff_status_t ff_plan_set_attention_impl(ff_plan_t *plan, int32_t impl);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FREQFORMER_H_ */

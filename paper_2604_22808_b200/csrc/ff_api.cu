@@ -1,0 +1,413 @@
+// Host side of the C ABI: configuration checks, band arithmetic, workspace layout, plan lifetime
+// and the launch sequence of the forward.  No device code lives here.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "ff_internal.h"
+
+static thread_local char g_err[512] = "";
+
+static ff_status_t fail(ff_plan* p, ff_status_t code, const char* fmt, const char* a = "", long long x = 0,
+                        long long y = 0) {
+  char* dst = p ? p->err : g_err;
+  snprintf(dst, 512, fmt, a, x, y);
+  return code;
+}
+
+#define FF_CUDA(p, call)                                                                        \
+  do {                                                                                          \
+    cudaError_t e__ = (call);                                                                   \
+    if (e__ != cudaSuccess) return fail((p), FF_ERR_CUDA, "CUDA error: %s (" #call ")", cudaGetErrorString(e__)); \
+  } while (0)
+
+static void dims_from_cfg(const ff_config_t& c, FFDims* dm) {
+  dm->B = c.batch; dm->T = c.T; dm->H = c.H; dm->W = c.W; dm->heads = c.heads; dm->d = c.head_dim;
+  dm->BH = c.batch * c.heads;
+  for (int a = 0; a < 3; ++a) { dm->L[a] = c.low_cut[a]; dm->M[a] = c.mid_cut[a]; }
+  dm->r = c.low_compress; dm->b = c.mid_block; dm->s = c.mid_stride; dm->R = c.high_radius;
+  dm->m = c.n_summary; dm->hid = c.router_hidden; dm->dt = c.t_embed_dim;
+  dm->fp32 = (c.dtype == FF_FP32);
+  dm->N = (long long)c.T * c.H * c.W;
+  dm->Nlow = (long long)c.low_cut[0] * c.low_cut[1] * c.low_cut[2];
+  dm->Nbar = (dm->Nlow + c.low_compress - 1) / (c.low_compress > 0 ? c.low_compress : 1);
+  dm->Nmid = (long long)c.mid_cut[0] * c.mid_cut[1] * c.mid_cut[2] - dm->Nlow;
+  dm->Nhigh = dm->N - (long long)c.mid_cut[0] * c.mid_cut[1] * c.mid_cut[2];
+  dm->nb = (dm->Nmid + c.mid_block - 1) / (c.mid_block > 0 ? c.mid_block : 1);
+}
+
+extern "C" ff_status_t ff_config_validate(const ff_config_t* c) {
+  if (!c) return fail(nullptr, FF_ERR_INVALID_ARG, "cfg is NULL%s");
+  if (c->batch < 1 || c->T < 1 || c->H < 1 || c->W < 1 || c->heads < 1 || c->head_dim < 1)
+    return fail(nullptr, FF_ERR_INVALID_ARG, "batch, grid, heads and head_dim must be positive%s");
+  if (c->dtype != FF_BF16 && c->dtype != FF_FP32) return fail(nullptr, FF_ERR_INVALID_ARG, "dtype must be FF_BF16 or FF_FP32%s");
+  const int n[3] = {c->T, c->H, c->W};
+  for (int a = 0; a < 3; ++a) {
+    if (c->low_cut[a] < 0 || c->low_cut[a] > c->mid_cut[a] || c->mid_cut[a] > n[a])
+      return fail(nullptr, FF_ERR_INVALID_ARG, "cut-offs must satisfy 0 <= L_a <= M_a <= n_a (axis %s%lld)", "", a);
+  }
+  if (c->low_compress < 1 || c->mid_block < 1 || c->mid_stride < 1 || c->high_radius < 0 || c->n_summary < 0)
+    return fail(nullptr, FF_ERR_INVALID_ARG, "need r >= 1, b >= 1, s >= 1, R >= 0, m >= 0%s");
+  if (c->router_hidden < 1 || c->t_embed_dim < 2 || (c->t_embed_dim & 1))
+    return fail(nullptr, FF_ERR_INVALID_ARG, "router_hidden >= 1 and an even t_embed_dim >= 2 are required%s");
+  if (c->head_dim % 32 != 0 || c->head_dim > 128)
+    return fail(nullptr, FF_ERR_UNSUPPORTED, "head_dim must be a multiple of 32 and <= 128%s");
+  if (c->T > 128 || c->H > 128 || c->W > 128) return fail(nullptr, FF_ERR_UNSUPPORTED, "axis lengths above 128 are not supported%s");
+  if (c->router_hidden > 1024 || c->n_summary > 64) return fail(nullptr, FF_ERR_UNSUPPORTED, "router_hidden <= 1024 and m <= 64 are supported%s");
+  FFDims dm; dims_from_cfg(*c, &dm);
+  if (dm.Nlow < 1 || dm.Nmid < 1 || dm.Nhigh < 1) return fail(nullptr, FF_ERR_EMPTY_BAND, "the cut-offs leave a band empty%s");
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_band_sizes(const ff_config_t* c, int64_t sizes[4]) {
+  if (!sizes) return fail(nullptr, FF_ERR_INVALID_ARG, "sizes is NULL%s");
+  ff_status_t s = ff_config_validate(c);
+  if (s != FF_OK && s != FF_ERR_EMPTY_BAND && s != FF_ERR_UNSUPPORTED) return s;
+  FFDims dm; dims_from_cfg(*c, &dm);
+  sizes[0] = dm.Nlow; sizes[1] = dm.Nbar; sizes[2] = dm.Nmid; sizes[3] = dm.Nhigh;
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_band_rank(const ff_config_t* c, int32_t kt, int32_t kh, int32_t kw, int32_t* band,
+                                    int64_t* rank) {
+  if (!band || !rank) return fail(nullptr, FF_ERR_INVALID_ARG, "band/rank is NULL%s");
+  ff_status_t s = ff_config_validate(c);
+  if (s != FF_OK && s != FF_ERR_EMPTY_BAND && s != FF_ERR_UNSUPPORTED) return s;
+  if (kt < 0 || kh < 0 || kw < 0 || kt >= c->T || kh >= c->H || kw >= c->W)
+    return fail(nullptr, FF_ERR_INVALID_ARG, "coefficient index outside the grid%s");
+  FFDims dm; dims_from_cfg(*c, &dm);
+  long long rk;
+  *band = ff_band_rank_of(dm, kt, kh, kw, &rk);
+  *rank = rk;
+  return FF_OK;
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+void ff_compute_layout(const FFDims& dm, bool with_staging, FFLayout* lay) {
+  const size_t e = dm.fp32 ? 4 : 2;
+  const size_t d = dm.d, BH = dm.BH;
+  // Tensor-heads per transform launch: as many as fit two fp32 scratch grids of ~4 GiB each.
+  const size_t per = (size_t)dm.N * d * 4;
+  size_t G = ((size_t)4 << 30) / per;
+  if (G < 1) G = 1;
+  if (G > 3 * BH) G = 3 * BH;
+  lay->group = (int)G;
+  const size_t sizes[19] = {
+      3 * BH * (size_t)dm.Nlow * d * 4,   // 0 spec_low
+      3 * BH * (size_t)dm.Nmid * d * e,   // 1 spec_mid
+      3 * BH * (size_t)dm.Nhigh * d * e,  // 2 spec_high
+      3 * BH * (size_t)dm.Nbar * d * 4,   // 3 pooled
+      BH * (size_t)dm.Nbar * d * 4,       // 4 y_low
+      BH * (size_t)dm.Nmid * d * e,       // 5 y_mid
+      BH * (size_t)dm.Nhigh * d * e,      // 6 y_high
+      BH * 3 * (size_t)(dm.m > 0 ? dm.m : 1) * d * 4,  // 7 summary
+      (size_t)dm.B * 3 * d * 8,           // 8 energy
+      BH,                                 // 9 alloc
+      (size_t)dm.B * 3 * 4,               // 10 pi
+      (size_t)dm.B * 4,                   // 11 timestep
+      256,                                // 12 status
+      G * per,                            // 13 scratchA
+      G * per,                            // 14 scratchB
+      with_staging ? BH * (size_t)dm.N * d * e : 0,  // 15..18 staging
+      with_staging ? BH * (size_t)dm.N * d * e : 0,
+      with_staging ? BH * (size_t)dm.N * d * e : 0,
+      with_staging ? BH * (size_t)dm.N * d * e : 0,
+  };
+  size_t off = 0;
+  for (int i = 0; i < 19; ++i) { lay->off[i] = off; off += align_up(sizes[i], 256); }
+  lay->total = off;
+}
+
+extern "C" ff_status_t ff_workspace_bytes(const ff_config_t* c, size_t* bytes) {
+  if (!bytes) return fail(nullptr, FF_ERR_INVALID_ARG, "bytes is NULL%s");
+  ff_status_t s = ff_config_validate(c);
+  if (s != FF_OK) return s;
+  FFDims dm; dims_from_cfg(*c, &dm);
+  FFLayout lay; ff_compute_layout(dm, false, &lay);
+  *bytes = lay.total;
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_workspace_bytes_host(const ff_config_t* c, size_t* bytes) {
+  if (!bytes) return fail(nullptr, FF_ERR_INVALID_ARG, "bytes is NULL%s");
+  ff_status_t s = ff_config_validate(c);
+  if (s != FF_OK) return s;
+  FFDims dm; dims_from_cfg(*c, &dm);
+  FFLayout lay; ff_compute_layout(dm, true, &lay);
+  *bytes = lay.total;
+  return FF_OK;
+}
+
+static ff_status_t upload(ff_plan* p, float** dst, const float* src, size_t n) {
+  FF_CUDA(p, cudaMalloc((void**)dst, n * sizeof(float)));
+  FF_CUDA(p, cudaMemcpy(*dst, src, n * sizeof(float), cudaMemcpyHostToDevice));
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_destroy(ff_plan_t* p) {
+  if (!p) return FF_OK;
+  for (int a = 0; a < 3; ++a) { cudaFree(p->basis[a]); cudaFree(p->basis_t[a]); }
+  if (p->ev[0]) for (int i = 0; i <= FF_STAGE_COUNT; ++i) cudaEventDestroy(p->ev[i]);
+  cudaFree(p->W1); cudaFree(p->b1); cudaFree(p->W2); cudaFree(p->b2); cudaFree(p->U);
+  delete p;
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_plan_create(const ff_config_t* c, const ff_weights_t* w, ff_plan_t** out) {
+  if (!out) return fail(nullptr, FF_ERR_INVALID_ARG, "out_plan is NULL%s");
+  *out = nullptr;
+  ff_status_t s = ff_config_validate(c);
+  if (s != FF_OK) return s;
+  ff_plan* p = new (std::nothrow) ff_plan();
+  if (!p) return fail(nullptr, FF_ERR_INVALID_ARG, "out of host memory%s");
+  memset(p, 0, sizeof(*p));
+  p->cfg = *c;
+  dims_from_cfg(*c, &p->dm);
+  cudaError_t ce = cudaGetDevice(&p->device);
+  if (ce != cudaSuccess) {
+    fail(nullptr, FF_ERR_CUDA, "no usable CUDA device: %s", cudaGetErrorString(ce));
+    delete p;
+    return FF_ERR_CUDA;
+  }
+  // DCT-II matrices C[k][i] = alpha_k cos(pi (2i+1) k / (2n)), evaluated in double.
+  const int n[3] = {c->T, c->H, c->W};
+  for (int a = 0; a < 3 && s == FF_OK; ++a) {
+    std::vector<float> C((size_t)n[a] * n[a]), Ct((size_t)n[a] * n[a]);
+    for (int k = 0; k < n[a]; ++k)
+      for (int i = 0; i < n[a]; ++i) {
+        const double alpha = (k == 0) ? sqrt(1.0 / n[a]) : sqrt(2.0 / n[a]);
+        const double v = alpha * cos(M_PI * (2.0 * i + 1.0) * k / (2.0 * n[a]));
+        C[(size_t)k * n[a] + i] = (float)v;
+        Ct[(size_t)i * n[a] + k] = (float)v;
+      }
+    s = upload(p, &p->basis[a], C.data(), C.size());
+    if (s == FF_OK) s = upload(p, &p->basis_t[a], Ct.data(), Ct.size());
+  }
+  const size_t d = c->head_dim, hid = c->router_hidden, nin = 3 * d + c->t_embed_dim;
+  if (s == FF_OK && w && w->W1 && w->b1 && w->W2 && w->b2) {
+    s = upload(p, &p->W1, w->W1, hid * nin);
+    if (s == FF_OK) s = upload(p, &p->b1, w->b1, hid);
+    if (s == FF_OK) s = upload(p, &p->W2, w->W2, 3 * hid);
+    if (s == FF_OK) s = upload(p, &p->b2, w->b2, 3);
+    p->has_router = true;
+  }
+  if (s == FF_OK) {
+    std::vector<float> U(3 * d * d, 0.f);
+    if (w && w->U) memcpy(U.data(), w->U, U.size() * sizeof(float));
+    else for (size_t l = 0; l < 3; ++l) for (size_t i = 0; i < d; ++i) U[(l * d + i) * d + i] = 1.f;
+    s = upload(p, &p->U, U.data(), U.size());
+  }
+  if (s != FF_OK) {
+    snprintf(g_err, 512, "%s", p->err);
+    ff_destroy(p);
+    return s;
+  }
+  ff_compute_layout(p->dm, false, &p->lay);
+  *out = p;
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_plan_workspace_bytes(const ff_plan_t* p, size_t* bytes) {
+  if (!p || !bytes) return fail(nullptr, FF_ERR_INVALID_ARG, "plan or bytes is NULL%s");
+  *bytes = p->lay.total;
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_plan_set_workspace(ff_plan_t* p, void* ptr, size_t bytes) {
+  if (!p) return fail(nullptr, FF_ERR_INVALID_ARG, "plan is NULL%s");
+  if (!ptr) return fail(p, FF_ERR_WORKSPACE, "workspace pointer is NULL%s");
+  if (((uintptr_t)ptr) & 255) return fail(p, FF_ERR_WORKSPACE, "workspace must be 256-byte aligned%s");
+  FFLayout plain, staged;
+  ff_compute_layout(p->dm, false, &plain);
+  ff_compute_layout(p->dm, true, &staged);
+  if (bytes < plain.total)
+    return fail(p, FF_ERR_WORKSPACE, "workspace too small%s: %lld bytes given, %lld needed", "", (long long)bytes, (long long)plain.total);
+  p->ws_has_staging = bytes >= staged.total;
+  p->lay = p->ws_has_staging ? staged : plain;
+  p->ws = ptr; p->ws_bytes = bytes;
+  char* base = (char*)ptr;
+  const size_t* o = p->lay.off;
+  FFBuffers& b = p->buf;
+  b.spec_low = (float*)(base + o[0]); b.spec_mid = base + o[1]; b.spec_high = base + o[2];
+  b.pooled = (float*)(base + o[3]); b.y_low = (float*)(base + o[4]); b.y_mid = base + o[5]; b.y_high = base + o[6];
+  b.summary = (float*)(base + o[7]); b.energy = (double*)(base + o[8]); b.alloc = (uint8_t*)(base + o[9]);
+  b.pi = (float*)(base + o[10]); b.timestep = (float*)(base + o[11]); b.status = (int*)(base + o[12]);
+  b.scratchA = (float*)(base + o[13]); b.scratchB = (float*)(base + o[14]);
+  b.stage_q = p->ws_has_staging ? base + o[15] : nullptr; b.stage_k = p->ws_has_staging ? base + o[16] : nullptr;
+  b.stage_v = p->ws_has_staging ? base + o[17] : nullptr; b.stage_out = p->ws_has_staging ? base + o[18] : nullptr;
+  FF_CUDA(p, cudaMemset(b.status, 0, 256));
+  return FF_OK;
+}
+
+extern "C" const char* ff_last_error(const ff_plan_t* p) { return p ? p->err : g_err; }
+
+extern "C" ff_status_t ff_plan_set_attention_impl(ff_plan_t* p, int32_t impl) {
+  if (!p) return fail(nullptr, FF_ERR_INVALID_ARG, "plan is NULL%s");
+  if (impl < 0 || impl > 1) return fail(p, FF_ERR_INVALID_ARG, "attention impl must be 0 or 1%s");
+  p->attn_impl = impl;
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_plan_last_launches(const ff_plan_t* p, int64_t* n) {
+  if (!p || !n) return fail(nullptr, FF_ERR_INVALID_ARG, "plan or output is NULL%s");
+  *n = p->launches;
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_plan_device_status(ff_plan_t* p, void* stream) {
+  if (!p) return fail(nullptr, FF_ERR_INVALID_ARG, "plan is NULL%s");
+  if (!p->ws) return fail(p, FF_ERR_WORKSPACE, "no workspace set%s");
+  cudaStream_t st = (cudaStream_t)stream;
+  int word = 0;
+  FF_CUDA(p, cudaMemcpyAsync(&word, p->buf.status, sizeof(int), cudaMemcpyDeviceToHost, st));
+  FF_CUDA(p, cudaStreamSynchronize(st));
+  if (word != 0) {
+    FF_CUDA(p, cudaMemsetAsync(p->buf.status, 0, sizeof(int), st));
+    return fail(p, (ff_status_t)word, "device status word reports an error%s (code %lld)", "", word);
+  }
+  return FF_OK;
+}
+
+static ff_status_t check_call(ff_plan* p, const void* Q, const void* K, const void* V) {
+  if (!p) return fail(nullptr, FF_ERR_INVALID_ARG, "plan is NULL%s");
+  if (!Q || !K || !V) return fail(p, FF_ERR_INVALID_ARG, "Q, K or V is NULL%s");
+  if (!p->ws) return fail(p, FF_ERR_WORKSPACE, "ff_plan_set_workspace has not been called%s");
+  if ((((uintptr_t)Q) | ((uintptr_t)K) | ((uintptr_t)V)) & 15)
+    return fail(p, FF_ERR_INVALID_ARG, "Q, K and V must be 16-byte aligned%s");
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_plan_set_profiling(ff_plan_t* p, int32_t enable) {
+  if (!p) return fail(nullptr, FF_ERR_INVALID_ARG, "plan is NULL%s");
+  if (enable && !p->ev[0])
+    for (int i = 0; i <= FF_STAGE_COUNT; ++i) FF_CUDA(p, cudaEventCreate(&p->ev[i]));
+  p->profiling = enable != 0;
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_plan_stage_times(ff_plan_t* p, float ms[FF_STAGE_COUNT], int64_t launches[FF_STAGE_COUNT]) {
+  if (!p || !ms || !launches) return fail(nullptr, FF_ERR_INVALID_ARG, "plan or output is NULL%s");
+  if (!p->profiling) return fail(p, FF_ERR_INVALID_ARG, "profiling is not enabled%s");
+  FF_CUDA(p, cudaEventSynchronize(p->ev[FF_STAGE_COUNT]));
+  for (int i = 0; i < FF_STAGE_COUNT; ++i) {
+    FF_CUDA(p, cudaEventElapsedTime(&ms[i], p->ev[i], p->ev[i + 1]));
+    launches[i] = p->stage_launches[i];
+  }
+  return FF_OK;
+}
+
+// Stage boundary: remembers the launches of the stage that just ended and records its end event.
+static cudaError_t mark(ff_plan* p, int boundary, cudaStream_t st) {
+  static thread_local long long before = 0;
+  if (boundary == 0) before = 0;
+  else { p->stage_launches[boundary - 1] = p->launches - before; before = p->launches; }
+  return p->profiling ? cudaEventRecord(p->ev[boundary], st) : cudaSuccess;
+}
+
+// Transform, statistics and router: the part ff_route and an internally routed ff_forward share.
+static ff_status_t transform_and_route(ff_plan* p, const void* Q, const void* K, const void* V, const float* timestep,
+                                       bool route, cudaStream_t st) {
+  FF_CUDA(p, mark(p, 0, st));
+  FF_CUDA(p, ffk_forward_transform(p, Q, K, V, st));
+  FF_CUDA(p, mark(p, 1, st));
+  if (route) {
+    if (!p->has_router) return fail(p, FF_ERR_NOT_ROUTED, "the plan was created without router weights%s");
+    if (!timestep) return fail(p, FF_ERR_NOT_ROUTED, "neither an allocation nor a timestep was given%s");
+    FF_CUDA(p, cudaMemcpyAsync(p->buf.timestep, timestep, sizeof(float) * p->dm.B, cudaMemcpyHostToDevice, st));
+    FF_CUDA(p, cudaMemsetAsync(p->buf.energy, 0, sizeof(double) * p->dm.B * 3 * p->dm.d, st));
+    FF_CUDA(p, ffk_band_energy(p, st));
+    FF_CUDA(p, ffk_router(p, p->buf.alloc, st));
+  }
+  FF_CUDA(p, mark(p, 2, st));
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_route(ff_plan_t* p, const void* Q, const void* K, const void* V, const float* timestep,
+                                uint8_t* alloc_dev, uint8_t* alloc_host, float* pi_host, void* stream) {
+  ff_status_t s = check_call(p, Q, K, V);
+  if (s != FF_OK) return s;
+  if (!timestep) return fail(p, FF_ERR_INVALID_ARG, "timestep is NULL%s");
+  cudaStream_t st = (cudaStream_t)stream;
+  p->launches = 0;
+  s = transform_and_route(p, Q, K, V, timestep, true, st);
+  if (s != FF_OK) return s;
+  if (alloc_dev) FF_CUDA(p, cudaMemcpyAsync(alloc_dev, p->buf.alloc, p->dm.BH, cudaMemcpyDeviceToDevice, st));
+  if (alloc_host) FF_CUDA(p, cudaMemcpyAsync(alloc_host, p->buf.alloc, p->dm.BH, cudaMemcpyDeviceToHost, st));
+  if (pi_host) FF_CUDA(p, cudaMemcpyAsync(pi_host, p->buf.pi, sizeof(float) * 3 * p->dm.B, cudaMemcpyDeviceToHost, st));
+  if (alloc_host || pi_host) FF_CUDA(p, cudaStreamSynchronize(st));
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_forward(ff_plan_t* p, const void* Q, const void* K, const void* V, const uint8_t* alloc_dev,
+                                  const float* timestep, void* out, void* stream) {
+  ff_status_t s = check_call(p, Q, K, V);
+  if (s != FF_OK) return s;
+  if (!out) return fail(p, FF_ERR_INVALID_ARG, "out is NULL%s");
+  if (((uintptr_t)out) & 15) return fail(p, FF_ERR_INVALID_ARG, "out must be 16-byte aligned%s");
+  if (!alloc_dev && !timestep) return fail(p, FF_ERR_NOT_ROUTED, "neither an allocation nor a timestep was given%s");
+  cudaStream_t st = (cudaStream_t)stream;
+  p->launches = 0;
+  s = transform_and_route(p, Q, K, V, timestep, alloc_dev == nullptr, st);
+  if (s != FF_OK) return s;
+  if (alloc_dev) FF_CUDA(p, cudaMemcpyAsync(p->buf.alloc, alloc_dev, p->dm.BH, cudaMemcpyDeviceToDevice, st));
+  FF_CUDA(p, ffk_pool_low(p, st));
+  FF_CUDA(p, ffk_attention_simt(p, st));
+  FF_CUDA(p, mark(p, 3, st));
+  if (p->dm.m > 0) FF_CUDA(p, ffk_summaries(p, st));
+  FF_CUDA(p, mark(p, 4, st));
+  FF_CUDA(p, ffk_exchange_inverse(p, out, st));
+  FF_CUDA(p, mark(p, 5, st));
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_forward_host(ff_plan_t* p, const void* Qh, const void* Kh, const void* Vh,
+                                       const uint8_t* alloc_host, const float* timestep, void* out_host, void* stream) {
+  if (!p) return fail(nullptr, FF_ERR_INVALID_ARG, "plan is NULL%s");
+  if (!Qh || !Kh || !Vh || !out_host) return fail(p, FF_ERR_INVALID_ARG, "a host buffer is NULL%s");
+  if (!p->ws) return fail(p, FF_ERR_WORKSPACE, "ff_plan_set_workspace has not been called%s");
+  if (!p->ws_has_staging) return fail(p, FF_ERR_WORKSPACE, "workspace lacks staging space: size it with ff_workspace_bytes_host%s");
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t bytes = (size_t)p->dm.BH * p->dm.N * p->dm.d * (p->dm.fp32 ? 4 : 2);
+  FF_CUDA(p, cudaMemcpyAsync(p->buf.stage_q, Qh, bytes, cudaMemcpyHostToDevice, st));
+  FF_CUDA(p, cudaMemcpyAsync(p->buf.stage_k, Kh, bytes, cudaMemcpyHostToDevice, st));
+  FF_CUDA(p, cudaMemcpyAsync(p->buf.stage_v, Vh, bytes, cudaMemcpyHostToDevice, st));
+  // The caller's masks travel through the tail of the (not yet used) output staging area.
+  uint8_t* alloc_dev = nullptr;
+  if (alloc_host) {
+    alloc_dev = (uint8_t*)p->buf.stage_out;
+    FF_CUDA(p, cudaMemcpyAsync(alloc_dev, alloc_host, p->dm.BH, cudaMemcpyHostToDevice, st));
+  }
+  ff_status_t s = ff_forward(p, p->buf.stage_q, p->buf.stage_k, p->buf.stage_v, alloc_dev, timestep, p->buf.stage_out, st);
+  if (s != FF_OK) return s;
+  FF_CUDA(p, cudaMemcpyAsync(out_host, p->buf.stage_out, bytes, cudaMemcpyDeviceToHost, st));
+  FF_CUDA(p, cudaStreamSynchronize(st));
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_get_tap(const ff_plan_t* p, int32_t which, const void** ptr, size_t* bytes) {
+  if (!p || !ptr || !bytes) return fail(nullptr, FF_ERR_INVALID_ARG, "plan, dev_ptr or bytes is NULL%s");
+  if (!p->ws) return FF_ERR_WORKSPACE;
+  const FFDims& dm = p->dm;
+  const size_t e = dm.fp32 ? 4 : 2, d = dm.d, BH = dm.BH;
+  const FFBuffers& b = p->buf;
+  switch (which) {
+    case FF_TAP_SPEC_LOW: *ptr = b.spec_low; *bytes = 3 * BH * dm.Nlow * d * 4; break;
+    case FF_TAP_SPEC_MID: *ptr = b.spec_mid; *bytes = 3 * BH * dm.Nmid * d * e; break;
+    case FF_TAP_SPEC_HIGH: *ptr = b.spec_high; *bytes = 3 * BH * dm.Nhigh * d * e; break;
+    case FF_TAP_POOLED_LOW: *ptr = b.pooled; *bytes = 3 * BH * dm.Nbar * d * 4; break;
+    case FF_TAP_Y_LOW: *ptr = b.y_low; *bytes = BH * dm.Nbar * d * 4; break;
+    case FF_TAP_Y_MID: *ptr = b.y_mid; *bytes = BH * dm.Nmid * d * e; break;
+    case FF_TAP_Y_HIGH: *ptr = b.y_high; *bytes = BH * dm.Nhigh * d * e; break;
+    case FF_TAP_SUMMARY: *ptr = b.summary; *bytes = BH * 3 * (size_t)dm.m * d * 4; break;
+    case FF_TAP_ENERGY: *ptr = b.energy; *bytes = (size_t)dm.B * 3 * d * 8; break;
+    case FF_TAP_ALLOC: *ptr = b.alloc; *bytes = BH; break;
+    case FF_TAP_PI: *ptr = b.pi; *bytes = (size_t)dm.B * 3 * 4; break;
+    default: return FF_ERR_INVALID_ARG;
+  }
+  return FF_OK;
+}

@@ -1,0 +1,109 @@
+// Internal declarations shared by the host API and the kernel translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "freqformer.h"
+
+#if defined(__CUDACC__)
+#define FF_HD __host__ __device__ __forceinline__
+#else
+#define FF_HD inline
+#endif
+
+// Problem sizes derived from ff_config_t ("Frequency band partitioning": N_low + N_mid + N_high = N).
+struct FFDims {
+  int B, T, H, W, heads, d, BH;
+  int L[3], M[3];
+  int r, b, s, R, m, hid, dt;
+  int fp32;              // storage type of Q,K,V,out and of the mid/high band buffers
+  long long N, Nlow, Nbar, Nmid, Nhigh;
+  long long nb;          // number of mid blocks
+};
+
+// Number of members of the box A = [0,A_t) x [0,A_h) x [0,A_w) whose flat index is below that of k.
+FF_HD long long ff_box_count_below(int At, int Ah, int Aw, int kt, int kh, int kw) {
+  long long c = (long long)(kt < At ? kt : At) * Ah * Aw;
+  if (kt < At) {
+    c += (long long)(kh < Ah ? kh : Ah) * Aw;
+    if (kh < Ah) c += (kw < Aw ? kw : Aw);
+  }
+  return c;
+}
+
+// Band (0 low, 1 mid, 2 high) and band-local rank of coefficient (kt,kh,kw): nested boxes, band
+// order = increasing flat index.
+FF_HD int ff_band_rank_of(const FFDims& dm, int kt, int kh, int kw, long long* rank) {
+  const long long cl = ff_box_count_below(dm.L[0], dm.L[1], dm.L[2], kt, kh, kw);
+  const long long cm = ff_box_count_below(dm.M[0], dm.M[1], dm.M[2], kt, kh, kw);
+  const bool in_low = kt < dm.L[0] && kh < dm.L[1] && kw < dm.L[2];
+  const bool in_mid = kt < dm.M[0] && kh < dm.M[1] && kw < dm.M[2];
+  if (in_low) { *rank = cl; return 0; }
+  if (in_mid) { *rank = cm - cl; return 1; }
+  *rank = ((long long)kt * dm.H + kh) * dm.W + kw - cm;
+  return 2;
+}
+
+// Device buffers inside the caller's workspace.
+struct FFBuffers {
+  float* spec_low;   // [3][BH][Nlow][d]
+  void* spec_mid;    // st [3][BH][Nmid][d]
+  void* spec_high;   // st [3][BH][Nhigh][d]
+  float* pooled;     // [3][BH][Nbar][d]
+  float* y_low;      // [BH][Nbar][d]
+  void* y_mid;       // st [BH][Nmid][d]
+  void* y_high;      // st [BH][Nhigh][d]
+  float* summary;    // [BH][3][m][d]
+  double* energy;    // [B][3][d]
+  uint8_t* alloc;    // [BH]
+  float* pi;         // [B][3]
+  float* timestep;   // [B]
+  int* status;       // device status word
+  float* scratchA;   // [G][N][d]
+  float* scratchB;   // [G][N][d]
+  void* stage_q;     // host-call staging (st [BH][N][d]) or NULL
+  void* stage_k;
+  void* stage_v;
+  void* stage_out;
+};
+
+struct FFLayout {
+  size_t off[24];
+  size_t total;
+  int group;         // G: tensor-heads processed per transform launch
+};
+
+struct ff_plan {
+  ff_config_t cfg;
+  FFDims dm;
+  int device;
+  // device tables owned by the plan
+  float* basis[3];    // C_T, C_H, C_W  [n][n], C[k][i]
+  float* basis_t[3];  // transposes
+  float* W1; float* b1; float* W2; float* b2; float* U;
+  bool has_router;
+  // workspace
+  void* ws; size_t ws_bytes;
+  FFBuffers buf;
+  FFLayout lay;
+  bool ws_has_staging;
+  int attn_impl;
+  long long launches;
+  bool profiling;
+  cudaEvent_t ev[FF_STAGE_COUNT + 1];
+  long long stage_launches[FF_STAGE_COUNT];
+  char err[512];
+};
+
+void ff_compute_layout(const FFDims& dm, bool with_staging, FFLayout* lay);
+
+// ---- kernel launchers (ff_simt.cu).  Each returns the cudaError_t of its launches. --------------
+cudaError_t ffk_forward_transform(ff_plan* p, const void* Q, const void* K, const void* V, cudaStream_t st);
+cudaError_t ffk_band_energy(ff_plan* p, cudaStream_t st);
+cudaError_t ffk_router(ff_plan* p, uint8_t* alloc_out, cudaStream_t st);
+cudaError_t ffk_pool_low(ff_plan* p, cudaStream_t st);
+cudaError_t ffk_attention_simt(ff_plan* p, cudaStream_t st);
+cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st);
+cudaError_t ffk_exchange_inverse(ff_plan* p, void* out, cudaStream_t st);
