@@ -97,7 +97,7 @@ void ff_compute_layout(const FFDims& dm, bool with_staging, FFLayout* lay) {
   if (G < 1) G = 1;
   if (G > 3 * BH) G = 3 * BH;
   lay->group = (int)G;
-  const size_t sizes[19] = {
+  const size_t sizes[20] = {
       3 * BH * (size_t)dm.Nlow * d * 4,   // 0 spec_low
       3 * BH * (size_t)dm.Nmid * d * e,   // 1 spec_mid
       3 * BH * (size_t)dm.Nhigh * d * e,  // 2 spec_high
@@ -117,9 +117,10 @@ void ff_compute_layout(const FFDims& dm, bool with_staging, FFLayout* lay) {
       with_staging ? BH * (size_t)dm.N * d * e : 0,
       with_staging ? BH * (size_t)dm.N * d * e : 0,
       with_staging ? BH * (size_t)dm.N * d * e : 0,
+      ffk_tc_work_bytes(),                // 19 worklist
   };
   size_t off = 0;
-  for (int i = 0; i < 19; ++i) { lay->off[i] = off; off += align_up(sizes[i], 256); }
+  for (int i = 0; i < 20; ++i) { lay->off[i] = off; off += align_up(sizes[i], 256); }
   lay->total = off;
 }
 
@@ -169,6 +170,7 @@ extern "C" ff_status_t ff_plan_create(const ff_config_t* c, const ff_weights_t* 
   p->cfg = *c;
   dims_from_cfg(*c, &p->dm);
   cudaError_t ce = cudaGetDevice(&p->device);
+  if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
   if (ce != cudaSuccess) {
     fail(nullptr, FF_ERR_CUDA, "no usable CUDA device: %s", cudaGetErrorString(ce));
     delete p;
@@ -240,7 +242,9 @@ extern "C" ff_status_t ff_plan_set_workspace(ff_plan_t* p, void* ptr, size_t byt
   b.scratchA = (float*)(base + o[13]); b.scratchB = (float*)(base + o[14]);
   b.stage_q = p->ws_has_staging ? base + o[15] : nullptr; b.stage_k = p->ws_has_staging ? base + o[16] : nullptr;
   b.stage_v = p->ws_has_staging ? base + o[17] : nullptr; b.stage_out = p->ws_has_staging ? base + o[18] : nullptr;
+  b.work = (int*)(base + o[19]);
   FF_CUDA(p, cudaMemset(b.status, 0, 256));
+  p->tc_ok = ffk_tc_supported(p->dm) && ffk_tc_prepare(p);
   return FF_OK;
 }
 
@@ -356,7 +360,12 @@ extern "C" ff_status_t ff_forward(ff_plan_t* p, const void* Q, const void* K, co
   if (s != FF_OK) return s;
   if (alloc_dev) FF_CUDA(p, cudaMemcpyAsync(p->buf.alloc, alloc_dev, p->dm.BH, cudaMemcpyDeviceToDevice, st));
   FF_CUDA(p, ffk_pool_low(p, st));
-  FF_CUDA(p, ffk_attention_simt(p, st));
+  if (p->tc_ok && p->attn_impl == 0) {
+    FF_CUDA(p, ffk_attention_simt(p, FF_BAND_LOW, st));
+    FF_CUDA(p, ffk_attention_tc(p, st));
+  } else {
+    FF_CUDA(p, ffk_attention_simt(p, FF_BAND_LOW | FF_BAND_MID | FF_BAND_HIGH, st));
+  }
   FF_CUDA(p, mark(p, 3, st));
   if (p->dm.m > 0) FF_CUDA(p, ffk_summaries(p, st));
   FF_CUDA(p, mark(p, 4, st));

@@ -1,0 +1,478 @@
+// Mid- and high-band attention on the 5th-generation tensor cores ("Hierarchical frequency-domain
+// attention": strided block-sparse attention on the mid band, sliding-window attention on the high
+// band), bf16 operands, fp32 accumulation, head_dim 128.
+//
+// One persistent launch runs both branches from a worklist of (head, band, query tile) items that
+// is rebuilt from the head-to-band allocation before every launch.  A CTA owns every gridDim-th
+// item.  Per CTA:
+//   warp 0      TMA producer: Q tile (double buffered), K and V tiles (two stages each)
+//   warp 1      tcgen05.mma issuer: S = Q K^T (A, B from shared memory), O += P V (A = P from
+//               tensor memory, B = V as an MN-major operand); owns the tensor-memory allocation
+//   warps 2..5  softmax: one query row per thread (row = TMEM lane), scores read with tcgen05.ld,
+//               key masks generated in registers from the row's band rank, P written back to
+//               tensor memory as bf16 over the scores it came from; O is accumulated in tensor
+//               memory and rescaled only when a row's running maximum grows by more than 2^8
+// Tensor memory (512 columns): S/P buffer 0, S/P buffer 1, O buffer 0, O buffer 1.
+// Every mbarrier wait is bounded; when one runs out the CTA raises FF_ERR_TIMEOUT in the plan's
+// status word, stops taking work, lets its copies drain, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "ff_internal.h"
+#include "ff_sm100.cuh"
+
+using namespace sm100;
+
+namespace {
+
+constexpr int TILE = 128;            // query rows per item = key rows per tile
+constexpr int HD = 128;              // head_dim
+constexpr int TILE_BYTES = TILE * HD * 2;
+constexpr int HALF_BYTES = TILE_BYTES / 2;
+constexpr int MAX_UNITS = 1024;
+constexpr int TC_THREADS = 192;
+constexpr float LAZY_LOG2 = 8.0f;    // rescale O only when the running max grows by more than this (log2 units)
+
+struct TcParams {
+  FFDims dm;
+  const uint8_t* alloc;
+  int* work;          // [0] = number of units, [1] = total items, then offsets[MAX_UNITS+1], desc[MAX_UNITS], tiles[MAX_UNITS]
+  __nv_bfloat16* y_mid;
+  __nv_bfloat16* y_high;
+  int* status;
+  int rb_mid;         // rows per TMA box of the mid map = min(b, 128)
+};
+
+// Worklist: one unit per (head, mid residue class) and per (head, high band) that the allocation
+// executes; mid units first (their items are the long ones).
+__global__ void build_worklist_kernel(TcParams P) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  const FFDims& dm = P.dm;
+  int* offsets = P.work + 2;
+  int* desc = offsets + MAX_UNITS + 1;
+  int* tiles = desc + MAX_UNITS;
+  int nu = 0, total = 0;
+  const int nclass = (int)(dm.nb < dm.s ? dm.nb : dm.s);
+  for (int bh = 0; bh < dm.BH; ++bh) {
+    if (!(P.alloc[bh] & FF_BAND_MID)) continue;
+    for (int c = 0; c < nclass && nu < MAX_UNITS; ++c) {
+      const long long nblk = (dm.nb - c + dm.s - 1) / dm.s;
+      const int nt = (int)((nblk * dm.b + TILE - 1) / TILE);
+      offsets[nu] = total; desc[nu] = (bh << 12) | (1 << 10) | c; tiles[nu] = nt;
+      total += nt; ++nu;
+    }
+  }
+  for (int bh = 0; bh < dm.BH && nu < MAX_UNITS; ++bh) {
+    if (!(P.alloc[bh] & FF_BAND_HIGH)) continue;
+    const int nt = (int)((dm.Nhigh + TILE - 1) / TILE);
+    offsets[nu] = total; desc[nu] = (bh << 12) | (2 << 10); tiles[nu] = nt;
+    total += nt; ++nu;
+  }
+  offsets[nu] = total;
+  P.work[0] = nu;
+  P.work[1] = total;
+}
+
+struct Item {
+  int band, bh, c, tile, nk;
+  long long n;        // band length
+  long long ks;       // high: first key rank of key tile 0
+};
+
+struct Shared {
+  uint64_t q_full[2], q_empty[2], k_full[2], k_empty[2], v_full[2], v_empty[2];
+  uint64_t s_full[2], p_full[2], o_full[2], o_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+  int n_units, total;
+  int offsets[MAX_UNITS + 1];
+  int desc[MAX_UNITS];
+};
+
+__device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, int it) {
+  int lo = 0, hi = sh.n_units - 1;
+  while (lo < hi) {                       // last unit whose offset <= it
+    const int mid = (lo + hi + 1) >> 1;
+    if (sh.offsets[mid] <= it) lo = mid; else hi = mid - 1;
+  }
+  Item x;
+  const int dsc = sh.desc[lo];
+  x.bh = dsc >> 12; x.band = (dsc >> 10) & 3; x.c = dsc & 1023;
+  x.tile = it - sh.offsets[lo];
+  if (x.band == 1) {
+    x.n = dm.Nmid;
+    x.nk = sh.offsets[lo + 1] - sh.offsets[lo];     // every query tile of a class sees all its key tiles
+    x.ks = 0;
+  } else {
+    x.n = dm.Nhigh;
+    const long long q0 = (long long)x.tile * TILE;
+    x.ks = q0 - dm.R > 0 ? q0 - dm.R : 0;
+    long long ke = q0 + TILE + dm.R;
+    if (ke > x.n) ke = x.n;
+    x.nk = (int)((ke - x.ks + TILE - 1) / TILE);
+  }
+  return x;
+}
+
+// Band rank of class-local position u of residue class c (mid band).
+__device__ __forceinline__ long long mid_rank(const FFDims& dm, int c, long long u) {
+  return ((long long)c + (u / dm.b) * dm.s) * dm.b + (u % dm.b);
+}
+
+// Issues the TMA loads of one 128-row tile (two 64-column halves) into `dst`.
+__device__ __forceinline__ void load_tile(uint8_t* dst, const CUtensorMap* map, uint64_t* bar, const FFDims& dm,
+                                          const Item& x, int slice, long long first, int rb) {
+  mbar_arrive_expect_tx(bar, TILE_BYTES);
+  if (x.band == 2) {
+    tma_load_3d(dst, map, bar, 0, (int)first, slice);
+    tma_load_3d(dst + HALF_BYTES, map, bar, 64, (int)first, slice);
+  } else {
+    for (int i = 0; i < TILE / rb; ++i) {
+      const long long row = mid_rank(dm, x.c, first + (long long)i * rb);
+      // a block past the end of the band starts beyond the tensor: the copy fills zeros
+      const int y = row < dm.Nmid ? (int)row : (int)dm.Nmid;
+      tma_load_3d(dst + i * rb * 128, map, bar, 0, y, slice);
+      tma_load_3d(dst + HALF_BYTES + i * rb * 128, map, bar, 64, y, slice);
+    }
+  }
+}
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap map_mid, const __grid_constant__ CUtensorMap map_high,
+                    const TcParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* sQ = smem;                       // 2 x 32 KB
+  uint8_t* sK = smem + 2 * TILE_BYTES;      // 2 x 32 KB
+  uint8_t* sV = smem + 4 * TILE_BYTES;      // 2 x 32 KB
+  Shared& sh = *(Shared*)(smem + 6 * TILE_BYTES);
+  const FFDims& dm = P.dm;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sh.q_full[i], 1); mbar_init(&sh.q_empty[i], 1);
+      mbar_init(&sh.k_full[i], 1); mbar_init(&sh.k_empty[i], 1);
+      mbar_init(&sh.v_full[i], 1); mbar_init(&sh.v_empty[i], 1);
+      mbar_init(&sh.s_full[i], 1); mbar_init(&sh.p_full[i], 128);
+      mbar_init(&sh.o_full[i], 1); mbar_init(&sh.o_empty[i], 128);
+    }
+    sh.abort_flag = 0;
+    sh.n_units = P.work[0];
+    sh.total = P.work[1];
+    fence_mbar_init();
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i <= sh.n_units; i += TC_THREADS) {
+    sh.offsets[i] = P.work[2 + i];
+    if (i < sh.n_units) sh.desc[i] = P.work[2 + MAX_UNITS + 1 + i];
+  }
+  if (warp == 1) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tm = sh.tmem_base;
+  const int total = sh.total;
+  volatile int* abort_flag = &sh.abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&map_mid); tma_prefetch_desc(&map_high);
+      int iter = 0; unsigned g = 0;
+      bool ok = true;
+      for (int it = blockIdx.x; it < total && ok; it += gridDim.x, ++iter) {
+        const Item x = decode_item(sh, dm, it);
+        const CUtensorMap* map = x.band == 1 ? &map_mid : &map_high;
+        const int rb = x.band == 1 ? P.rb_mid : TILE;
+        const int qb = iter & 1;
+        if (iter >= 2) ok = mbar_wait(&sh.q_empty[qb], ((iter >> 1) - 1) & 1, abort_flag);
+        if (!ok) break;
+        load_tile(sQ + qb * TILE_BYTES, map, &sh.q_full[qb], dm, x, x.bh, (long long)x.tile * TILE, rb);
+        for (int j = 0; j < x.nk && ok; ++j, ++g) {
+          const int st = g & 1;
+          const long long first = x.band == 1 ? (long long)j * TILE : x.ks + (long long)j * TILE;
+          if (g >= 2) ok = mbar_wait(&sh.k_empty[st], ((g >> 1) - 1) & 1, abort_flag);
+          if (!ok) break;
+          load_tile(sK + st * TILE_BYTES, map, &sh.k_full[st], dm, x, dm.BH + x.bh, first, rb);
+          if (g >= 2) ok = mbar_wait(&sh.v_empty[st], ((g >> 1) - 1) & 1, abort_flag);
+          if (!ok) break;
+          load_tile(sV + st * TILE_BYTES, map, &sh.v_full[st], dm, x, 2 * dm.BH + x.bh, first, rb);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_qk = idesc_bf16_f32(TILE, TILE, false, false);
+      const uint32_t idesc_pv = idesc_bf16_f32(TILE, HD, false, true);
+      int iter = 0; unsigned g = 0;
+      bool ok = true, have_prev = false;
+      unsigned pg = 0; int pob = 0, piter = 0; bool pfirst = false;
+      auto issue_pv = [&]() -> bool {
+        const int sb = pg & 1, st = pg & 1;
+        if (!mbar_wait(&sh.p_full[sb], (pg >> 1) & 1, abort_flag)) return false;
+        if (!mbar_wait(&sh.v_full[st], (pg >> 1) & 1, abort_flag)) return false;
+        if (pfirst && piter >= 2 && !mbar_wait(&sh.o_empty[pob], ((piter >> 1) - 1) & 1, abort_flag)) return false;
+        tc_fence_after();
+        const uint32_t vbase = smem_u32(sV + st * TILE_BYTES);
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          umma_ts(tm + 256 + pob * 128, tm + sb * 128 + k * 8, smem_desc_sw128(vbase + k * 2048, HALF_BYTES, 1024),
+                  idesc_pv, (pfirst && k == 0) ? 0u : 1u);
+        umma_commit(&sh.v_empty[st]);
+        umma_commit(&sh.o_full[pob]);
+        return true;
+      };
+      for (int it = blockIdx.x; it < total && ok; it += gridDim.x, ++iter) {
+        const Item x = decode_item(sh, dm, it);
+        const int qb = iter & 1;
+        ok = mbar_wait(&sh.q_full[qb], (iter >> 1) & 1, abort_flag);
+        for (int j = 0; j < x.nk && ok; ++j, ++g) {
+          const int st = g & 1, sb = g & 1;
+          ok = mbar_wait(&sh.k_full[st], (g >> 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t qbase = smem_u32(sQ + qb * TILE_BYTES), kbase = smem_u32(sK + st * TILE_BYTES);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const uint32_t off = (k >> 2) * HALF_BYTES + (k & 3) * 32;
+            umma_ss(tm + sb * 128, smem_desc_sw128(qbase + off, 16, 1024), smem_desc_sw128(kbase + off, 16, 1024),
+                    idesc_qk, k > 0 ? 1u : 0u);
+          }
+          umma_commit(&sh.k_empty[st]);
+          umma_commit(&sh.s_full[sb]);
+          if (j == x.nk - 1) umma_commit(&sh.q_empty[qb]);
+          if (have_prev) ok = issue_pv();
+          pg = g; pob = iter & 1; piter = iter; pfirst = (j == 0); have_prev = true;
+        }
+      }
+      if (ok && have_prev) issue_pv();
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax, one row per thread
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const float sl2 = rsqrtf((float)HD) * 1.4426950408889634f;
+    int iter = 0; unsigned g = 0;
+    unsigned ocount[2] = {0, 0};
+    bool ok = true;
+    for (int it = blockIdx.x; it < total && ok; it += gridDim.x, ++iter) {
+      const Item x = decode_item(sh, dm, it);
+      const int ob = iter & 1;
+      const uint32_t o_addr = tm + lane_addr + 256 + ob * 128;
+      // band rank of this thread's query row
+      const long long u_q = (long long)x.tile * TILE + row;
+      const long long p = x.band == 1 ? mid_rank(dm, x.c, u_q) : u_q;
+      float m_ref = -1e30f, l = 0.f;
+      for (int j = 0; j < x.nk && ok; ++j, ++g) {
+        const int sb = g & 1;
+        const uint32_t s_addr = tm + lane_addr + sb * 128;
+        // valid key columns [clo, chi] of this row in this tile
+        int clo = 0, chi = TILE - 1;
+        bool full;
+        if (x.band == 1) {
+          const long long u0 = (long long)j * TILE;
+          // ranks grow with the class-local position, so the valid keys are a prefix
+          const long long last = mid_rank(dm, x.c, u0 + TILE - 1);
+          full = last < dm.Nmid;
+          if (!full) {
+            chi = -1;
+            for (int cc = TILE - 1; cc >= 0; --cc)
+              if (mid_rank(dm, x.c, u0 + cc) < dm.Nmid) { chi = cc; break; }
+          }
+        } else {
+          const long long t0 = x.ks + (long long)j * TILE;
+          const long long q0 = (long long)x.tile * TILE;
+          full = (t0 >= q0 + TILE - 1 - dm.R) && (t0 + TILE - 1 <= q0 + dm.R) && (t0 + TILE <= x.n);
+          if (!full) {
+            const long long lo = p - dm.R - t0, hi = (p + dm.R < x.n - 1 ? p + dm.R : x.n - 1) - t0;
+            clo = lo > 0 ? (int)(lo < TILE ? lo : TILE) : 0;
+            chi = hi < TILE - 1 ? (int)(hi < -1 ? -1 : hi) : TILE - 1;
+          }
+        }
+        ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full[sb], (g >> 1) & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        // pass 1: row maximum of the raw scores
+        float tmax = -INFINITY;
+        uint32_t r[32];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          tmem_ld32(s_addr + c * 32, r);
+          tmem_wait_ld();
+          if (full) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, __uint_as_float(r[i]));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int col = c * 32 + i;
+              if (col >= clo && col <= chi) tmax = fmaxf(tmax, __uint_as_float(r[i]));
+            }
+          }
+        }
+        const float m_new = fmaxf(m_ref, tmax);
+        const bool need = (m_new - m_ref) * sl2 > LAZY_LOG2;
+        const float alpha = need ? ex2((m_ref - m_new) * sl2) : 1.f;
+        if (j > 0) {
+          // PV of the previous key tile must have landed before O may be touched
+          ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[ob], ocount[ob] & 1, abort_flag));
+          ++ocount[ob];
+          if (!ok) break;
+          tc_fence_after();
+          if (__any_sync(0xffffffffu, need)) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              tmem_ld32(o_addr + c * 32, r);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+              tmem_st32(o_addr + c * 32, r);
+            }
+            tmem_wait_st();
+          }
+        }
+        if (need) { l *= alpha; m_ref = m_new; }
+        // pass 2: P = 2^(s*scale*log2e - m) as bf16 over the scores, row sum
+        const float mb = m_ref * sl2;
+        float sum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          tmem_ld32(s_addr + c * 32, r);
+          tmem_wait_ld();
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float p0 = ex2(fmaf(__uint_as_float(r[2 * i]), sl2, -mb));
+            float p1 = ex2(fmaf(__uint_as_float(r[2 * i + 1]), sl2, -mb));
+            if (!full) {
+              const int col = c * 32 + 2 * i;
+              if (col < clo || col > chi) p0 = 0.f;
+              if (col + 1 < clo || col + 1 > chi) p1 = 0.f;
+            }
+            sum += p0 + p1;
+            const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
+            pk[i] = *(const uint32_t*)&v;
+          }
+          tmem_st16(s_addr + c * 16, pk);
+        }
+        l += sum;
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&sh.p_full[sb]);
+      }
+      if (!ok) break;
+      // epilogue: O / l -> Y
+      ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[ob], ocount[ob] & 1, abort_flag));
+      ++ocount[ob];
+      if (!ok) break;
+      tc_fence_after();
+      const float inv = 1.f / l;
+      const bool store = p < x.n && (x.band != 1 || u_q < (long long)x.nk * TILE);
+      __nv_bfloat16* y = (x.band == 1 ? P.y_mid : P.y_high) + ((size_t)x.bh * x.n + (store ? p : 0)) * HD;
+      uint32_t r[32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        tmem_ld32(o_addr + c * 32, r);
+        tmem_wait_ld();
+        if (store) {
+#pragma unroll
+          for (int v4 = 0; v4 < 4; ++v4) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[v4 * 8 + 2 * i]) * inv,
+                                                             __uint_as_float(r[v4 * 8 + 2 * i + 1]) * inv);
+              w[i] = *(const uint32_t*)&v;
+            }
+            *(uint4*)(y + c * 32 + v4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(&sh.o_empty[ob]);
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (sh.abort_flag) {
+    if (threadIdx.x == 0) atomicExch(P.status, FF_ERR_TIMEOUT);
+    // let copies that were already issued land before the shared memory is released
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tm, 512);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+bool encode_band_map(CUtensorMap* map, void* base, long long rows, int slices, int box_rows) {
+  static EncodeTiledFn enc = nullptr;
+  if (!enc) {
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", (void**)&enc, cudaEnableDefault, &qr) != cudaSuccess || !enc)
+      return false;
+  }
+  cuuint64_t dims[3] = {(cuuint64_t)HD, (cuuint64_t)rows, (cuuint64_t)slices};
+  cuuint64_t strides[2] = {(cuuint64_t)HD * 2, (cuuint64_t)rows * HD * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+size_t ffk_tc_work_bytes() { return (size_t)(2 + 3 * MAX_UNITS + 1) * sizeof(int); }
+
+// The tensor-core kernel covers bf16, head_dim 128 and block sizes that tile 128 rows evenly.
+bool ffk_tc_supported(const FFDims& dm) {
+  if (dm.fp32 || dm.d != HD) return false;
+  const bool b_ok = (dm.b <= TILE) ? (dm.b >= 8 && TILE % dm.b == 0) : (dm.b % TILE == 0);
+  if (!b_ok) return false;
+  const long long nclass = dm.nb < dm.s ? dm.nb : dm.s;
+  if ((long long)dm.BH * (nclass + 1) > MAX_UNITS || dm.BH >= (1 << 19)) return false;
+  if (dm.Nmid >= (1LL << 31) - 256 || dm.Nhigh >= (1LL << 31) - 256) return false;
+  return true;
+}
+
+bool ffk_tc_prepare(ff_plan* p) {
+  static_assert(sizeof(CUtensorMap) <= sizeof(p->tmap_mid), "tensor map storage too small");
+  const FFDims& dm = p->dm;
+  const int rb = dm.b < TILE ? dm.b : TILE;
+  return encode_band_map((CUtensorMap*)p->tmap_mid, p->buf.spec_mid, dm.Nmid, 3 * dm.BH, rb) &&
+         encode_band_map((CUtensorMap*)p->tmap_high, p->buf.spec_high, dm.Nhigh, 3 * dm.BH, TILE);
+}
+
+cudaError_t ffk_attention_tc(ff_plan* p, cudaStream_t st) {
+  const FFDims& dm = p->dm;
+  TcParams P;
+  P.dm = dm; P.alloc = p->buf.alloc; P.work = p->buf.work;
+  P.y_mid = (__nv_bfloat16*)p->buf.y_mid; P.y_high = (__nv_bfloat16*)p->buf.y_high;
+  P.status = p->buf.status; P.rb_mid = dm.b < TILE ? dm.b : TILE;
+  build_worklist_kernel<<<1, 32, 0, st>>>(P);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const size_t smem = 6 * TILE_BYTES + sizeof(Shared) + 1024;
+  e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  attention_tc_kernel<<<p->sm_count, TC_THREADS, smem, st>>>(*(const CUtensorMap*)p->tmap_mid,
+                                                             *(const CUtensorMap*)p->tmap_high, P);
+  p->launches += 2;
+  return cudaGetLastError();
+}

@@ -61,6 +61,7 @@ struct FFBuffers {
   float* pi;         // [B][3]
   float* timestep;   // [B]
   int* status;       // device status word
+  int* work;         // worklist of the tensor-core attention kernel
   float* scratchA;   // [G][N][d]
   float* scratchB;   // [G][N][d]
   void* stage_q;     // host-call staging (st [BH][N][d]) or NULL
@@ -90,6 +91,10 @@ struct ff_plan {
   FFLayout lay;
   bool ws_has_staging;
   int attn_impl;
+  int sm_count;
+  bool tc_ok;                                  // tensor-core attention usable with this plan + workspace
+  alignas(64) unsigned char tmap_mid[128];     // CUtensorMap over the mid-band / high-band coefficient buffers
+  alignas(64) unsigned char tmap_high[128];
   long long launches;
   bool profiling;
   cudaEvent_t ev[FF_STAGE_COUNT + 1];
@@ -104,6 +109,11 @@ cudaError_t ffk_forward_transform(ff_plan* p, const void* Q, const void* K, cons
 cudaError_t ffk_band_energy(ff_plan* p, cudaStream_t st);
 cudaError_t ffk_router(ff_plan* p, uint8_t* alloc_out, cudaStream_t st);
 cudaError_t ffk_pool_low(ff_plan* p, cudaStream_t st);
-cudaError_t ffk_attention_simt(ff_plan* p, cudaStream_t st);
+cudaError_t ffk_attention_simt(ff_plan* p, int band_bits, cudaStream_t st);   // band_bits: which bands to run
+// ---- tensor-core attention (ff_attn_tc.cu) -------------------------------------------------------
+size_t ffk_tc_work_bytes();
+bool ffk_tc_supported(const FFDims& dm);
+bool ffk_tc_prepare(ff_plan* p);               // builds the tensor maps over the workspace
+cudaError_t ffk_attention_tc(ff_plan* p, cudaStream_t st);
 cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st);
 cudaError_t ffk_exchange_inverse(ff_plan* p, void* out, cudaStream_t st);

@@ -283,9 +283,9 @@ __device__ __forceinline__ void attend_range(const KT* __restrict__ Kp, const KT
 }
 
 template <typename ST, int DPL>
-__global__ void __launch_bounds__(ATT_WARPS * 32) attention_simt_kernel(FFBuffers buf, FFDims dm) {
+__global__ void __launch_bounds__(ATT_WARPS * 32) attention_simt_kernel(FFBuffers buf, FFDims dm, int band_bits) {
   const int band = blockIdx.z, bh = blockIdx.y;
-  if (!(buf.alloc[bh] & (1 << band))) return;
+  if (!(buf.alloc[bh] & band_bits & (1 << band))) return;
   const long long n = band == 0 ? dm.Nbar : (band == 1 ? dm.Nmid : dm.Nhigh);
   const long long p = (long long)blockIdx.x * ATT_WARPS + (threadIdx.x >> 5);
   if (p >= n) return;
@@ -521,23 +521,26 @@ cudaError_t ffk_pool_low(ff_plan* p, cudaStream_t st) {
 }
 
 template <typename ST>
-static cudaError_t attention_simt_t(ff_plan* p, cudaStream_t st) {
+static cudaError_t attention_simt_t(ff_plan* p, int band_bits, cudaStream_t st) {
   const FFDims& dm = p->dm;
-  long long nmax = dm.Nhigh > dm.Nmid ? dm.Nhigh : dm.Nmid;
-  if (dm.Nbar > nmax) nmax = dm.Nbar;
-  dim3 grid((unsigned)((nmax + ATT_WARPS - 1) / ATT_WARPS), (unsigned)dm.BH, 3);
+  long long nmax = 0;
+  if ((band_bits & FF_BAND_LOW) && dm.Nbar > nmax) nmax = dm.Nbar;
+  if ((band_bits & FF_BAND_MID) && dm.Nmid > nmax) nmax = dm.Nmid;
+  if ((band_bits & FF_BAND_HIGH) && dm.Nhigh > nmax) nmax = dm.Nhigh;
+  const int zdim = (band_bits & FF_BAND_HIGH) ? 3 : ((band_bits & FF_BAND_MID) ? 2 : 1);
+  dim3 grid((unsigned)((nmax + ATT_WARPS - 1) / ATT_WARPS), (unsigned)dm.BH, zdim);
   switch (dm.d / 32) {
-    case 1: attention_simt_kernel<ST, 1><<<grid, ATT_WARPS * 32, 0, st>>>(p->buf, dm); break;
-    case 2: attention_simt_kernel<ST, 2><<<grid, ATT_WARPS * 32, 0, st>>>(p->buf, dm); break;
-    case 3: attention_simt_kernel<ST, 3><<<grid, ATT_WARPS * 32, 0, st>>>(p->buf, dm); break;
-    default: attention_simt_kernel<ST, 4><<<grid, ATT_WARPS * 32, 0, st>>>(p->buf, dm); break;
+    case 1: attention_simt_kernel<ST, 1><<<grid, ATT_WARPS * 32, 0, st>>>(p->buf, dm, band_bits); break;
+    case 2: attention_simt_kernel<ST, 2><<<grid, ATT_WARPS * 32, 0, st>>>(p->buf, dm, band_bits); break;
+    case 3: attention_simt_kernel<ST, 3><<<grid, ATT_WARPS * 32, 0, st>>>(p->buf, dm, band_bits); break;
+    default: attention_simt_kernel<ST, 4><<<grid, ATT_WARPS * 32, 0, st>>>(p->buf, dm, band_bits); break;
   }
   p->launches += 1;
   return cudaGetLastError();
 }
 
-cudaError_t ffk_attention_simt(ff_plan* p, cudaStream_t st) {
-  return p->dm.fp32 ? attention_simt_t<float>(p, st) : attention_simt_t<__nv_bfloat16>(p, st);
+cudaError_t ffk_attention_simt(ff_plan* p, int band_bits, cudaStream_t st) {
+  return p->dm.fp32 ? attention_simt_t<float>(p, band_bits, st) : attention_simt_t<__nv_bfloat16>(p, band_bits, st);
 }
 
 cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st) {
