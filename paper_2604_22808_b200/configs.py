@@ -83,13 +83,13 @@ G128K = _make("128k_sweep", 2, (32, 64, 64), 24, 128, "bf16", (1, 8), 8, 64, 8, 
 CONFIGS = (TINY, G64K, G256K, G1M, G128K)
 BY_NAME = {c.name: c for c in CONFIGS}
 
-# Scaled-down replicas (same operator parameters, grids of 4K-16K tokens, fewer heads) on which
+# Scaled-down replicas (same operator parameters, grids of 8K-16K tokens, axis lengths the tensor-core transform covers, fewer heads) on which
 # the fp64 oracle can run every stage in full within seconds.
-R64K = _make("64k_replica", 1, (8, 32, 32), 6, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 11, (800,))
-R256K = _make("256k_replica", 1, (8, 32, 32), 6, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 12, (200,),
+R64K = _make("64k_replica", 1, (16, 32, 32), 6, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 11, (800,))
+R256K = _make("256k_replica", 1, (16, 32, 32), 6, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 12, (200,),
               smooth_cosines=8, smooth_amplitude=3.0)
 R1M = _make("1m_replica", 1, (16, 32, 32), 4, 128, "bf16", (1, 16), 16, 128, 16, 512, 32, 13, (500,))
-R128K = _make("128k_replica", 2, (8, 32, 16), 6, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 14,
+R128K = _make("128k_replica", 2, (16, 32, 16), 6, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 14,
               (999, 750, 500, 250, 1))
 
 REPLICAS = (R64K, R256K, R1M, R128K)

@@ -245,6 +245,14 @@ extern "C" ff_status_t ff_plan_set_workspace(ff_plan_t* p, void* ptr, size_t byt
   b.work = (int*)(base + o[19]);
   FF_CUDA(p, cudaMemset(b.status, 0, 256));
   p->tc_ok = ffk_tc_supported(p->dm) && ffk_tc_prepare(p);
+  // The tensor-core transform shares the scratch region (scratchA and scratchB are adjacent).
+  p->dct_tc_ok = false;
+  if (ffk_dct_tc_supported(p->dm)) {
+    const size_t room = (size_t)((char*)base + o[14] - (char*)b.scratchA) + (size_t)p->lay.group * p->dm.N * p->dm.d * 4;
+    int G = 3 * p->dm.BH < 3 ? 3 * p->dm.BH : 3;
+    while (G > 1 && ffk_dct_tc_scratch_bytes(p->dm, G) > room) --G;
+    if (ffk_dct_tc_scratch_bytes(p->dm, G) <= room) { p->dct_tc_ok = true; p->dct_group = G; }
+  }
   return FF_OK;
 }
 
@@ -252,7 +260,7 @@ extern "C" const char* ff_last_error(const ff_plan_t* p) { return p ? p->err : g
 
 extern "C" ff_status_t ff_plan_set_attention_impl(ff_plan_t* p, int32_t impl) {
   if (!p) return fail(nullptr, FF_ERR_INVALID_ARG, "plan is NULL%s");
-  if (impl < 0 || impl > 1) return fail(p, FF_ERR_INVALID_ARG, "attention impl must be 0 or 1%s");
+  if (impl < 0 || impl > 3) return fail(p, FF_ERR_INVALID_ARG, "impl must be in [0, 3]%s");
   p->attn_impl = impl;
   return FF_OK;
 }
@@ -317,14 +325,18 @@ static cudaError_t mark(ff_plan* p, int boundary, cudaStream_t st) {
 static ff_status_t transform_and_route(ff_plan* p, const void* Q, const void* K, const void* V, const float* timestep,
                                        bool route, cudaStream_t st) {
   FF_CUDA(p, mark(p, 0, st));
-  FF_CUDA(p, ffk_forward_transform(p, Q, K, V, st));
-  FF_CUDA(p, mark(p, 1, st));
   if (route) {
     if (!p->has_router) return fail(p, FF_ERR_NOT_ROUTED, "the plan was created without router weights%s");
     if (!timestep) return fail(p, FF_ERR_NOT_ROUTED, "neither an allocation nor a timestep was given%s");
     FF_CUDA(p, cudaMemcpyAsync(p->buf.timestep, timestep, sizeof(float) * p->dm.B, cudaMemcpyHostToDevice, st));
     FF_CUDA(p, cudaMemsetAsync(p->buf.energy, 0, sizeof(double) * p->dm.B * 3 * p->dm.d, st));
-    FF_CUDA(p, ffk_band_energy(p, st));
+  }
+  const bool tc_transform = p->dct_tc_ok && !(p->attn_impl & 2);
+  if (tc_transform) FF_CUDA(p, ffk_forward_transform_tc(p, Q, K, V, route, st));   // band energies come from its epilogue
+  else FF_CUDA(p, ffk_forward_transform(p, Q, K, V, st));
+  FF_CUDA(p, mark(p, 1, st));
+  if (route) {
+    if (!tc_transform) FF_CUDA(p, ffk_band_energy(p, st));
     FF_CUDA(p, ffk_router(p, p->buf.alloc, st));
   }
   FF_CUDA(p, mark(p, 2, st));
@@ -360,7 +372,7 @@ extern "C" ff_status_t ff_forward(ff_plan_t* p, const void* Q, const void* K, co
   if (s != FF_OK) return s;
   if (alloc_dev) FF_CUDA(p, cudaMemcpyAsync(p->buf.alloc, alloc_dev, p->dm.BH, cudaMemcpyDeviceToDevice, st));
   FF_CUDA(p, ffk_pool_low(p, st));
-  if (p->tc_ok && p->attn_impl == 0) {
+  if (p->tc_ok && !(p->attn_impl & 1)) {
     FF_CUDA(p, ffk_attention_simt(p, FF_BAND_LOW, st));
     FF_CUDA(p, ffk_attention_tc(p, st));
   } else {

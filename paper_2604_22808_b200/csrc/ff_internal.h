@@ -93,6 +93,8 @@ struct ff_plan {
   int attn_impl;
   int sm_count;
   bool tc_ok;                                  // tensor-core attention usable with this plan + workspace
+  bool dct_tc_ok;                              // tensor-core transform usable
+  int dct_group;                               // tensor-heads per tensor-core transform launch
   alignas(64) unsigned char tmap_mid[128];     // CUtensorMap over the mid-band / high-band coefficient buffers
   alignas(64) unsigned char tmap_high[128];
   long long launches;
@@ -115,5 +117,11 @@ size_t ffk_tc_work_bytes();
 bool ffk_tc_supported(const FFDims& dm);
 bool ffk_tc_prepare(ff_plan* p);               // builds the tensor maps over the workspace
 cudaError_t ffk_attention_tc(ff_plan* p, cudaStream_t st);
+// ---- tensor-core transform (ff_dct_tc.cu) --------------------------------------------------------
+bool ffk_dct_tc_supported(const FFDims& dm);
+size_t ffk_dct_tc_scratch_bytes(const FFDims& dm, int group);
+cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, const void* V, bool want_energy,
+                                     cudaStream_t st);
+cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaStream_t st);
 cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st);
 cudaError_t ffk_exchange_inverse(ff_plan* p, void* out, cudaStream_t st);

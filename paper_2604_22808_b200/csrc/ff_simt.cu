@@ -399,9 +399,9 @@ __global__ void summary_kernel(FFBuffers buf, const float* U, FFDims dm) {
 // tokens of the other two bands, and write the row at its coefficient position (fp32 grid).
 constexpr int EXC_WARPS = 8;
 
-template <typename ST, int DPL>
+template <typename ST, int DPL, typename OT>
 __global__ void __launch_bounds__(EXC_WARPS * 32) exchange_recombine_kernel(FFBuffers buf, FFDims dm, int bh0,
-                                                                             float* grid_out) {
+                                                                             OT* grid_out, OT* grid_lo) {
   extern __shared__ float S[];   // [3][m][d]
   const int gi = blockIdx.y, bh = bh0 + gi;
   const int d = dm.d, m = dm.m;
@@ -443,9 +443,16 @@ __global__ void __launch_bounds__(EXC_WARPS * 32) exchange_recombine_kernel(FFBu
 #pragma unroll
     for (int j = 0; j < DPL; ++j) acc[j] /= den;
   }
-  float* dst = grid_out + ((size_t)gi * dm.N + f) * d;
+  // With a second grid the value is stored as a hi/lo pair (hi = rounded value, lo = rounded
+  // remainder): a band's tokens share almost the same exchange offset, so a single rounding would
+  // bias whole bands coherently and the inverse transform would focus that bias on a few tokens.
+  OT* dst = grid_out + ((size_t)gi * dm.N + f) * d;
 #pragma unroll
-  for (int j = 0; j < DPL; ++j) dst[lane + 32 * j] = y[j] + acc[j];
+  for (int j = 0; j < DPL; ++j) {
+    const float v = y[j] + acc[j];
+    stf<OT>(dst + lane + 32 * j, v);
+    if (grid_lo) stf<OT>(grid_lo + ((size_t)gi * dm.N + f) * d + lane + 32 * j, v - ldf<OT>(dst + lane + 32 * j));
+  }
 }
 
 }  // namespace
@@ -553,6 +560,29 @@ cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// Tensor-core inverse: exchange + recombination into a bf16 grid, then the three axis passes.
+static cudaError_t exchange_inverse_tc(ff_plan* p, void* out, cudaStream_t st) {
+  const FFDims& dm = p->dm;
+  const int G = p->dct_group;
+  const size_t smem = (size_t)3 * dm.m * dm.d * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(exchange_recombine_kernel<__nv_bfloat16, 4, __nv_bfloat16>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  for (int h0 = 0; h0 < dm.BH; h0 += G) {
+    const int g = (dm.BH - h0 < G) ? dm.BH - h0 : G;
+    dim3 grid((unsigned)((dm.N + EXC_WARPS - 1) / EXC_WARPS), (unsigned)g);
+    const size_t grid_bytes = ((size_t)G * dm.N * dm.d * 2 + 255) / 256 * 256;
+    exchange_recombine_kernel<__nv_bfloat16, 4, __nv_bfloat16><<<grid, EXC_WARPS * 32, smem, st>>>(
+        p->buf, dm, h0, (__nv_bfloat16*)p->buf.scratchA, (__nv_bfloat16*)((char*)p->buf.scratchA + grid_bytes));
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    p->launches += 1;
+    e = ffk_inverse_transform_tc(p, h0, g, out, st);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
 template <typename ST>
 static cudaError_t exchange_inverse_t(ff_plan* p, void* out, cudaStream_t st) {
   const FFDims& dm = p->dm;
@@ -565,8 +595,8 @@ static cudaError_t exchange_inverse_t(ff_plan* p, void* out, cudaStream_t st) {
     dim3 grid((unsigned)((dm.N + EXC_WARPS - 1) / EXC_WARPS), (unsigned)g);
     cudaError_t e = cudaSuccess;
 #define FF_EXC(DPL)                                                                                                   \
-  e = cudaFuncSetAttribute(exchange_recombine_kernel<ST, DPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-  if (e == cudaSuccess) exchange_recombine_kernel<ST, DPL><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, dm, h0, p->buf.scratchA);
+  e = cudaFuncSetAttribute(exchange_recombine_kernel<ST, DPL, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+  if (e == cudaSuccess) exchange_recombine_kernel<ST, DPL, float><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, dm, h0, p->buf.scratchA, (float*)nullptr);
     switch (dm.d / 32) {
       case 1: FF_EXC(1) break;
       case 2: FF_EXC(2) break;
@@ -597,5 +627,6 @@ static cudaError_t exchange_inverse_t(ff_plan* p, void* out, cudaStream_t st) {
 }
 
 cudaError_t ffk_exchange_inverse(ff_plan* p, void* out, cudaStream_t st) {
+  if (p->dct_tc_ok && !(p->attn_impl & 2)) return exchange_inverse_tc(p, out, st);
   return p->dm.fp32 ? exchange_inverse_t<float>(p, out, st) : exchange_inverse_t<__nv_bfloat16>(p, out, st);
 }
