@@ -91,9 +91,9 @@ static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 void ff_compute_layout(const FFDims& dm, bool with_staging, FFLayout* lay) {
   const size_t e = dm.fp32 ? 4 : 2;
   const size_t d = dm.d, BH = dm.BH;
-  // Tensor-heads per transform launch: as many as fit two fp32 scratch grids of ~4 GiB each.
+  // Tensor-heads per generic transform launch: as many as fit two fp32 scratch grids of ~1 GiB each.
   const size_t per = (size_t)dm.N * d * 4;
-  size_t G = ((size_t)4 << 30) / per;
+  size_t G = ((size_t)1 << 30) / per;
   if (G < 1) G = 1;
   if (G > 3 * BH) G = 3 * BH;
   lay->group = (int)G;

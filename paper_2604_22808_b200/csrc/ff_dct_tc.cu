@@ -237,17 +237,27 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
           tmem_ld16(tm + lane_addr + ab * 128 + l * n + a0, r);
           tmem_wait_ld();
           if (P.mode == MODE_SPLIT) {
+            // Band and rank of (k_t, h, w) for k_t = a0 .. a0+15 from per-line constants: along k_t
+            // the counts of box members below the coefficient are piecewise linear.
             const int tensor = th / dm.BH, bh = th % dm.BH;
+            const bool hw_low = h < dm.L[1] && w < dm.L[2], hw_mid = h < dm.M[1] && w < dm.M[2];
+            const int Lhw = dm.L[1] * dm.L[2], Mhw = dm.M[1] * dm.M[2];
+            const int offL = (h < dm.L[1] ? h : dm.L[1]) * dm.L[2] + (h < dm.L[1] ? (w < dm.L[2] ? w : dm.L[2]) : 0);
+            const int offM = (h < dm.M[1] ? h : dm.M[1]) * dm.M[2] + (h < dm.M[1] ? (w < dm.M[2] ? w : dm.M[2]) : 0);
+            __nv_bfloat16* mid_base = P.spec_mid + ((size_t)tensor * dm.BH + bh) * dm.Nmid * CH + c;
+            __nv_bfloat16* high_base = P.spec_high + ((size_t)tensor * dm.BH + bh) * dm.Nhigh * CH + c;
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
               const float v = __uint_as_float(r[i]);
-              long long rank;
-              const int band = ff_band_rank_of(dm, a0 + i, h, w, &rank);          // axis 0: a = k_t
-              if (band == 1) {
-                P.spec_mid[(((size_t)tensor * dm.BH + bh) * dm.Nmid + rank) * CH + c] = __float2bfloat16_rn(v);
+              const int kt = a0 + i;
+              const long long cl = kt < dm.L[0] ? (long long)kt * Lhw + offL : dm.Nlow;
+              const long long cm = kt < dm.M[0] ? (long long)kt * Mhw + offM : (long long)dm.M[0] * Mhw;
+              if (kt < dm.L[0] && hw_low) continue;                                   // low band: fp32 path
+              if (kt < dm.M[0] && hw_mid) {
+                mid_base[(cm - cl) * CH] = __float2bfloat16_rn(v);
                 e_mid = fmaf(v, v, e_mid);
-              } else if (band == 2) {
-                P.spec_high[(((size_t)tensor * dm.BH + bh) * dm.Nhigh + rank) * CH + c] = __float2bfloat16_rn(v);
+              } else {
+                high_base[((((long long)kt * dm.H + h) * dm.W + w) - cm) * CH] = __float2bfloat16_rn(v);
                 e_high = fmaf(v, v, e_high);
               }
             }
@@ -301,39 +311,59 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
 
 // Low band at full precision from the fp32 copy of the w-transformed columns k_w < L_w:
 //   low[k_t][k_h][k_w][c] = sum_t C_T[k_t][t] sum_h C_H[k_h][h] side[t][h][k_w][c]
-// One CTA per (tensor-head, k_h, k_w), one thread per channel; also the low band's energy.
+// One CTA per (tensor-head, k_h, k_w); thread = (t group, channel); the t groups are combined through
+// shared memory.  Also accumulates the low band's energy.
 constexpr int LOW_MAX_LT = 16;
+constexpr int LOW_TG = 8;
 
-__global__ void __launch_bounds__(CH) low_band_kernel(const float* side, const float* CT, const float* CHm, float* spec_low,
-                                                      double* energy, FFDims dm, int group_start) {
+__global__ void __launch_bounds__(CH * LOW_TG) low_band_kernel(const float* side, const float* CT, const float* CHm,
+                                                               float* spec_low, double* energy, FFDims dm, int group_start) {
   const int kw = blockIdx.x % dm.L[2], kh = blockIdx.x / dm.L[2];
   const int gi = blockIdx.y, th = group_start + gi;
-  const int c = threadIdx.x;
+  const int c = threadIdx.x % CH, tg = threadIdx.x / CH;
   __shared__ float ch_row[128];
-  for (int i = threadIdx.x; i < dm.H; i += CH) ch_row[i] = CHm[(size_t)kh * dm.H + i];
-  __syncthreads();
+  __shared__ float red[LOW_MAX_LT][CH];
+  for (int i = threadIdx.x; i < dm.H; i += CH * LOW_TG) ch_row[i] = CHm[(size_t)kh * dm.H + i];
   float e = 0.f;
   for (int kt0 = 0; kt0 < dm.L[0]; kt0 += LOW_MAX_LT) {
+    for (int i = threadIdx.x; i < LOW_MAX_LT * CH; i += CH * LOW_TG) red[i / CH][i % CH] = 0.f;
+    __syncthreads();
     float acc[LOW_MAX_LT];
 #pragma unroll
     for (int i = 0; i < LOW_MAX_LT; ++i) acc[i] = 0.f;
-    for (int t = 0; t < dm.T; ++t) {
+    for (int t = tg; t < dm.T; t += LOW_TG) {
       const float* col = side + ((((size_t)gi * dm.T + t) * dm.H) * dm.L[2] + kw) * CH + c;
-      float s = 0.f;
-      for (int h = 0; h < dm.H; ++h) s = fmaf(ch_row[h], col[(size_t)h * dm.L[2] * CH], s);
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+      int h = 0;
+      for (; h + 3 < dm.H; h += 4) {
+        s0 = fmaf(ch_row[h], col[(size_t)h * dm.L[2] * CH], s0);
+        s1 = fmaf(ch_row[h + 1], col[(size_t)(h + 1) * dm.L[2] * CH], s1);
+        s2 = fmaf(ch_row[h + 2], col[(size_t)(h + 2) * dm.L[2] * CH], s2);
+        s3 = fmaf(ch_row[h + 3], col[(size_t)(h + 3) * dm.L[2] * CH], s3);
+      }
+      for (; h < dm.H; ++h) s0 = fmaf(ch_row[h], col[(size_t)h * dm.L[2] * CH], s0);
+      const float sh_ = (s0 + s1) + (s2 + s3);
 #pragma unroll
       for (int i = 0; i < LOW_MAX_LT; ++i)
-        if (kt0 + i < dm.L[0]) acc[i] = fmaf(CT[(size_t)(kt0 + i) * dm.T + t], s, acc[i]);
+        if (kt0 + i < dm.L[0]) acc[i] = fmaf(CT[(size_t)(kt0 + i) * dm.T + t], sh_, acc[i]);
     }
 #pragma unroll
-    for (int i = 0; i < LOW_MAX_LT; ++i) {
-      if (kt0 + i >= dm.L[0]) break;
-      const long long rank = ((long long)(kt0 + i) * dm.L[1] + kh) * dm.L[2] + kw;
-      spec_low[((size_t)th * dm.Nlow + rank) * CH + c] = acc[i];
-      e = fmaf(acc[i], acc[i], e);
+    for (int i = 0; i < LOW_MAX_LT; ++i)
+      if (kt0 + i < dm.L[0]) atomicAdd(&red[i][c], acc[i]);
+    __syncthreads();
+    if (tg == 0) {
+#pragma unroll
+      for (int i = 0; i < LOW_MAX_LT; ++i) {
+        if (kt0 + i >= dm.L[0]) break;
+        const long long rank = ((long long)(kt0 + i) * dm.L[1] + kh) * dm.L[2] + kw;
+        const float v = red[i][c];
+        spec_low[((size_t)th * dm.Nlow + rank) * CH + c] = v;
+        e = fmaf(v, v, e);
+      }
     }
+    __syncthreads();
   }
-  if (energy) atomicAdd(energy + ((size_t)((th % dm.BH) / dm.heads) * 3) * CH + c, (double)e);
+  if (energy && tg == 0) atomicAdd(energy + ((size_t)((th % dm.BH) / dm.heads) * 3) * CH + c, (double)e);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -439,7 +469,7 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
     e = launch_pass(p, m2h, m2l, m2l, P, st);
     if (e != cudaSuccess) return e;
     dim3 lgrid((unsigned)(dm.L[1] * dm.L[2]), (unsigned)g);
-    low_band_kernel<<<lgrid, CH, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
+    low_band_kernel<<<lgrid, CH * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
     p->launches += 1;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
