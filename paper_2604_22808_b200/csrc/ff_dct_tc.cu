@@ -1,25 +1,27 @@
 // Separable transform on the tensor cores ("Separable spectral decomposition", "Reconstruction"),
-// bf16 storage, head_dim 128.  Every axis pass is the same batched contraction: for one line of n
-// grid positions along the axis (all other coordinates fixed),
-//     D[c][a] = sum_b X[b][c] * Mat[a][b]          c = channel (128), a = output index, b = input index
-// The data tile X (n rows of 128 channels, 256 bytes each) is the A operand, taken straight from a
-// TMA box in shared memory as an MN-major matrix (M = channels), the transform matrix is the
-// K-major B operand, and the 128 x n fp32 result sits in tensor memory with one channel per lane.
+// bf16 storage, head_dim 128.  Every axis pass is a batched contraction over "lines" of n grid
+// positions along the axis (all other coordinates fixed): out[a][c] = sum_b Mat[a][b] in[b][c].
+// A CTA works on tiles of 128 grid positions = 128/n adjacent lines, fetched by one TMA box per
+// 64-channel half (a contiguous run of memory for the w axis; 128/n neighbouring w positions per
+// axis position for the h and t axes, so that the strided axes also read contiguous pieces).
+// One tile is one 128 x 128 x 128 contraction
+//     D[j][c] = sum_r A[j][r] * X[r][c],   A = Mat kron I (or I kron Mat) over the lines of the tile
+// with A the K-major operand built once per CTA in shared memory, X the TMA tile used in place as
+// the MN-major B operand, and D in tensor memory with one output position per lane, so that an
+// epilogue thread owns a whole 256-byte output row and stores it with 16-byte accesses.
+//
 // Precision: the transform matrix is split into bf16 hi + lo parts, and so is every intermediate
 // between two axis passes (two bf16 grids, hi = bf16(v), lo = bf16(v - hi)); a pass then issues
-// X_hi*C_hi + X_hi*C_lo + X_lo*C_hi per k-step.  Intermediates can be far larger than the final
+// C_hi*X_hi + C_lo*X_hi + C_hi*X_lo per k-step.  Intermediates can be far larger than the final
 // values (low-frequency content, the constant offset the exchange adds to a whole band), so a
 // single bf16 rounding between passes would not meet the output tolerance.
 //
-// A CTA is persistent over "stages" of LPS consecutive lines (LPS * n = 128 rows; 32 KB of bf16
-// input, or 64 KB when the input is a hi/lo pair).
 //   warp 0      TMA producer (ring of 2-4 stages, as many as fit beside the matrix images)
 //   warp 1      tcgen05.mma issuer, 4 accumulator buffers of 128 TMEM columns
-//   warps 2..5  epilogue: tcgen05.ld, convert, store (thread = channel, so a warp writes 32
-//               consecutive channels of one output position per instruction)
-// Modes: FIRST  caller's Q/K/V -> hi/lo intermediate, plus an fp32 copy of the columns k_w < L_w
+//   warps 2..5  epilogue: tcgen05.ld, convert, store
+// Modes: FIRST  caller's Q/K/V -> hi/lo intermediate, plus an fp32 copy of the rows k_w < L_w
 //               from which the low band is computed at full precision
-//        MIDDLE intermediate (hi/lo, or a single bf16 grid) -> hi/lo intermediate
+//        MIDDLE hi/lo intermediate -> hi/lo intermediate
 //        SPLIT  intermediate -> band-major mid/high coefficient buffers (rank evaluated in
 //               registers) with the router's band energies accumulated from the fp32 accumulators
 //        LAST   intermediate -> the caller's out tensor
@@ -33,8 +35,9 @@ using namespace sm100;
 namespace {
 
 constexpr int CH = 128;
-constexpr int STAGE_ROWS = 128;
-constexpr int TILE_BYTES = STAGE_ROWS * CH * 2;    // 32 KB: 128 rows of bf16
+constexpr int TILE_ROWS = 128;
+constexpr int TILE_BYTES = TILE_ROWS * CH * 2;     // 32 KB: 128 rows of bf16
+constexpr int HALF_BYTES = TILE_BYTES / 2;
 constexpr int MAX_STAGE = 4;
 constexpr int NACC = 4;
 constexpr int DCT_TC_THREADS = 192;
@@ -49,7 +52,6 @@ struct DctTcParams {
   int mode;
   int group;               // tensor-heads in this launch
   int group_start;         // index of the first one (tensor * BH + bh for the forward, bh for the inverse)
-  int lines_per_th;        // lines per tensor-head = N / n
   int in_split;            // input is a hi/lo pair of grids (map0 = hi, map1 = lo)
   int nstage;              // ring depth
   __nv_bfloat16* dst;      // hi grid [group][T][H][W][128], or the out tensor (MODE_LAST)
@@ -66,11 +68,12 @@ struct DctShared {
   int abort_flag;
 };
 
-// Coordinates (w, h, t) of the first position of line `line` of a tensor-head, for the given axis.
-__device__ __forceinline__ void line_origin(const FFDims& dm, int axis, int line, int& w, int& h, int& t) {
-  if (axis == 2) { w = 0; h = line % dm.H; t = line / dm.H; }
-  else if (axis == 1) { h = 0; w = line % dm.W; t = line / dm.W; }
-  else { t = 0; w = line % dm.W; h = line / dm.W; }
+// Grid coordinates (w, h, t) of the first position of tile `u` of a tensor-head.  A tile holds
+// kf = 128/n lines: kf consecutive h for the w axis, kf consecutive w for the h and t axes.
+__device__ __forceinline__ void tile_origin(const FFDims& dm, int axis, int kf, int u, int& w, int& h, int& t) {
+  if (axis == 2) { const int q = dm.H / kf; w = 0; h = (u % q) * kf; t = u / q; }
+  else if (axis == 1) { const int q = dm.W / kf; h = 0; w = (u % q) * kf; t = u / q; }
+  else { const int q = dm.W / kf; t = 0; w = (u % q) * kf; h = u / q; }
 }
 
 __device__ __forceinline__ void tma_load_5d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2,
@@ -78,16 +81,6 @@ __device__ __forceinline__ void tma_load_5d(void* smem_dst, const CUtensorMap* m
   asm volatile(
       "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
       ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-      : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
       : "memory");
 }
 
@@ -99,17 +92,19 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const FFDims& dm = P.dm;
   const int n = P.n;
+  const int kf = TILE_ROWS / n;                           // lines per tile
+  const int lkf = 31 - __clz(kf);
+  const int ln = 31 - __clz(n);
+  const bool seq = P.axis == 2;                           // lines follow one another (w axis) or interleave
   const int NSTAGE = P.nstage;
   const int STAGE_BYTES = P.in_split ? 2 * TILE_BYTES : TILE_BYTES;
-  const int img_bytes = (n > 64 ? 2 : 1) * n * 128;       // one matrix image
   uint8_t* sData = smem;                                  // NSTAGE x STAGE_BYTES
-  uint8_t* sHi = smem + NSTAGE * STAGE_BYTES;             // basis hi: [half][n rows][128 B], swizzled
-  uint8_t* sLo = sHi + img_bytes;                         // basis lo
-  DctShared& sh = *(DctShared*)(sLo + img_bytes);
-  const int lps = STAGE_ROWS / n;                         // lines per stage
+  uint8_t* sHi = smem + NSTAGE * STAGE_BYTES;             // matrix hi: [K half][128 rows][128 B], swizzled
+  uint8_t* sLo = sHi + TILE_BYTES;                        // matrix lo
+  DctShared& sh = *(DctShared*)(sLo + TILE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_lines = P.group * P.lines_per_th;
-  const int total_stages = (total_lines + lps - 1) / lps;
+  const int tiles_per_th = (int)(dm.N / TILE_ROWS);
+  const int total_tiles = P.group * tiles_per_th;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NSTAGE; ++i) { mbar_init(&sh.full[i], 1); mbar_init(&sh.empty[i], 1); }
@@ -117,15 +112,19 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     sh.abort_flag = 0;
     fence_mbar_init();
   }
-  // Transform matrix as the K-major B operand: row a = output index, 64 input indices per 128-byte
-  // row, 16-byte chunks XOR-swizzled with the row index (the 128-byte swizzle the MMA expects).
-  for (int idx = threadIdx.x; idx < n * n; idx += DCT_TC_THREADS) {
-    const int a = idx / n, b = idx % n;
-    const float v = P.mat[idx];
+  // Matrix image, the K-major A operand: row j = output position of the tile, 64 input positions per
+  // 128-byte row, 16-byte chunks XOR-swizzled with the row index (the 128-byte swizzle the MMA
+  // expects).  Lines that follow one another (w axis): I kron Mat, index = line*n + a.  Interleaved
+  // lines (h, t axes): Mat kron I, index = a*kf + line.
+  for (int idx = threadIdx.x; idx < TILE_ROWS * TILE_ROWS; idx += DCT_TC_THREADS) {
+    const int j = idx >> 7, r = idx & 127;
+    float v;
+    if (seq) v = ((j >> ln) == (r >> ln)) ? P.mat[(j & (n - 1)) * n + (r & (n - 1))] : 0.f;
+    else v = ((j & (kf - 1)) == (r & (kf - 1))) ? P.mat[(j >> lkf) * n + (r >> lkf)] : 0.f;
     const __nv_bfloat16 hi = __float2bfloat16_rn(v);
     const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-    const int half = b >> 6, bk = b & 63;
-    const uint32_t off = half * (n * 128) + a * 128 + ((((bk >> 3) ^ (a & 7)) << 4) | ((bk & 7) << 1));
+    const int half = r >> 6, rk = r & 63;
+    const uint32_t off = half * HALF_BYTES + j * 128 + ((((rk >> 3) ^ (j & 7)) << 4) | ((rk & 7) << 1));
     *(__nv_bfloat16*)(sHi + off) = hi;
     *(__nv_bfloat16*)(sLo + off) = lo;
   }
@@ -136,65 +135,58 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tm = sh.tmem_base;
   volatile int* abort_flag = &sh.abort_flag;
-  const int half_stride = lps * n * 128;                  // bytes between the two 64-channel halves of a stage (= 16 KB)
 
   if (warp == 0) {
     if (lane == 0) {
       tma_prefetch_desc(&map0);
       unsigned it = 0;
       bool ok = true;
-      for (int s = blockIdx.x; s < total_stages && ok; s += gridDim.x, ++it) {
+      for (int s = blockIdx.x; s < total_tiles && ok; s += gridDim.x, ++it) {
         const int slot = it % NSTAGE;
-        if (it >= NSTAGE) ok = mbar_wait(&sh.empty[slot], ((it / NSTAGE) - 1) & 1, abort_flag);
+        if (it >= (unsigned)NSTAGE) ok = mbar_wait(&sh.empty[slot], ((it / NSTAGE) - 1) & 1, abort_flag);
         if (!ok) break;
         uint8_t* dst = sData + slot * STAGE_BYTES;
-        int nl = total_lines - s * lps; if (nl > lps) nl = lps;
-        mbar_arrive_expect_tx(&sh.full[slot], nl * n * 256 * (P.in_split ? 2 : 1));
-        for (int l = 0; l < nl; ++l) {
-          const int gl = s * lps + l;
-          const int gi = gl / P.lines_per_th, line = gl % P.lines_per_th;
-          int w, h, t; line_origin(dm, P.axis, line, w, h, t);
-          const CUtensorMap* map = &map0;
-          int slice = gi;
-          if (P.mode == MODE_FIRST) {
-            const int th = P.group_start + gi;
-            const int tensor = th / dm.BH;
-            map = tensor == 0 ? &map0 : (tensor == 1 ? &map1 : &map2);
-            slice = th % dm.BH;
-          }
-          tma_load_5d(dst + l * n * 128, map, &sh.full[slot], 0, w, h, t, slice);
-          tma_load_5d(dst + half_stride + l * n * 128, map, &sh.full[slot], 64, w, h, t, slice);
-          if (P.in_split) {
-            tma_load_5d(dst + TILE_BYTES + l * n * 128, &map1, &sh.full[slot], 0, w, h, t, slice);
-            tma_load_5d(dst + TILE_BYTES + half_stride + l * n * 128, &map1, &sh.full[slot], 64, w, h, t, slice);
-          }
+        const int gi = s / tiles_per_th, u = s % tiles_per_th;
+        int w, h, t; tile_origin(dm, P.axis, kf, u, w, h, t);
+        const CUtensorMap* map = &map0;
+        int slice = gi;
+        if (P.mode == MODE_FIRST) {
+          const int th = P.group_start + gi;
+          const int tensor = th / dm.BH;
+          map = tensor == 0 ? &map0 : (tensor == 1 ? &map1 : &map2);
+          slice = th % dm.BH;
+        }
+        mbar_arrive_expect_tx(&sh.full[slot], STAGE_BYTES);
+        tma_load_5d(dst, map, &sh.full[slot], 0, w, h, t, slice);
+        tma_load_5d(dst + HALF_BYTES, map, &sh.full[slot], 64, w, h, t, slice);
+        if (P.in_split) {
+          tma_load_5d(dst + TILE_BYTES, &map1, &sh.full[slot], 0, w, h, t, slice);
+          tma_load_5d(dst + TILE_BYTES + HALF_BYTES, &map1, &sh.full[slot], 64, w, h, t, slice);
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      const uint32_t idesc = idesc_bf16_f32(CH, n, /*a_mn_major=*/true, /*b_mn_major=*/false);
+      const uint32_t idesc = idesc_bf16_f32(TILE_ROWS, CH, /*a_mn_major=*/false, /*b_mn_major=*/true);
+      const uint32_t hi_base = smem_u32(sHi), lo_base = smem_u32(sLo);
       unsigned it = 0;
       bool ok = true;
-      for (int s = blockIdx.x; s < total_stages && ok; s += gridDim.x, ++it) {
+      for (int s = blockIdx.x; s < total_tiles && ok; s += gridDim.x, ++it) {
         const int slot = it % NSTAGE, ab = it % NACC;
         ok = mbar_wait(&sh.full[slot], (it / NSTAGE) & 1, abort_flag);
         if (ok && it >= NACC) ok = mbar_wait(&sh.acc_empty[ab], ((it / NACC) - 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        int nl = total_lines - s * lps; if (nl > lps) nl = lps;
         const uint32_t dbase = smem_u32(sData + slot * STAGE_BYTES);
-        for (int l = 0; l < nl; ++l) {
-          const uint32_t d_tm = tm + ab * 128 + l * n;
-          for (int ks = 0; ks < n / 16; ++ks) {
-            const uint64_t adesc = smem_desc_sw128(dbase + l * n * 128 + ks * 2048, half_stride, 1024);
-            const uint32_t boff = (ks >> 2) * (n * 128) + (ks & 3) * 32;
-            const uint64_t bhi = smem_desc_sw128(smem_u32(sHi) + boff, 16, 1024);
-            umma_ss(d_tm, adesc, bhi, idesc, ks > 0 ? 1u : 0u);
-            umma_ss(d_tm, adesc, smem_desc_sw128(smem_u32(sLo) + boff, 16, 1024), idesc, 1u);
-            if (P.in_split)
-              umma_ss(d_tm, smem_desc_sw128(dbase + TILE_BYTES + l * n * 128 + ks * 2048, half_stride, 1024), bhi, idesc, 1u);
-          }
+        const uint32_t d_tm = tm + ab * 128;
+#pragma unroll
+        for (int ks = 0; ks < TILE_ROWS / 16; ++ks) {
+          const uint32_t aoff = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+          const uint64_t ahi = smem_desc_sw128(hi_base + aoff, 16, 1024);
+          const uint64_t xhi = smem_desc_sw128(dbase + ks * 2048, HALF_BYTES, 1024);
+          umma_ss(d_tm, ahi, xhi, idesc, ks > 0 ? 1u : 0u);
+          umma_ss(d_tm, smem_desc_sw128(lo_base + aoff, 16, 1024), xhi, idesc, 1u);
+          if (P.in_split) umma_ss(d_tm, ahi, smem_desc_sw128(dbase + TILE_BYTES + ks * 2048, HALF_BYTES, 1024), idesc, 1u);
         }
         umma_commit(&sh.empty[slot]);
         umma_commit(&sh.acc_full[ab]);
@@ -202,97 +194,125 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     }
   } else {
     const int quarter = warp & 3;
-    const int c = quarter * 32 + lane;                    // channel of this thread
+    const int j = quarter * 32 + lane;                    // output position of this thread inside a tile
+    const int a = seq ? j & (n - 1) : j >> lkf;           // output index along the axis
+    const int l = seq ? j >> ln : j & (kf - 1);           // line of the tile
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const long long N_d = dm.N * CH;
     const long long axis_stride = (P.axis == 2 ? 1LL : (P.axis == 1 ? (long long)dm.W : (long long)dm.W * dm.H)) * CH;
-    float e_mid = 0.f, e_high = 0.f;
+    const long long line_stride = (P.axis == 2 ? (long long)dm.W : 1LL) * CH;   // between the lines of a tile
+    const long long row_off = (long long)a * axis_stride + (long long)l * line_stride;
+    const int Lhw = dm.L[1] * dm.L[2], Mhw = dm.M[1] * dm.M[2];
+    // lane k of a warp accumulates the energies of channels 32 q + k over the warp's rows
+    float em[4] = {0.f, 0.f, 0.f, 0.f}, eh[4] = {0.f, 0.f, 0.f, 0.f};
     int e_sample = -1;
     unsigned it = 0;
     bool ok = true;
-    for (int s = blockIdx.x; s < total_stages && ok; s += gridDim.x, ++it) {
+    auto flush_energy = [&]() {
+      if (e_sample >= 0 && P.energy) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          atomicAdd(P.energy + ((size_t)e_sample * 3 + 1) * CH + q * 32 + lane, (double)em[q]);
+          atomicAdd(P.energy + ((size_t)e_sample * 3 + 2) * CH + q * 32 + lane, (double)eh[q]);
+          em[q] = eh[q] = 0.f;
+        }
+      }
+    };
+    for (int s = blockIdx.x; s < total_tiles && ok; s += gridDim.x, ++it) {
       const int ab = it % NACC;
       ok = __all_sync(0xffffffffu, mbar_wait(&sh.acc_full[ab], (it / NACC) & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
-      int nl = total_lines - s * lps; if (nl > lps) nl = lps;
-      for (int l = 0; l < nl; ++l) {
-        const int gl = s * lps + l;
-        const int gi = gl / P.lines_per_th, line = gl % P.lines_per_th;
-        int w, h, t; line_origin(dm, P.axis, line, w, h, t);
-        const long long pos0 = (((long long)t * dm.H + h) * dm.W + w) * CH + c;     // first position of the line
-        const int th = P.group_start + gi;
-        if (P.mode == MODE_SPLIT) {
-          const int sample = (th % dm.BH) / dm.heads;
-          if (sample != e_sample) {
-            if (e_sample >= 0 && P.energy) {
-              atomicAdd(P.energy + ((size_t)e_sample * 3 + 1) * CH + c, (double)e_mid);
-              atomicAdd(P.energy + ((size_t)e_sample * 3 + 2) * CH + c, (double)e_high);
-            }
-            e_mid = e_high = 0.f; e_sample = sample;
-          }
+      const int gi = s / tiles_per_th, u = s % tiles_per_th;
+      int w, h, t; tile_origin(dm, P.axis, kf, u, w, h, t);
+      const long long pos0 = (((long long)t * dm.H + h) * dm.W + w) * CH;           // first position of the tile
+      const int th = P.group_start + gi;
+      const int tensor = th / dm.BH, bh = th % dm.BH;
+      // where this thread's row goes
+      __nv_bfloat16* row_hi = nullptr; __nv_bfloat16* row_lo = nullptr; float* row_f32 = nullptr;
+      int band = -1;
+      if (P.mode == MODE_SPLIT) {
+        const int sample = bh / dm.heads;
+        if (sample != e_sample) { flush_energy(); e_sample = sample; }
+        // Band and rank of coefficient (k_t = a, h, w + l): the counts of box members below it are
+        // piecewise linear in the coordinates.
+        const int kt = a, ww = w + l;
+        const bool hw_low = h < dm.L[1] && ww < dm.L[2], hw_mid = h < dm.M[1] && ww < dm.M[2];
+        const int offM = (h < dm.M[1] ? h : dm.M[1]) * dm.M[2] + (h < dm.M[1] ? (ww < dm.M[2] ? ww : dm.M[2]) : 0);
+        const long long cm = kt < dm.M[0] ? (long long)kt * Mhw + offM : (long long)dm.M[0] * Mhw;
+        if (kt < dm.L[0] && hw_low) {
+          band = 0;                                                                  // low band: fp32 path
+        } else if (kt < dm.M[0] && hw_mid) {
+          const int offL = (h < dm.L[1] ? h : dm.L[1]) * dm.L[2] + (h < dm.L[1] ? (ww < dm.L[2] ? ww : dm.L[2]) : 0);
+          const long long cl = kt < dm.L[0] ? (long long)kt * Lhw + offL : dm.Nlow;
+          band = 1;
+          row_hi = P.spec_mid + (((size_t)tensor * dm.BH + bh) * dm.Nmid + (cm - cl)) * CH;
+        } else {
+          band = 2;
+          row_hi = P.spec_high + (((size_t)tensor * dm.BH + bh) * dm.Nhigh + ((((long long)kt * dm.H + h) * dm.W + ww) - cm)) * CH;
         }
-        for (int a0 = 0; a0 < n; a0 += 16) {
-          uint32_t r[16];
-          tmem_ld16(tm + lane_addr + ab * 128 + l * n + a0, r);
-          tmem_wait_ld();
-          if (P.mode == MODE_SPLIT) {
-            // Band and rank of (k_t, h, w) for k_t = a0 .. a0+15 from per-line constants: along k_t
-            // the counts of box members below the coefficient are piecewise linear.
-            const int tensor = th / dm.BH, bh = th % dm.BH;
-            const bool hw_low = h < dm.L[1] && w < dm.L[2], hw_mid = h < dm.M[1] && w < dm.M[2];
-            const int Lhw = dm.L[1] * dm.L[2], Mhw = dm.M[1] * dm.M[2];
-            const int offL = (h < dm.L[1] ? h : dm.L[1]) * dm.L[2] + (h < dm.L[1] ? (w < dm.L[2] ? w : dm.L[2]) : 0);
-            const int offM = (h < dm.M[1] ? h : dm.M[1]) * dm.M[2] + (h < dm.M[1] ? (w < dm.M[2] ? w : dm.M[2]) : 0);
-            __nv_bfloat16* mid_base = P.spec_mid + ((size_t)tensor * dm.BH + bh) * dm.Nmid * CH + c;
-            __nv_bfloat16* high_base = P.spec_high + ((size_t)tensor * dm.BH + bh) * dm.Nhigh * CH + c;
+      } else {
+        const size_t o = (size_t)(P.mode == MODE_LAST ? th : gi) * N_d + pos0 + row_off;
+        row_hi = P.dst + o;
+        if (P.mode != MODE_LAST) row_lo = P.dst_lo + o;
+        if (P.mode == MODE_FIRST && a < dm.L[2]) row_f32 = P.side + ((((size_t)gi * dm.T + t) * dm.H + h + l) * dm.L[2] + a) * CH;
+      }
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float v = __uint_as_float(r[i]);
-              const int kt = a0 + i;
-              const long long cl = kt < dm.L[0] ? (long long)kt * Lhw + offL : dm.Nlow;
-              const long long cm = kt < dm.M[0] ? (long long)kt * Mhw + offM : (long long)dm.M[0] * Mhw;
-              if (kt < dm.L[0] && hw_low) continue;                                   // low band: fp32 path
-              if (kt < dm.M[0] && hw_mid) {
-                mid_base[(cm - cl) * CH] = __float2bfloat16_rn(v);
-                e_mid = fmaf(v, v, e_mid);
-              } else {
-                high_base[((((long long)kt * dm.H + h) * dm.W + w) - cm) * CH] = __float2bfloat16_rn(v);
-                e_high = fmaf(v, v, e_high);
-              }
+      for (int q = 0; q < 4; ++q) {
+        uint32_t r[32];
+        tmem_ld32(tm + lane_addr + ab * 128 + q * 32, r);
+        tmem_wait_ld();
+        if (row_f32) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            *(uint4*)(row_f32 + q * 32 + i * 4) = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+        }
+        if (P.mode == MODE_SPLIT && P.energy) {
+          // channel energies of this 32-channel chunk, summed over the warp's 32 rows with a
+          // halving butterfly: afterwards lane k holds the sum for channel 32 q + k
+          float sm_[32], sh_[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float v = __uint_as_float(r[i]);
+            const float v2 = v * v;
+            sm_[i] = band == 1 ? v2 : 0.f;
+            sh_[i] = band == 2 ? v2 : 0.f;
+          }
+#pragma unroll
+          for (int step = 16; step >= 1; step >>= 1) {
+            const bool upper = lane & step;
+#pragma unroll
+            for (int i = 0; i < step; ++i) {
+              const float keep_m = upper ? sm_[i + step] : sm_[i], send_m = upper ? sm_[i] : sm_[i + step];
+              const float keep_h = upper ? sh_[i + step] : sh_[i], send_h = upper ? sh_[i] : sh_[i + step];
+              sm_[i] = keep_m + __shfl_xor_sync(0xffffffffu, send_m, step);
+              sh_[i] = keep_h + __shfl_xor_sync(0xffffffffu, send_h, step);
             }
-          } else {
-            const size_t o0 = (size_t)(P.mode == MODE_LAST ? th : gi) * N_d + pos0 + (long long)a0 * axis_stride;
-            __nv_bfloat16* dst = P.dst + o0;
-            if (P.mode == MODE_LAST) {
+          }
+          em[q] += sm_[0]; eh[q] += sh_[0];
+        }
+        if (row_hi) {
+          uint32_t hi[16], lo[16];
 #pragma unroll
-              for (int i = 0; i < 16; ++i) dst[(long long)i * axis_stride] = __float2bfloat16_rn(__uint_as_float(r[i]));
-            } else {
-              __nv_bfloat16* dlo = P.dst_lo + o0;
+          for (int i = 0; i < 16; ++i) {
+            const float v0 = __uint_as_float(r[2 * i]), v1 = __uint_as_float(r[2 * i + 1]);
+            const __nv_bfloat162 hp = __floats2bfloat162_rn(v0, v1);
+            hi[i] = *(const uint32_t*)&hp;
+            const __nv_bfloat162 lp = __floats2bfloat162_rn(v0 - __uint_as_float(hi[i] << 16), v1 - __uint_as_float(hi[i] & 0xffff0000u));
+            lo[i] = *(const uint32_t*)&lp;
+          }
 #pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const float v = __uint_as_float(r[i]);
-                const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-                dst[(long long)i * axis_stride] = hi;
-                dlo[(long long)i * axis_stride] = __float2bfloat16_rn(v - __bfloat162float(hi));
-              }
-            }
-            if (P.mode == MODE_FIRST && a0 < dm.L[2]) {
-              float* sd = P.side + ((((size_t)gi * dm.T + t) * dm.H + h) * dm.L[2]) * CH + c;
+          for (int i = 0; i < 4; ++i) *(uint4*)(row_hi + q * 32 + i * 8) = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
+          if (row_lo) {
 #pragma unroll
-              for (int i = 0; i < 16; ++i)
-                if (a0 + i < dm.L[2]) sd[(size_t)(a0 + i) * CH] = __uint_as_float(r[i]);
-            }
+            for (int i = 0; i < 4; ++i) *(uint4*)(row_lo + q * 32 + i * 8) = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
           }
         }
       }
       tc_fence_before();
       mbar_arrive(&sh.acc_empty[ab]);
     }
-    if (P.mode == MODE_SPLIT && e_sample >= 0 && P.energy) {
-      atomicAdd(P.energy + ((size_t)e_sample * 3 + 1) * CH + c, (double)e_mid);
-      atomicAdd(P.energy + ((size_t)e_sample * 3 + 2) * CH + c, (double)e_high);
-    }
+    if (P.mode == MODE_SPLIT) flush_energy();
   }
 
   tc_fence_before();
@@ -370,7 +390,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// 5-D map over a [slices][T][H][W][128] bf16 grid whose box is one line along `axis`.
+// 5-D map over a [slices][T][H][W][128] bf16 grid whose box is one tile of 128 positions for a pass
+// along `axis`: 128/n whole lines that are neighbours in memory.
 bool encode_grid_map(CUtensorMap* map, const void* base, const FFDims& dm, int slices, int axis) {
   static EncodeTiledFn enc = nullptr;
   if (!enc) {
@@ -381,8 +402,11 @@ bool encode_grid_map(CUtensorMap* map, const void* base, const FFDims& dm, int s
   cuuint64_t dims[5] = {(cuuint64_t)CH, (cuuint64_t)dm.W, (cuuint64_t)dm.H, (cuuint64_t)dm.T, (cuuint64_t)slices};
   cuuint64_t strides[4] = {(cuuint64_t)CH * 2, (cuuint64_t)dm.W * CH * 2, (cuuint64_t)dm.H * dm.W * CH * 2,
                            (cuuint64_t)dm.N * CH * 2};
+  const int n = axis == 2 ? dm.W : (axis == 1 ? dm.H : dm.T);
+  const int kf = TILE_ROWS / n;
   cuuint32_t box[5] = {64, 1, 1, 1, 1};
-  box[1 + (2 - axis)] = (cuuint32_t)(axis == 2 ? dm.W : (axis == 1 ? dm.H : dm.T));
+  box[1 + (2 - axis)] = (cuuint32_t)n;
+  if (axis == 2) box[2] = (cuuint32_t)kf; else box[1] = (cuuint32_t)kf;
   cuuint32_t es[5] = {1, 1, 1, 1, 1};
   return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, es,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -391,7 +415,7 @@ bool encode_grid_map(CUtensorMap* map, const void* base, const FFDims& dm, int s
 
 cudaError_t launch_pass(ff_plan* p, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& m2, DctTcParams& P,
                         cudaStream_t st) {
-  const size_t img = (size_t)(P.n > 64 ? 2 : 1) * P.n * 128;
+  const size_t img = TILE_BYTES;
   const size_t stage = P.in_split ? 2 * TILE_BYTES : TILE_BYTES;
   const size_t fixed = 2 * img + sizeof(DctShared) + 1024;
   int nstage = (int)((220 * 1024 - fixed) / stage);
@@ -400,8 +424,7 @@ cudaError_t launch_pass(ff_plan* p, const CUtensorMap& m0, const CUtensorMap& m1
   const size_t smem = nstage * stage + fixed;
   cudaError_t e = cudaFuncSetAttribute(dct_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const int lps = STAGE_ROWS / P.n;
-  const int stages = (P.group * P.lines_per_th + lps - 1) / lps;
+  const int stages = (int)(P.group * (P.dm.N / TILE_ROWS));
   const int grid = stages < p->sm_count ? stages : p->sm_count;
   dct_tc_kernel<<<grid, DCT_TC_THREADS, smem, st>>>(m0, m1, m2, P);
   p->launches += 1;
@@ -414,7 +437,9 @@ bool axis_ok(int n) { return n == 16 || n == 32 || n == 64 || n == 128; }
 
 // bf16, head_dim 128, power-of-two axis lengths 16..128, low box small enough for the fp32 side path.
 bool ffk_dct_tc_supported(const FFDims& dm) {
-  return !dm.fp32 && dm.d == CH && axis_ok(dm.T) && axis_ok(dm.H) && axis_ok(dm.W) && dm.L[2] <= 16;
+  if (dm.fp32 || dm.d != CH || !axis_ok(dm.T) || !axis_ok(dm.H) || !axis_ok(dm.W)) return false;
+  // a tile groups 128/n lines: consecutive h for the w pass, consecutive w for the h and t passes
+  return dm.H % (TILE_ROWS / dm.W) == 0 && dm.W % (TILE_ROWS / dm.H) == 0 && dm.W % (TILE_ROWS / dm.T) == 0;
 }
 
 // Scratch: two hi/lo pairs of bf16 grids and the fp32 side buffer for `group` tensor-heads.
@@ -457,15 +482,15 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
   for (int g0 = 0; g0 < total; g0 += G) {
     const int g = total - g0 < G ? total - g0 : G;
     P.group = g; P.group_start = g0;
-    P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.mat = p->basis[2]; P.lines_per_th = dm.T * dm.H;
+    P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.mat = p->basis[2];
     P.dst = sc.a_hi; P.dst_lo = sc.a_lo; P.side = side;
     cudaError_t e = launch_pass(p, mq, mk, mv, P, st);
     if (e != cudaSuccess) return e;
-    P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.mat = p->basis[1]; P.lines_per_th = dm.T * dm.W;
+    P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.mat = p->basis[1];
     P.dst = sc.b_hi; P.dst_lo = sc.b_lo;
     e = launch_pass(p, m1h, m1l, m1l, P, st);
     if (e != cudaSuccess) return e;
-    P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.mat = p->basis[0]; P.lines_per_th = dm.H * dm.W; P.dst = nullptr;
+    P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.mat = p->basis[0]; P.dst = nullptr;
     e = launch_pass(p, m2h, m2l, m2l, P, st);
     if (e != cudaSuccess) return e;
     dim3 lgrid((unsigned)(dm.L[1] * dm.L[2]), (unsigned)g);
@@ -490,15 +515,15 @@ cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaS
     return cudaErrorInvalidValue;
   DctTcParams P{};
   P.dm = dm; P.status = p->buf.status; P.group = g; P.group_start = h0;
-  P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 0; P.n = dm.T; P.mat = p->basis_t[0]; P.lines_per_th = dm.H * dm.W;
+  P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 0; P.n = dm.T; P.mat = p->basis_t[0];
   P.dst = sc.b_hi; P.dst_lo = sc.b_lo;
   cudaError_t e = launch_pass(p, m_in, m_inl, m_inl, P, st);
   if (e != cudaSuccess) return e;
-  P.in_split = 1; P.axis = 1; P.n = dm.H; P.mat = p->basis_t[1]; P.lines_per_th = dm.T * dm.W;
+  P.in_split = 1; P.axis = 1; P.n = dm.H; P.mat = p->basis_t[1];
   P.dst = sc.a_hi; P.dst_lo = sc.a_lo;
   e = launch_pass(p, mbh, mbl, mbl, P, st);
   if (e != cudaSuccess) return e;
-  P.mode = MODE_LAST; P.axis = 2; P.n = dm.W; P.mat = p->basis_t[2]; P.lines_per_th = dm.T * dm.H;
+  P.mode = MODE_LAST; P.axis = 2; P.n = dm.W; P.mat = p->basis_t[2];
   P.dst = (__nv_bfloat16*)out; P.dst_lo = nullptr;
   return launch_pass(p, mah, mal, mal, P, st);
 }
