@@ -97,6 +97,12 @@ void ff_compute_layout(const FFDims& dm, bool with_staging, FFLayout* lay) {
   if (G < 1) G = 1;
   if (G > 3 * BH) G = 3 * BH;
   lay->group = (int)G;
+  // Tensor-core transform: as many tensor-heads per launch as fit ~2 GiB of scratch (at least 3).
+  size_t Gt = ((size_t)2 << 30) / (4 * (size_t)dm.N * d * 2);
+  if (Gt < 3) Gt = 3;
+  if (Gt > 3 * BH) Gt = 3 * BH;
+  lay->tc_group = (int)Gt;
+  const size_t tc_scratch = ffk_dct_tc_supported(dm) ? ffk_dct_tc_scratch_bytes(dm, (int)Gt) : 0;
   const size_t sizes[20] = {
       3 * BH * (size_t)dm.Nlow * d * 4,   // 0 spec_low
       3 * BH * (size_t)dm.Nmid * d * e,   // 1 spec_mid
@@ -111,8 +117,8 @@ void ff_compute_layout(const FFDims& dm, bool with_staging, FFLayout* lay) {
       (size_t)dm.B * 3 * 4,               // 10 pi
       (size_t)dm.B * 4,                   // 11 timestep
       256,                                // 12 status
-      G * per,                            // 13 scratchA
-      G * per,                            // 14 scratchB
+      tc_scratch > 2 * G * per ? tc_scratch - G * per : G * per,   // 13 scratchA (the tensor-core transform
+      G * per,                            // 14 scratchB                  uses A and B as one region)
       with_staging ? BH * (size_t)dm.N * d * e : 0,  // 15..18 staging
       with_staging ? BH * (size_t)dm.N * d * e : 0,
       with_staging ? BH * (size_t)dm.N * d * e : 0,
@@ -154,6 +160,7 @@ extern "C" ff_status_t ff_destroy(ff_plan_t* p) {
   if (!p) return FF_OK;
   for (int a = 0; a < 3; ++a) { cudaFree(p->basis[a]); cudaFree(p->basis_t[a]); }
   if (p->ev[0]) for (int i = 0; i <= FF_STAGE_COUNT; ++i) cudaEventDestroy(p->ev[i]);
+  cudaFree(p->dct_images);
   cudaFree(p->W1); cudaFree(p->b1); cudaFree(p->W2); cudaFree(p->b2); cudaFree(p->U);
   delete p;
   return FF_OK;
@@ -189,6 +196,9 @@ extern "C" ff_status_t ff_plan_create(const ff_config_t* c, const ff_weights_t* 
       }
     s = upload(p, &p->basis[a], C.data(), C.size());
     if (s == FF_OK) s = upload(p, &p->basis_t[a], Ct.data(), Ct.size());
+    if (s == FF_OK && ffk_dct_tc_supported(p->dm) &&
+        !(ffk_dct_tc_build_image(p, a, 0, C.data(), n[a]) && ffk_dct_tc_build_image(p, a, 1, Ct.data(), n[a])))
+      s = fail(p, FF_ERR_CUDA, "could not upload the transform matrix images%s");
   }
   const size_t d = c->head_dim, hid = c->router_hidden, nin = 3 * d + c->t_embed_dim;
   if (s == FF_OK && w && w->W1 && w->b1 && w->W2 && w->b2) {
@@ -249,9 +259,8 @@ extern "C" ff_status_t ff_plan_set_workspace(ff_plan_t* p, void* ptr, size_t byt
   p->dct_tc_ok = false;
   if (ffk_dct_tc_supported(p->dm)) {
     const size_t room = (size_t)((char*)base + o[14] - (char*)b.scratchA) + (size_t)p->lay.group * p->dm.N * p->dm.d * 4;
-    int G = 3 * p->dm.BH < 3 ? 3 * p->dm.BH : 3;
-    while (G > 1 && ffk_dct_tc_scratch_bytes(p->dm, G) > room) --G;
-    if (ffk_dct_tc_scratch_bytes(p->dm, G) <= room) { p->dct_tc_ok = true; p->dct_group = G; }
+    const int G = p->lay.tc_group;
+    if (p->dct_images && ffk_dct_tc_scratch_bytes(p->dm, G) <= room) { p->dct_tc_ok = true; p->dct_group = G; }
   }
   return FF_OK;
 }

@@ -27,6 +27,8 @@
 //        LAST   intermediate -> the caller's out tensor
 #include <cuda.h>
 
+#include <vector>
+
 #include "ff_internal.h"
 #include "ff_sm100.cuh"
 
@@ -46,7 +48,7 @@ enum { MODE_FIRST = 0, MODE_MIDDLE = 1, MODE_SPLIT = 2, MODE_LAST = 3 };
 
 struct DctTcParams {
   FFDims dm;
-  const float* mat;        // [n][n] fp32, out[a] = sum_b mat[a][b] in[b]
+  const uint8_t* image;    // matrix images (hi then lo, 32 KB each) in their shared-memory layout
   int n;                   // axis length
   int axis;                // 0 = t, 1 = h, 2 = w
   int mode;
@@ -63,7 +65,7 @@ struct DctTcParams {
 };
 
 struct DctShared {
-  uint64_t full[MAX_STAGE], empty[MAX_STAGE], acc_full[NACC], acc_empty[NACC];
+  uint64_t full[MAX_STAGE], empty[MAX_STAGE], acc_full[NACC], acc_empty[NACC], img_full;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -82,6 +84,12 @@ __device__ __forceinline__ void tma_load_5d(void* smem_dst, const CUtensorMap* m
       "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
       ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
       : "memory");
+}
+
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(smem_dst)), "l"((uint64_t)gsrc), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
 }
 
 // Three source maps (Q, K, V) in MODE_FIRST; otherwise map0 (= hi) and, for split input, map1 (= lo).
@@ -109,26 +117,10 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NSTAGE; ++i) { mbar_init(&sh.full[i], 1); mbar_init(&sh.empty[i], 1); }
     for (int i = 0; i < NACC; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 128); }
+    mbar_init(&sh.img_full, 1);
     sh.abort_flag = 0;
     fence_mbar_init();
   }
-  // Matrix image, the K-major A operand: row j = output position of the tile, 64 input positions per
-  // 128-byte row, 16-byte chunks XOR-swizzled with the row index (the 128-byte swizzle the MMA
-  // expects).  Lines that follow one another (w axis): I kron Mat, index = line*n + a.  Interleaved
-  // lines (h, t axes): Mat kron I, index = a*kf + line.
-  for (int idx = threadIdx.x; idx < TILE_ROWS * TILE_ROWS; idx += DCT_TC_THREADS) {
-    const int j = idx >> 7, r = idx & 127;
-    float v;
-    if (seq) v = ((j >> ln) == (r >> ln)) ? P.mat[(j & (n - 1)) * n + (r & (n - 1))] : 0.f;
-    else v = ((j & (kf - 1)) == (r & (kf - 1))) ? P.mat[(j >> lkf) * n + (r >> lkf)] : 0.f;
-    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-    const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-    const int half = r >> 6, rk = r & 63;
-    const uint32_t off = half * HALF_BYTES + j * 128 + ((((rk >> 3) ^ (j & 7)) << 4) | ((rk & 7) << 1));
-    *(__nv_bfloat16*)(sHi + off) = hi;
-    *(__nv_bfloat16*)(sLo + off) = lo;
-  }
-  fence_proxy_async();                                    // generic-proxy writes -> visible to the MMA's async proxy
   if (warp == 1) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
@@ -139,6 +131,10 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
   if (warp == 0) {
     if (lane == 0) {
       tma_prefetch_desc(&map0);
+      // the two matrix images (prepared at plan creation, already in the operand layout)
+      mbar_arrive_expect_tx(&sh.img_full, 2 * TILE_BYTES);
+      bulk_load(sHi, P.image, TILE_BYTES, &sh.img_full);
+      bulk_load(sLo, P.image + TILE_BYTES, TILE_BYTES, &sh.img_full);
       unsigned it = 0;
       bool ok = true;
       for (int s = blockIdx.x; s < total_tiles && ok; s += gridDim.x, ++it) {
@@ -170,7 +166,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
       const uint32_t idesc = idesc_bf16_f32(TILE_ROWS, CH, /*a_mn_major=*/false, /*b_mn_major=*/true);
       const uint32_t hi_base = smem_u32(sHi), lo_base = smem_u32(sLo);
       unsigned it = 0;
-      bool ok = true;
+      bool ok = mbar_wait(&sh.img_full, 0, abort_flag);
       for (int s = blockIdx.x; s < total_tiles && ok; s += gridDim.x, ++it) {
         const int slot = it % NSTAGE, ab = it % NACC;
         ok = mbar_wait(&sh.full[slot], (it / NSTAGE) & 1, abort_flag);
@@ -442,6 +438,35 @@ bool ffk_dct_tc_supported(const FFDims& dm) {
   return dm.H % (TILE_ROWS / dm.W) == 0 && dm.W % (TILE_ROWS / dm.H) == 0 && dm.W % (TILE_ROWS / dm.T) == 0;
 }
 
+// Matrix images of one axis (0 = t, 1 = h, 2 = w) and direction, in the layout the kernel's A
+// operand has in shared memory: row j = output position of a tile, 64 input positions per 128-byte
+// row, 16-byte chunks XOR-swizzled with the row index (the 128-byte swizzle the MMA expects), the
+// bf16 hi part followed by the lo part.  Lines that follow one another (w axis): I kron Mat,
+// index = line*n + a.  Interleaved lines (h, t axes): Mat kron I, index = a*kf + line.
+// `mat` is the host matrix [n][n] with out[a] = sum_b mat[a][b] in[b].
+bool ffk_dct_tc_build_image(ff_plan* p, int axis, int inverse, const float* mat, int n) {
+  if (!p->dct_images && cudaMalloc((void**)&p->dct_images, (size_t)12 * TILE_BYTES) != cudaSuccess) return false;
+  const int kf = TILE_ROWS / n;
+  const bool seq = axis == 2;
+  std::vector<__nv_bfloat16> img((size_t)TILE_BYTES);          // hi and lo: 2 x 16384 elements
+  __nv_bfloat16* hi_img = img.data();
+  __nv_bfloat16* lo_img = img.data() + TILE_ROWS * TILE_ROWS;
+  for (int j = 0; j < TILE_ROWS; ++j)
+    for (int r = 0; r < TILE_ROWS; ++r) {
+      float v;
+      if (seq) v = (j / n == r / n) ? mat[(j % n) * n + (r % n)] : 0.f;
+      else v = (j % kf == r % kf) ? mat[(j / kf) * n + (r / kf)] : 0.f;
+      const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+      const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+      const int half = r >> 6, rk = r & 63;
+      const size_t off = (size_t)half * HALF_BYTES + (size_t)j * 128 + ((((rk >> 3) ^ (j & 7)) << 4) | ((rk & 7) << 1));
+      hi_img[off / 2] = hi;
+      lo_img[off / 2] = lo;
+    }
+  const int slot = (inverse ? 3 : 0) + axis;
+  return cudaMemcpy(p->dct_images + (size_t)2 * slot * TILE_BYTES, img.data(), 2 * TILE_BYTES, cudaMemcpyHostToDevice) == cudaSuccess;
+}
+
 // Scratch: two hi/lo pairs of bf16 grids and the fp32 side buffer for `group` tensor-heads.
 size_t ffk_dct_tc_scratch_bytes(const FFDims& dm, int group) {
   const size_t grid = (size_t)group * dm.N * CH * 2;
@@ -482,15 +507,15 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
   for (int g0 = 0; g0 < total; g0 += G) {
     const int g = total - g0 < G ? total - g0 : G;
     P.group = g; P.group_start = g0;
-    P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.mat = p->basis[2];
+    P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 2 + 0) * TILE_BYTES;
     P.dst = sc.a_hi; P.dst_lo = sc.a_lo; P.side = side;
     cudaError_t e = launch_pass(p, mq, mk, mv, P, st);
     if (e != cudaSuccess) return e;
-    P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.mat = p->basis[1];
+    P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 1 + 0) * TILE_BYTES;
     P.dst = sc.b_hi; P.dst_lo = sc.b_lo;
     e = launch_pass(p, m1h, m1l, m1l, P, st);
     if (e != cudaSuccess) return e;
-    P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.mat = p->basis[0]; P.dst = nullptr;
+    P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 0 + 0) * TILE_BYTES; P.dst = nullptr;
     e = launch_pass(p, m2h, m2l, m2l, P, st);
     if (e != cudaSuccess) return e;
     dim3 lgrid((unsigned)(dm.L[1] * dm.L[2]), (unsigned)g);
@@ -515,15 +540,15 @@ cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaS
     return cudaErrorInvalidValue;
   DctTcParams P{};
   P.dm = dm; P.status = p->buf.status; P.group = g; P.group_start = h0;
-  P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 0; P.n = dm.T; P.mat = p->basis_t[0];
+  P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 3 + 0) * TILE_BYTES;
   P.dst = sc.b_hi; P.dst_lo = sc.b_lo;
   cudaError_t e = launch_pass(p, m_in, m_inl, m_inl, P, st);
   if (e != cudaSuccess) return e;
-  P.in_split = 1; P.axis = 1; P.n = dm.H; P.mat = p->basis_t[1];
+  P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 4 + 0) * TILE_BYTES;
   P.dst = sc.a_hi; P.dst_lo = sc.a_lo;
   e = launch_pass(p, mbh, mbl, mbl, P, st);
   if (e != cudaSuccess) return e;
-  P.mode = MODE_LAST; P.axis = 2; P.n = dm.W; P.mat = p->basis_t[2];
+  P.mode = MODE_LAST; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 5 + 0) * TILE_BYTES;
   P.dst = (__nv_bfloat16*)out; P.dst_lo = nullptr;
   return launch_pass(p, mah, mal, mal, P, st);
 }

@@ -73,7 +73,8 @@ struct FFBuffers {
 struct FFLayout {
   size_t off[24];
   size_t total;
-  int group;         // G: tensor-heads processed per transform launch
+  int group;         // G: tensor-heads processed per generic transform launch
+  int tc_group;      // tensor-heads per tensor-core transform launch
 };
 
 struct ff_plan {
@@ -95,6 +96,7 @@ struct ff_plan {
   bool tc_ok;                                  // tensor-core attention usable with this plan + workspace
   bool dct_tc_ok;                              // tensor-core transform usable
   int dct_group;                               // tensor-heads per tensor-core transform launch
+  uint8_t* dct_images;                         // 6 x (hi, lo) matrix images of the tensor-core transform (plan-owned)
   alignas(64) unsigned char tmap_mid[128];     // CUtensorMap over the mid-band / high-band coefficient buffers
   alignas(64) unsigned char tmap_high[128];
   long long launches;
@@ -119,6 +121,7 @@ bool ffk_tc_prepare(ff_plan* p);               // builds the tensor maps over th
 cudaError_t ffk_attention_tc(ff_plan* p, cudaStream_t st);
 // ---- tensor-core transform (ff_dct_tc.cu) --------------------------------------------------------
 bool ffk_dct_tc_supported(const FFDims& dm);
+bool ffk_dct_tc_build_image(ff_plan* p, int axis, int inverse, const float* mat_host, int n);
 size_t ffk_dct_tc_scratch_bytes(const FFDims& dm, int group);
 cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, const void* V, bool want_energy,
                                      cudaStream_t st);
