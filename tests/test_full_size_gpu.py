@@ -1,0 +1,93 @@
+"""Full-size parity: the five benchmark workloads at their real sizes, in the launch configuration
+bench.py times (router-driven allocation), compared stage by stage with the fp64 oracle on sampled
+rows: 4096 seeded band-query rows per checked head for the transform and the band operators, the
+summary tokens in full, and the exchange + recombination + inverse transform as whole output heads.
+The router statistics (every head's full fp64 transform) fix the head allocation bit for bit."""
+import numpy as np
+import pytest
+
+from oracle import freqformer_oracle as O
+from paper_2604_22808_b200 import configs as C
+from paper_2604_22808_b200 import inputs as I
+
+import harness as Hn
+
+pytestmark = pytest.mark.gpu
+
+
+def _device_inputs(cfg):
+    import torch
+    dt = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
+    shape = (cfg.batch, cfg.heads, cfg.T, cfg.H, cfg.W, cfg.head_dim)
+    dev = [torch.empty(shape, dtype=dt, device="cuda") for _ in range(3)]
+    for t in range(3):
+        for bi in range(cfg.batch):
+            for h in range(cfg.heads):
+                dev[t][bi, h].copy_(torch.from_numpy(I.qkv_head(cfg, t, bi, h)))
+    return dev
+
+
+def _pick_heads(alloc, per_band=2):
+    """A few heads of every band type the allocation uses."""
+    picked = []
+    for bit in (1, 2, 4):
+        picked += [i for i, m in enumerate(alloc) if m == bit][:per_band]
+    return sorted(set(picked))
+
+
+def _run_full(cfg, timestep_indices, per_band=2):
+    import torch
+    from paper_2604_22808_b200 import binding as B
+    weights = I.router_weights(cfg)
+    U = I.summary_projection(cfg)
+    q, k, v = _device_inputs(cfg)
+    out = torch.empty_like(q)
+    plan = B.Plan(cfg, weights)
+    source = lambda t, bi, h: (q, k, v)[t][bi, h].float().cpu().numpy()
+    g_cache = None
+    for n_call, ti in enumerate(timestep_indices):
+        ts = [cfg.timesteps[ti]] * cfg.batch
+        plan.forward(q, k, v, out, timesteps=ts)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        alloc = plan.tap(B.TAP_ALLOC).cpu().numpy()
+        heads = _pick_heads(alloc.tolist(), per_band)
+        out_of = lambda bi, h: out[bi, h].float().cpu().numpy()
+        if n_call == 0:
+            errs = Hn.stagewise_check(cfg, plan, None, None, None, out_of, weights, U, ts, routed=True,
+                                      check_heads=heads, inverse_heads=heads, head_source=source)
+            g_cache = errs.pop("g")
+        else:
+            # later timesteps of a sweep: same inputs, so the pooled statistics are known; the router
+            # decision is checked for every sample and the device path on the picked heads
+            for bi in range(cfg.batch):
+                pi, _ = O.router_probabilities(g_cache[bi], O.timestep_embedding(float(ts[bi]), cfg.t_embed_dim),
+                                               weights["W1"], weights["b1"], weights["W2"], weights["b2"])
+                counts, margin = O.head_quota(pi, cfg.heads)
+                assert np.abs(plan.tap(B.TAP_PI).cpu().numpy()[bi] - pi).max() < 2e-3
+                if Hn.allocation_is_stable(pi, cfg.heads):
+                    assert np.array_equal(alloc.reshape(cfg.batch, cfg.heads)[bi], O.head_allocation(counts))
+            errs = Hn.stagewise_check(cfg, plan, None, None, None, out_of, weights, U, ts, routed=False,
+                                      check_heads=heads, inverse_heads=heads, head_source=source)
+        print(cfg.name, "t =", ts[0], "heads per band", [int((alloc == b).sum()) for b in (1, 2, 4)], errs)
+    plan.destroy()
+
+
+def test_tiny_fp32_full():
+    _run_full(C.TINY, [0])
+
+
+def test_64k_full():
+    _run_full(C.G64K, [0])
+
+
+def test_256k_full():
+    _run_full(C.G256K, [0], per_band=1)
+
+
+def test_1m_full():
+    _run_full(C.G1M, [0], per_band=1)
+
+
+def test_128k_sweep_full():
+    _run_full(C.G128K, [0, 1, 2, 3, 4], per_band=1)
