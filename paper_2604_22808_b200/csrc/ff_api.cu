@@ -160,7 +160,7 @@ extern "C" ff_status_t ff_destroy(ff_plan_t* p) {
   if (!p) return FF_OK;
   for (int a = 0; a < 3; ++a) { cudaFree(p->basis[a]); cudaFree(p->basis_t[a]); }
   if (p->ev[0]) for (int i = 0; i <= FF_STAGE_COUNT; ++i) cudaEventDestroy(p->ev[i]);
-  cudaFree(p->dct_images);
+  cudaFree(p->dct_images); cudaFree(p->pos_table);
   cudaFree(p->W1); cudaFree(p->b1); cudaFree(p->W2); cudaFree(p->b2); cudaFree(p->U);
   delete p;
   return FF_OK;
@@ -214,6 +214,8 @@ extern "C" ff_status_t ff_plan_create(const ff_config_t* c, const ff_weights_t* 
     else for (size_t l = 0; l < 3; ++l) for (size_t i = 0; i < d; ++i) U[(l * d + i) * d + i] = 1.f;
     s = upload(p, &p->U, U.data(), U.size());
   }
+  if (s == FF_OK && ffk_exchange_tc_supported(p->dm) && !ffk_exchange_tc_build_tables(p))
+    s = fail(p, FF_ERR_CUDA, "could not upload the band position tables%s");
   if (s != FF_OK) {
     snprintf(g_err, 512, "%s", p->err);
     ff_destroy(p);
@@ -255,6 +257,7 @@ extern "C" ff_status_t ff_plan_set_workspace(ff_plan_t* p, void* ptr, size_t byt
   b.work = (int*)(base + o[19]);
   FF_CUDA(p, cudaMemset(b.status, 0, 256));
   p->tc_ok = ffk_tc_supported(p->dm) && ffk_tc_prepare(p);
+  p->xtc_ok = p->pos_table && ffk_exchange_tc_supported(p->dm) && ffk_exchange_tc_prepare(p);
   // The tensor-core transform shares the scratch region (scratchA and scratchB are adjacent).
   p->dct_tc_ok = false;
   if (ffk_dct_tc_supported(p->dm)) {

@@ -1,0 +1,363 @@
+// Cross-band residual exchange + recombination on the tensor cores ("Cross-band residual
+// exchange", "Reconstruction"), bf16 storage, head_dim 128, for the mid and high bands:
+//     Y^[p] = Y[p] + softmax(Y[p] Z^T / sqrt(d)) Z,   Z = the 2m summary tokens of the other two bands
+// written to the coefficient grid at the position of band rank p (a table built at plan creation).
+//
+// A CTA owns a contiguous run of (head, band, 128-rank tile) items, so the summary tokens of a head
+// are re-staged only a few times per CTA.  Per tile:
+//   TMA     the 128 band tokens (operator output where the head's mask has the band, V~ otherwise)
+//   MMA 1   S[128 x 3m] = Y Z^T against all 3m summaries of the head (own band masked in the softmax)
+//   softmax one token per thread (row = TMEM lane); normalised P written back to TMEM as bf16 hi + lo
+//   MMA 2   D[128 x 128] = P Z  (A = P from tensor memory, B = the same Z image read MN-major)
+//   store   Y + D as a bf16 hi/lo pair, one 256-byte grid row per thread
+// Z and P are split into bf16 hi + lo parts (Y is exact bf16), so the logits and the update carry
+// about 16 bits: the summary logits of a band with large low-frequency content reach O(100).
+// The low band (fp32, a few hundred tokens) is handled by the generic kernel.
+#include <cuda.h>
+
+#include "ff_internal.h"
+#include "ff_sm100.cuh"
+
+using namespace sm100;
+
+namespace {
+
+constexpr int XT = 128;                 // tokens per tile
+constexpr int XD = 128;                 // head_dim
+constexpr int X_TILE_BYTES = XT * XD * 2;
+constexpr int X_HALF = X_TILE_BYTES / 2;
+constexpr int X_THREADS = 192;
+constexpr int MAX_KEYS = 96;            // 3m rounded up to 16, m <= 32
+
+struct XParams {
+  FFDims dm;
+  const uint8_t* alloc;
+  const float* summary;       // [BH][3][m][d]
+  const int* pos_mid;         // [N_mid]  flat coefficient index of each band rank
+  const int* pos_high;        // [N_high]
+  __nv_bfloat16* grid_hi;     // [g][N][d]
+  __nv_bfloat16* grid_lo;
+  int h0, g;                  // heads [h0, h0+g)
+  int nkeys;                  // 3m rounded up to a multiple of 16
+  int* status;
+};
+
+struct XShared {
+  uint64_t y_full[2], y_empty[2], z_ready, s_full, p_full, d_full, d_empty;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct XItem { int bh, band, tile; };
+
+__device__ __forceinline__ XItem x_decode(const FFDims& dm, int h0, int it, int tm, int th) {
+  XItem x;
+  const int per = tm + th;
+  x.bh = h0 + it / per;
+  const int rem = it % per;
+  x.band = rem < tm ? 1 : 2;
+  x.tile = rem < tm ? rem : rem - tm;
+  return x;
+}
+
+__global__ void __launch_bounds__(X_THREADS, 1)
+exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_constant__ CUtensorMap map_v_mid,
+                   const __grid_constant__ CUtensorMap map_y_high, const __grid_constant__ CUtensorMap map_v_high,
+                   const XParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* sY = smem;                                    // 2 x 32 KB
+  uint8_t* sZhi = smem + 2 * X_TILE_BYTES;               // [2 halves][nkeys rows][128 B]
+  uint8_t* sZlo = sZhi + 2 * MAX_KEYS * 128;
+  XShared& sh = *(XShared*)(sZlo + 2 * MAX_KEYS * 128);
+  const FFDims& dm = P.dm;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m = dm.m, nk = P.nkeys;
+  const int tm_tiles = (int)((dm.Nmid + XT - 1) / XT), th_tiles = (int)((dm.Nhigh + XT - 1) / XT);
+  const int total = P.g * (tm_tiles + th_tiles);
+  const int chunk = (total + gridDim.x - 1) / gridDim.x;
+  const int it0 = blockIdx.x * chunk;
+  const int it1 = it0 + chunk < total ? it0 + chunk : total;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.y_full[i], 1); mbar_init(&sh.y_empty[i], 128); }
+    mbar_init(&sh.z_ready, 128); mbar_init(&sh.s_full, 1); mbar_init(&sh.p_full, 128);
+    mbar_init(&sh.d_full, 1); mbar_init(&sh.d_empty, 128);
+    sh.abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+  volatile int* abort_flag = &sh.abort_flag;
+  // tensor-memory columns: S [0,96)  P_hi [128,176)  P_lo [192,240)  D [256,384)
+
+  if (warp == 0) {
+    if (lane == 0) {
+      bool ok = true;
+      int n = 0;
+      for (int it = it0; it < it1 && ok; ++it, ++n) {
+        const XItem x = x_decode(dm, P.h0, it, tm_tiles, th_tiles);
+        const bool exec = P.alloc[x.bh] & (1 << x.band);
+        const CUtensorMap* map = x.band == 1 ? (exec ? &map_y_mid : &map_v_mid) : (exec ? &map_y_high : &map_v_high);
+        const int slice = exec ? x.bh : 2 * dm.BH + x.bh;
+        const int slot = n & 1;
+        if (n >= 2) ok = mbar_wait(&sh.y_empty[slot], ((n >> 1) - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&sh.y_full[slot], X_TILE_BYTES);
+        tma_load_3d(sY + slot * X_TILE_BYTES, map, &sh.y_full[slot], 0, x.tile * XT, slice);
+        tma_load_3d(sY + slot * X_TILE_BYTES + X_HALF, map, &sh.y_full[slot], 64, x.tile * XT, slice);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc1 = idesc_bf16_f32(XT, nk, false, false);
+      const uint32_t idesc2 = idesc_bf16_f32(XT, XD, false, true);
+      const uint32_t zhi = smem_u32(sZhi), zlo = smem_u32(sZlo);
+      const uint32_t zhalf = nk * 128;                    // bytes between the two 64-channel halves of a Z image
+      bool ok = true;
+      int n = 0, prev_bh = -1, zc = 0;
+      for (int it = it0; it < it1 && ok; ++it, ++n) {
+        const XItem x = x_decode(dm, P.h0, it, tm_tiles, th_tiles);
+        if (x.bh != prev_bh) {                            // the softmax warps re-staged Z for this head
+          ok = mbar_wait(&sh.z_ready, zc & 1, abort_flag); ++zc; prev_bh = x.bh;
+          if (!ok) break;
+        }
+        const int slot = n & 1;
+        ok = mbar_wait(&sh.y_full[slot], (n >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t ybase = smem_u32(sY + slot * X_TILE_BYTES);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {                     // S = Y (Zhi + Zlo)^T, K = head_dim
+          const uint64_t a = smem_desc_sw128(ybase + (k >> 2) * X_HALF + (k & 3) * 32, 16, 1024);
+          const uint32_t zo = (k >> 2) * zhalf + (k & 3) * 32;
+          umma_ss(tmem, a, smem_desc_sw128(zhi + zo, 16, 1024), idesc1, k > 0 ? 1u : 0u);
+          umma_ss(tmem, a, smem_desc_sw128(zlo + zo, 16, 1024), idesc1, 1u);
+        }
+        umma_commit(&sh.s_full);
+        ok = mbar_wait(&sh.p_full, n & 1, abort_flag);
+        if (ok && n >= 1) ok = mbar_wait(&sh.d_empty, (n - 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        for (int k = 0; k < nk / 16; ++k) {               // D = (Phi + Plo) (Zhi + Zlo) without lo*lo, K = keys
+          const uint64_t bh_ = smem_desc_sw128(zhi + k * 2048, zhalf, 1024);
+          umma_ts(tmem + 256, tmem + 128 + k * 8, bh_, idesc2, k > 0 ? 1u : 0u);
+          umma_ts(tmem + 256, tmem + 128 + k * 8, smem_desc_sw128(zlo + k * 2048, zhalf, 1024), idesc2, 1u);
+          umma_ts(tmem + 256, tmem + 192 + k * 8, bh_, idesc2, 1u);
+        }
+        umma_commit(&sh.d_full);
+      }
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int tid = row;                                  // 0..127 among the softmax threads
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const float sl2 = rsqrtf((float)XD) * 1.4426950408889634f;
+    bool ok = true;
+    int n = 0, prev_bh = -1;
+    for (int it = it0; it < it1 && ok; ++it, ++n) {
+      const XItem x = x_decode(dm, P.h0, it, tm_tiles, th_tiles);
+      if (x.bh != prev_bh) {
+        // Stage the head's 3m summaries as two bf16 images (hi, lo) in the operand layout: row = key,
+        // 64 channels per 128-byte row, 16-byte chunks XOR-swizzled with the row.  Rows >= 3m are zero.
+        // Every MMA of the previous tile has completed (its D was read before this point).
+        prev_bh = x.bh;
+        const float* S = P.summary + (size_t)x.bh * 3 * m * XD;
+        for (int idx = tid; idx < nk * XD; idx += 128) {
+          const int j = idx >> 7, c = idx & 127;
+          const float v = j < 3 * m ? S[j * XD + c] : 0.f;
+          const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+          const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+          const int half = c >> 6, ck = c & 63;
+          const uint32_t off = half * (nk * 128) + j * 128 + ((((ck >> 3) ^ (j & 7)) << 4) | ((ck & 7) << 1));
+          *(__nv_bfloat16*)(sZhi + off) = hi;
+          *(__nv_bfloat16*)(sZlo + off) = lo;
+        }
+        fence_proxy_async();
+        mbar_arrive(&sh.z_ready);
+      }
+      const int slot = n & 1;
+      const long long n_band = x.band == 1 ? dm.Nmid : dm.Nhigh;
+      const long long p = (long long)x.tile * XT + row;
+      // ---- softmax over the 2m summaries of the other bands
+      ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full, n & 1, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const int own0 = x.band * m, own1 = own0 + m;       // this band's own summaries are not attended
+      float mx = -INFINITY;
+      uint32_t r[32];
+      for (int c0 = 0; c0 < nk; c0 += 32) {               // nk is 48 or 96: the last chunk may read stale columns
+        tmem_ld32(tmem + lane_addr + c0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int j = c0 + i;
+          if (j < 3 * m && (j < own0 || j >= own1)) mx = fmaxf(mx, __uint_as_float(r[i]));
+        }
+      }
+      float den = 0.f;
+      for (int c0 = 0; c0 < nk; c0 += 32) {
+        tmem_ld32(tmem + lane_addr + c0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int j = c0 + i;
+          if (j < 3 * m && (j < own0 || j >= own1)) den += exp2f((__uint_as_float(r[i]) - mx) * sl2);
+        }
+      }
+      const float inv = 1.f / den;
+      for (int c0 = 0; c0 < nk; c0 += 32) {
+        tmem_ld32(tmem + lane_addr + c0, r);
+        tmem_wait_ld();
+        uint32_t ph[16], pl[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float pv[2];
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int j = c0 + 2 * i + e;
+            pv[e] = (j < 3 * m && (j < own0 || j >= own1)) ? exp2f((__uint_as_float(r[2 * i + e]) - mx) * sl2) * inv : 0.f;
+          }
+          const __nv_bfloat162 h2 = __floats2bfloat162_rn(pv[0], pv[1]);
+          ph[i] = *(const uint32_t*)&h2;
+          const __nv_bfloat162 l2 = __floats2bfloat162_rn(pv[0] - __uint_as_float(ph[i] << 16),
+                                                          pv[1] - __uint_as_float(ph[i] & 0xffff0000u));
+          pl[i] = *(const uint32_t*)&l2;
+        }
+        if (c0 + 32 <= nk || true) {
+          tmem_st16(tmem + lane_addr + 128 + (c0 >> 1), ph);
+          tmem_st16(tmem + lane_addr + 192 + (c0 >> 1), pl);
+        }
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&sh.p_full);
+      // ---- residual add and store
+      ok = __all_sync(0xffffffffu, mbar_wait(&sh.d_full, n & 1, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const bool valid = p < n_band;
+      const int f = valid ? (x.band == 1 ? P.pos_mid[p] : P.pos_high[p]) : 0;
+      const size_t o = ((size_t)(x.bh - P.h0) * dm.N + f) * XD;
+      const uint8_t* yrow = sY + slot * X_TILE_BYTES + row * 128;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        tmem_ld32(tmem + lane_addr + 256 + q * 32, r);
+        tmem_wait_ld();
+        if (valid) {
+#pragma unroll
+          for (int v4 = 0; v4 < 4; ++v4) {
+            // channels 32q + 8v4 .. +7 of this token: one 16-byte chunk of the swizzled Y tile
+            const int cch = q * 4 + v4;                    // 16-byte chunk index along the row, 0..15
+            const uint4 yv = *(const uint4*)(yrow + (cch >> 3) * X_HALF + (((cch & 7) ^ (row & 7)) << 4));
+            const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float v0 = __uint_as_float(yw[i] << 16) + __uint_as_float(r[v4 * 8 + 2 * i]);
+              const float v1 = __uint_as_float(yw[i] & 0xffff0000u) + __uint_as_float(r[v4 * 8 + 2 * i + 1]);
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+              hi[i] = *(const uint32_t*)&h2;
+              const __nv_bfloat162 l2 = __floats2bfloat162_rn(v0 - __uint_as_float(hi[i] << 16), v1 - __uint_as_float(hi[i] & 0xffff0000u));
+              lo[i] = *(const uint32_t*)&l2;
+            }
+            *(uint4*)(P.grid_hi + o + q * 32 + v4 * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *(uint4*)(P.grid_lo + o + q * 32 + v4 * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(&sh.d_empty);
+      mbar_arrive(&sh.y_empty[slot]);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (sh.abort_flag) {
+    if (threadIdx.x == 0) atomicExch(P.status, FF_ERR_TIMEOUT);
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+bool encode_rows_map(CUtensorMap* map, void* base, long long rows, int slices) {
+  static EncodeTiledFn enc = nullptr;
+  if (!enc) {
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", (void**)&enc, cudaEnableDefault, &qr) != cudaSuccess || !enc)
+      return false;
+  }
+  cuuint64_t dims[3] = {(cuuint64_t)XD, (cuuint64_t)rows, (cuuint64_t)slices};
+  cuuint64_t strides[2] = {(cuuint64_t)XD * 2, (cuuint64_t)rows * XD * 2};
+  cuuint32_t box[3] = {64, XT, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool ffk_exchange_tc_supported(const FFDims& dm) {
+  return !dm.fp32 && dm.d == XD && dm.m >= 1 && dm.m <= 32 && dm.N < (1LL << 31);
+}
+
+// Rank -> flat coefficient index tables of the mid and high bands (plan-owned device memory).
+bool ffk_exchange_tc_build_tables(ff_plan* p) {
+  const FFDims& dm = p->dm;
+  int* host = (int*)malloc((size_t)(dm.Nmid + dm.Nhigh) * sizeof(int));
+  if (!host) return false;
+  for (int kt = 0; kt < dm.T; ++kt)
+    for (int kh = 0; kh < dm.H; ++kh)
+      for (int kw = 0; kw < dm.W; ++kw) {
+        long long rank;
+        const int band = ff_band_rank_of(dm, kt, kh, kw, &rank);
+        const int f = (kt * dm.H + kh) * dm.W + kw;
+        if (band == 1) host[rank] = f;
+        else if (band == 2) host[dm.Nmid + rank] = f;
+      }
+  bool ok = cudaMalloc((void**)&p->pos_table, (size_t)(dm.Nmid + dm.Nhigh) * sizeof(int)) == cudaSuccess &&
+            cudaMemcpy(p->pos_table, host, (size_t)(dm.Nmid + dm.Nhigh) * sizeof(int), cudaMemcpyHostToDevice) == cudaSuccess;
+  free(host);
+  return ok;
+}
+
+bool ffk_exchange_tc_prepare(ff_plan* p) {
+  const FFDims& dm = p->dm;
+  return encode_rows_map((CUtensorMap*)p->tmap_x[0], p->buf.y_mid, dm.Nmid, dm.BH) &&
+         encode_rows_map((CUtensorMap*)p->tmap_x[1], p->buf.spec_mid, dm.Nmid, 3 * dm.BH) &&
+         encode_rows_map((CUtensorMap*)p->tmap_x[2], p->buf.y_high, dm.Nhigh, dm.BH) &&
+         encode_rows_map((CUtensorMap*)p->tmap_x[3], p->buf.spec_high, dm.Nhigh, 3 * dm.BH);
+}
+
+// Exchange + recombination of the mid and high bands of heads [h0, h0+g) into the hi/lo grids.
+cudaError_t ffk_exchange_tc(ff_plan* p, int h0, int g, void* grid_hi, void* grid_lo, cudaStream_t st) {
+  const FFDims& dm = p->dm;
+  XParams P;
+  P.dm = dm; P.alloc = p->buf.alloc; P.summary = p->buf.summary;
+  P.pos_mid = p->pos_table; P.pos_high = p->pos_table + dm.Nmid;
+  P.grid_hi = (__nv_bfloat16*)grid_hi; P.grid_lo = (__nv_bfloat16*)grid_lo;
+  P.h0 = h0; P.g = g; P.nkeys = (3 * dm.m + 15) / 16 * 16; P.status = p->buf.status;
+  const size_t smem = 2 * X_TILE_BYTES + 4 * MAX_KEYS * 128 + sizeof(XShared) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(exchange_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  const long long tiles = (long long)g * ((dm.Nmid + XT - 1) / XT + (dm.Nhigh + XT - 1) / XT);
+  const int grid = tiles < p->sm_count ? (int)tiles : p->sm_count;
+  exchange_tc_kernel<<<grid, X_THREADS, smem, st>>>(*(const CUtensorMap*)p->tmap_x[0], *(const CUtensorMap*)p->tmap_x[1],
+                                                   *(const CUtensorMap*)p->tmap_x[2], *(const CUtensorMap*)p->tmap_x[3], P);
+  p->launches += 1;
+  return cudaGetLastError();
+}

@@ -96,6 +96,9 @@ struct ff_plan {
   bool tc_ok;                                  // tensor-core attention usable with this plan + workspace
   bool dct_tc_ok;                              // tensor-core transform usable
   int dct_group;                               // tensor-heads per tensor-core transform launch
+  bool xtc_ok;                                 // tensor-core exchange usable
+  int* pos_table;                              // rank -> flat coefficient index of the mid, then the high band (plan-owned)
+  alignas(64) unsigned char tmap_x[4][128];    // CUtensorMaps of the exchange kernel (Y / V~ of the mid and high bands)
   uint8_t* dct_images;                         // 6 x (hi, lo) matrix images of the tensor-core transform (plan-owned)
   alignas(64) unsigned char tmap_mid[128];     // CUtensorMap over the mid-band / high-band coefficient buffers
   alignas(64) unsigned char tmap_high[128];
@@ -119,6 +122,11 @@ size_t ffk_tc_work_bytes();
 bool ffk_tc_supported(const FFDims& dm);
 bool ffk_tc_prepare(ff_plan* p);               // builds the tensor maps over the workspace
 cudaError_t ffk_attention_tc(ff_plan* p, cudaStream_t st);
+// ---- tensor-core exchange (ff_exchange_tc.cu) -----------------------------------------------------
+bool ffk_exchange_tc_supported(const FFDims& dm);
+bool ffk_exchange_tc_build_tables(ff_plan* p);
+bool ffk_exchange_tc_prepare(ff_plan* p);
+cudaError_t ffk_exchange_tc(ff_plan* p, int h0, int g, void* grid_hi, void* grid_lo, cudaStream_t st);
 // ---- tensor-core transform (ff_dct_tc.cu) --------------------------------------------------------
 bool ffk_dct_tc_supported(const FFDims& dm);
 bool ffk_dct_tc_build_image(ff_plan* p, int axis, int inverse, const float* mat_host, int n);

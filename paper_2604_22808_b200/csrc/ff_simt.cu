@@ -401,16 +401,24 @@ constexpr int EXC_WARPS = 8;
 
 template <typename ST, int DPL, typename OT>
 __global__ void __launch_bounds__(EXC_WARPS * 32) exchange_recombine_kernel(FFBuffers buf, FFDims dm, int bh0,
-                                                                             OT* grid_out, OT* grid_lo) {
+                                                                             OT* grid_out, OT* grid_lo, int low_only) {
   extern __shared__ float S[];   // [3][m][d]
   const int gi = blockIdx.y, bh = bh0 + gi;
   const int d = dm.d, m = dm.m;
   for (int i = threadIdx.x; i < 3 * m * d; i += blockDim.x) S[i] = buf.summary[(size_t)bh * 3 * m * d + i];
   __syncthreads();
-  const long long f = (long long)blockIdx.x * EXC_WARPS + (threadIdx.x >> 5);
-  if (f >= dm.N) return;
+  // low_only: the launch covers the low band's coefficients only (the other bands are exchanged
+  // by the tensor-core kernel); the index is then a low rank, unravelled inside the low box.
+  long long f = (long long)blockIdx.x * EXC_WARPS + (threadIdx.x >> 5);
+  if (f >= (low_only ? dm.Nlow : dm.N)) return;
   const int lane = threadIdx.x & 31;
-  const int kw = (int)(f % dm.W), kh = (int)((f / dm.W) % dm.H), kt = (int)(f / ((long long)dm.W * dm.H));
+  int kw, kh, kt;
+  if (low_only) {
+    kw = (int)(f % dm.L[2]); kh = (int)((f / dm.L[2]) % dm.L[1]); kt = (int)(f / ((long long)dm.L[2] * dm.L[1]));
+    f = ((long long)kt * dm.H + kh) * dm.W + kw;
+  } else {
+    kw = (int)(f % dm.W); kh = (int)((f / dm.W) % dm.H); kt = (int)(f / ((long long)dm.W * dm.H));
+  }
   long long rank;
   const int band = ff_band_rank_of(dm, kt, kh, kw, &rank);
   const BandView<ST> v = band_view<ST>(buf, dm, bh, band);
@@ -572,9 +580,18 @@ static cudaError_t exchange_inverse_tc(ff_plan* p, void* out, cudaStream_t st) {
     const int g = (dm.BH - h0 < G) ? dm.BH - h0 : G;
     dim3 grid((unsigned)((dm.N + EXC_WARPS - 1) / EXC_WARPS), (unsigned)g);
     const size_t grid_bytes = ((size_t)G * dm.N * dm.d * 2 + 255) / 256 * 256;
-    exchange_recombine_kernel<__nv_bfloat16, 4, __nv_bfloat16><<<grid, EXC_WARPS * 32, smem, st>>>(
-        p->buf, dm, h0, (__nv_bfloat16*)p->buf.scratchA, (__nv_bfloat16*)((char*)p->buf.scratchA + grid_bytes));
-    e = cudaGetLastError();
+    __nv_bfloat16* ghi = (__nv_bfloat16*)p->buf.scratchA;
+    __nv_bfloat16* glo = (__nv_bfloat16*)((char*)p->buf.scratchA + grid_bytes);
+    if (p->xtc_ok) {
+      // mid and high bands on the tensor cores, the (small, fp32) low band with the generic kernel
+      dim3 lgrid((unsigned)((dm.Nlow + EXC_WARPS - 1) / EXC_WARPS), (unsigned)g);
+      exchange_recombine_kernel<__nv_bfloat16, 4, __nv_bfloat16><<<lgrid, EXC_WARPS * 32, smem, st>>>(p->buf, dm, h0, ghi, glo, 1);
+      e = cudaGetLastError();
+      if (e == cudaSuccess) e = ffk_exchange_tc(p, h0, g, ghi, glo, st);
+    } else {
+      exchange_recombine_kernel<__nv_bfloat16, 4, __nv_bfloat16><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, dm, h0, ghi, glo, 0);
+      e = cudaGetLastError();
+    }
     if (e != cudaSuccess) return e;
     p->launches += 1;
     e = ffk_inverse_transform_tc(p, h0, g, out, st);
@@ -596,7 +613,7 @@ static cudaError_t exchange_inverse_t(ff_plan* p, void* out, cudaStream_t st) {
     cudaError_t e = cudaSuccess;
 #define FF_EXC(DPL)                                                                                                   \
   e = cudaFuncSetAttribute(exchange_recombine_kernel<ST, DPL, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-  if (e == cudaSuccess) exchange_recombine_kernel<ST, DPL, float><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, dm, h0, p->buf.scratchA, (float*)nullptr);
+  if (e == cudaSuccess) exchange_recombine_kernel<ST, DPL, float><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, dm, h0, p->buf.scratchA, (float*)nullptr, 0);
     switch (dm.d / 32) {
       case 1: FF_EXC(1) break;
       case 2: FF_EXC(2) break;
