@@ -202,6 +202,37 @@ ff_status_t ff_get_tap(const ff_plan_t *plan, int32_t which, const void **dev_pt
  * 1 = force the generic SIMT kernel.  For tests. */
 ff_status_t ff_plan_set_attention_impl(ff_plan_t *plan, int32_t impl);
 
+/* ---- for callers that cannot allocate device memory ---------------------------------------------
+ *
+ * The paper has no counterpart of this entry point; it exists for integration reasons only.
+ *
+ * ff_high_attention_noalloc runs the high-band operator alone -- sliding-window softmax attention,
+ * |p - p'| <= radius, clipped to the band, scale 1/sqrt(128) -- on tensors the caller already holds,
+ * and calls no cudaMalloc, cudaFree or any other allocating routine.  It is meant for hosts where
+ * the plan-based calls above cannot be used because they need a fresh workspace: a serving process
+ * that handed every byte of device memory to its own pool at start-up (a raw allocation would fail
+ * or fragment the pool), a latency-critical loop that cannot afford the device-wide synchronisation
+ * an allocation implies, or a plug-in that is only ever given pointers.
+ *
+ *   q, k, v   device, bf16, contiguous [heads][n][128]: the band's tokens in band order
+ *   y         device, bf16, [heads][n][128]: the operator's output (written by the call)
+ *   heads     1 .. 1024;  n  1 .. 2^31-257;  larger sizes are rejected with FF_ERR_UNSUPPORTED
+ *   sync      non-zero: synchronise the stream before returning and report a device-side
+ *             FF_ERR_TIMEOUT; zero: return right after the launches
+ *
+ * The kernel's scratch (worklist, per-head masks, status word: 16 KB) lives in a fixed array inside
+ * the library image, so every GPU on which the library is loaded carries those 16 KB until the
+ * process ends.  The first call on a device looks up the array's device address and sets the
+ * kernel's shared-memory limit; make that first call before starting any stream capture.  All calls
+ * on a device share the one array, and it keeps what the previous call left: the call rewrites the
+ * masks and the worklist and clears the status word itself, but two calls whose kernels overlap on
+ * the GPU (different streams, or different host threads) would race on it -- serialise them.
+ * Errors: FF_ERR_INVALID_ARG (NULL or misaligned pointer, non-positive size), FF_ERR_UNSUPPORTED
+ * (beyond the limits above), FF_ERR_CUDA; the message is available from ff_last_error(NULL). */
+ff_status_t ff_high_attention_noalloc(const void *q, const void *k, const void *v, void *y,
+                                      int32_t heads, int64_t n, int32_t radius, int32_t sync,
+                                      void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -28,7 +28,7 @@ FF_BAND_LOW, FF_BAND_MID, FF_BAND_HIGH = 1, 2, 4
 EXPORTS = ("ff_config_validate", "ff_band_sizes", "ff_band_rank", "ff_workspace_bytes", "ff_workspace_bytes_host",
            "ff_plan_create", "ff_plan_workspace_bytes", "ff_plan_set_workspace", "ff_destroy", "ff_last_error",
            "ff_route", "ff_forward", "ff_forward_host", "ff_plan_device_status", "ff_plan_last_launches",
-           "ff_get_tap", "ff_plan_set_attention_impl", "ff_plan_set_profiling", "ff_plan_stage_times")
+           "ff_get_tap", "ff_plan_set_attention_impl", "ff_plan_set_profiling", "ff_plan_stage_times", "ff_high_attention_noalloc")
 STAGES = ("transform", "router", "attention", "summary", "inverse")
 
 
@@ -76,6 +76,7 @@ def library() -> C.CDLL:
         lib.ff_plan_set_attention_impl.argtypes = [C.c_void_p, C.c_int32]
         lib.ff_plan_set_profiling.argtypes = [C.c_void_p, C.c_int32]
         lib.ff_plan_stage_times.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
+        lib.ff_high_attention_noalloc.argtypes = [C.c_void_p] * 4 + [C.c_int32, C.c_int64, C.c_int32, C.c_int32, C.c_void_p]
         lib.ff_config_validate.argtypes = [C.POINTER(ff_config_t)]
         lib.ff_band_sizes.argtypes = [C.POINTER(ff_config_t), C.POINTER(C.c_int64)]
         lib.ff_band_rank.argtypes = [C.POINTER(ff_config_t), C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_int32),
@@ -275,6 +276,22 @@ def ff_forward(plan: Plan, Q, K, V, out, alloc=None, timesteps=None):
 
 def ff_forward_host(plan: Plan, Qh, Kh, Vh, out_h, alloc_host=None, timesteps=None):
     return plan.forward_host(Qh, Kh, Vh, out_h, alloc_host, timesteps)
+
+
+def ff_high_attention_noalloc(q, k, v, y, radius: int, sync: bool = True):
+    """High-band sliding-window attention on bf16 CUDA tensors [heads][n][128] without any device
+    allocation inside the call (the kernel's scratch is a fixed array in the library): for hosts
+    whose device memory is fully owned by their own pool, or that cannot tolerate the device-wide
+    synchronisation of an allocation.  Calls on one device share that scratch: do not overlap them."""
+    import torch
+    for t in (q, k, v, y):
+        if t.dtype != torch.bfloat16 or not t.is_contiguous() or t.dim() != 3 or t.shape[2] != 128 or t.shape != q.shape:
+            raise FFError(1, "expected contiguous bf16 CUDA tensors of one shape [heads][n][128]")
+    stream = C.c_void_p(torch.cuda.current_stream(q.device).cuda_stream)
+    with torch.cuda.device(q.device):
+        _check(library().ff_high_attention_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), y.data_ptr(), q.shape[0],
+                                                   q.shape[1], radius, int(sync), stream))
+    return y
 
 
 def ff_destroy(plan: Plan):

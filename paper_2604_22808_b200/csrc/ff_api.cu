@@ -12,6 +12,8 @@
 
 static thread_local char g_err[512] = "";
 
+void ff_set_thread_error(const char* msg) { snprintf(g_err, 512, "%s", msg ? msg : ""); }
+
 static ff_status_t fail(ff_plan* p, ff_status_t code, const char* fmt, const char* a = "", long long x = 0,
                         long long y = 0) {
   char* dst = p ? p->err : g_err;

@@ -142,9 +142,13 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-__global__ void __launch_bounds__(TC_THREADS, 1)
-attention_tc_kernel(const __grid_constant__ CUtensorMap map_mid, const __grid_constant__ CUtensorMap map_high,
-                    const TcParams P) {
+// The kernel body.  QKV_MAPS = false: map_a / map_b cover the plan's mid / high coefficient buffers,
+// which hold Q~, K~ and V~ of head bh in slices bh, BH + bh and 2 BH + bh.  QKV_MAPS = true (the entry
+// point that allocates nothing): map_a, map_b, map_c are the caller's separate Q, K, V tensors of one
+// band, head bh in slice bh.
+template <bool QKV_MAPS>
+__device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, const CUtensorMap& map_b,
+                                                  const CUtensorMap& map_c, const TcParams& P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sQ = smem;                       // 2 x 32 KB
@@ -183,26 +187,30 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_mid, const __grid_co
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      tma_prefetch_desc(&map_mid); tma_prefetch_desc(&map_high);
+      tma_prefetch_desc(&map_a); tma_prefetch_desc(&map_b);
       int iter = 0; unsigned g = 0;
       bool ok = true;
       for (int it = blockIdx.x; it < total && ok; it += gridDim.x, ++iter) {
         const Item x = decode_item(sh, dm, it);
-        const CUtensorMap* map = x.band == 1 ? &map_mid : &map_high;
+        const CUtensorMap* map = x.band == 1 ? &map_a : &map_b;
+        const CUtensorMap* mapq = QKV_MAPS ? &map_a : map;
+        const CUtensorMap* mapk = QKV_MAPS ? &map_b : map;
+        const CUtensorMap* mapv = QKV_MAPS ? &map_c : map;
+        const int slice_k = QKV_MAPS ? x.bh : dm.BH + x.bh, slice_v = QKV_MAPS ? x.bh : 2 * dm.BH + x.bh;
         const int rb = x.band == 1 ? P.rb_mid : TILE;
         const int qb = iter & 1;
         if (iter >= 2) ok = mbar_wait(&sh.q_empty[qb], ((iter >> 1) - 1) & 1, abort_flag);
         if (!ok) break;
-        load_tile(sQ + qb * TILE_BYTES, map, &sh.q_full[qb], dm, x, x.bh, (long long)x.tile * TILE, rb);
+        load_tile(sQ + qb * TILE_BYTES, mapq, &sh.q_full[qb], dm, x, x.bh, (long long)x.tile * TILE, rb);
         for (int j = 0; j < x.nk && ok; ++j, ++g) {
           const int st = g & 1;
           const long long first = x.band == 1 ? (long long)j * TILE : x.ks + (long long)j * TILE;
           if (g >= 2) ok = mbar_wait(&sh.k_empty[st], ((g >> 1) - 1) & 1, abort_flag);
           if (!ok) break;
-          load_tile(sK + st * TILE_BYTES, map, &sh.k_full[st], dm, x, dm.BH + x.bh, first, rb);
+          load_tile(sK + st * TILE_BYTES, mapk, &sh.k_full[st], dm, x, slice_k, first, rb);
           if (g >= 2) ok = mbar_wait(&sh.v_empty[st], ((g >> 1) - 1) & 1, abort_flag);
           if (!ok) break;
-          load_tile(sV + st * TILE_BYTES, map, &sh.v_full[st], dm, x, 2 * dm.BH + x.bh, first, rb);
+          load_tile(sV + st * TILE_BYTES, mapv, &sh.v_full[st], dm, x, slice_v, first, rb);
         }
       }
     }
@@ -417,6 +425,26 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_mid, const __grid_co
   }
 }
 
+__global__ void __launch_bounds__(TC_THREADS, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap map_mid, const __grid_constant__ CUtensorMap map_high,
+                    const TcParams P) {
+  attention_tc_body<false>(map_mid, map_high, map_high, P);
+}
+
+// Same kernel on the caller's separate Q, K, V tensors of one band (see ff_high_attention_noalloc).
+__global__ void __launch_bounds__(TC_THREADS, 1)
+attention_tc_qkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                        const __grid_constant__ CUtensorMap map_v, const TcParams P) {
+  attention_tc_body<true>(map_q, map_k, map_v, P);
+}
+
+// Scratch of ff_high_attention_noalloc: the worklist, one band mask per head and a status word.
+// 16 KB in every GPU context that loads this library, held until the process exits.
+constexpr int NOALLOC_MAX_HEADS = MAX_UNITS;
+constexpr size_t NOALLOC_WORK_BYTES = ((2 + 3 * MAX_UNITS + 1) * sizeof(int) + 255) / 256 * 256;
+constexpr size_t NOALLOC_BYTES = NOALLOC_WORK_BYTES + NOALLOC_MAX_HEADS + 256;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -475,4 +503,84 @@ cudaError_t ffk_attention_tc(ff_plan* p, cudaStream_t st) {
                                                              *(const CUtensorMap*)p->tmap_high, P);
   p->launches += 2;
   return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// ff_high_attention_noalloc: the high-band operator for callers that cannot allocate.
+// ------------------------------------------------------------------------------------------------
+#include <mutex>
+
+extern "C" ff_status_t ff_high_attention_noalloc(const void* q, const void* k, const void* v, void* y, int32_t heads,
+                                                 int64_t n, int32_t radius, int32_t sync, void* cuda_stream) {
+  if (!q || !k || !v || !y) { ff_set_thread_error("ff_high_attention_noalloc: a tensor pointer is NULL"); return FF_ERR_INVALID_ARG; }
+  if ((((uintptr_t)q) | ((uintptr_t)k) | ((uintptr_t)v) | ((uintptr_t)y)) & 15) {
+    ff_set_thread_error("ff_high_attention_noalloc: tensors must be 16-byte aligned");
+    return FF_ERR_INVALID_ARG;
+  }
+  if (heads < 1 || n < 1 || radius < 0) {
+    ff_set_thread_error("ff_high_attention_noalloc: need heads >= 1, n >= 1, radius >= 0");
+    return FF_ERR_INVALID_ARG;
+  }
+  if (heads > NOALLOC_MAX_HEADS || n >= (1LL << 31) - 256) {
+    ff_set_thread_error("ff_high_attention_noalloc: the built-in scratch covers at most 1024 heads and 2^31-257 tokens per head");
+    return FF_ERR_UNSUPPORTED;
+  }
+  // Device address of the scratch array, looked up once per device with that device current: in host
+  // code the array's name is only a handle, not an address a kernel could use.
+  static std::mutex mu;
+  static unsigned char* dev_scratch[64] = {};
+  static int sm_counts[64] = {};
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= 64) { ff_set_thread_error("ff_high_attention_noalloc: no usable current device"); return FF_ERR_CUDA; }
+  unsigned char* scratch = nullptr;
+  int sms = 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!dev_scratch[dev]) {
+      void* ptr = nullptr;
+      e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+      if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_counts[dev], cudaDevAttrMultiProcessorCount, dev);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(attention_tc_qkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(6 * TILE_BYTES + sizeof(Shared) + 1024));
+      if (e != cudaSuccess || !ptr) { ff_set_thread_error(cudaGetErrorString(e)); return FF_ERR_CUDA; }
+      dev_scratch[dev] = (unsigned char*)ptr;
+    }
+    scratch = dev_scratch[dev];
+    sms = sm_counts[dev];
+  }
+  CUtensorMap mq, mk, mv;
+  if (!encode_band_map(&mq, const_cast<void*>(q), n, heads, TILE) || !encode_band_map(&mk, const_cast<void*>(k), n, heads, TILE) ||
+      !encode_band_map(&mv, const_cast<void*>(v), n, heads, TILE)) {
+    ff_set_thread_error("ff_high_attention_noalloc: could not encode the tensor maps");
+    return FF_ERR_CUDA;
+  }
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  TcParams P{};
+  P.dm.B = 1; P.dm.heads = heads; P.dm.BH = heads; P.dm.d = HD; P.dm.R = radius;
+  P.dm.Nhigh = n; P.dm.Nmid = 0; P.dm.nb = 0; P.dm.s = 1; P.dm.b = TILE; P.dm.r = 1;
+  P.work = (int*)scratch;
+  uint8_t* masks = scratch + NOALLOC_WORK_BYTES;
+  P.alloc = masks;
+  P.status = (int*)(scratch + NOALLOC_WORK_BYTES + NOALLOC_MAX_HEADS);
+  P.y_mid = nullptr; P.y_high = (__nv_bfloat16*)y; P.rb_mid = TILE;
+  // The array keeps the previous call's contents: rewrite the masks and clear the status word; the
+  // worklist is rebuilt by its kernel.
+  e = cudaMemsetAsync(masks, FF_BAND_HIGH, (size_t)heads, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(P.status, 0, sizeof(int), st);
+  if (e == cudaSuccess) { build_worklist_kernel<<<1, 32, 0, st>>>(P); e = cudaGetLastError(); }
+  if (e == cudaSuccess) {
+    attention_tc_qkv_kernel<<<sms, TC_THREADS, 6 * TILE_BYTES + sizeof(Shared) + 1024, st>>>(mq, mk, mv, P);
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) { ff_set_thread_error(cudaGetErrorString(e)); return FF_ERR_CUDA; }
+  if (sync) {
+    int word = 0;
+    e = cudaMemcpyAsync(&word, P.status, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) { ff_set_thread_error(cudaGetErrorString(e)); return FF_ERR_CUDA; }
+    if (word != 0) { ff_set_thread_error("ff_high_attention_noalloc: a bounded device-side wait expired"); return FF_ERR_TIMEOUT; }
+  }
+  return FF_OK;
 }

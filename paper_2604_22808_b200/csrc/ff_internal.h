@@ -109,6 +109,9 @@ struct ff_plan {
   char err[512];
 };
 
+// Records `msg` as the calling thread's plan-less error (what ff_last_error(NULL) returns).
+void ff_set_thread_error(const char* msg);
+
 void ff_compute_layout(const FFDims& dm, bool with_staging, FFLayout* lay);
 
 // ---- kernel launchers (ff_simt.cu).  Each returns the cudaError_t of its launches. --------------
