@@ -365,33 +365,75 @@ __device__ __forceinline__ BandView<ST> band_view(const FFBuffers& buf, const FF
 }
 
 // Summary tokens S = U_l Pool(Y^(l)): segment j covers [floor(j n/m), max(a+1, floor((j+1) n/m))).
+// Two steps: segment sums (each segment split over several CTAs, 16-byte loads, partial sums
+// added atomically into the summary buffer), then mean and projection in place.
+constexpr int SUM_THREADS = 256;
+
 template <typename ST>
-__global__ void summary_kernel(FFBuffers buf, const float* U, FFDims dm) {
-  __shared__ float pooled[128];
-  __shared__ float part[8][128];
-  const int j = blockIdx.x, band = blockIdx.y, bh = blockIdx.z;
-  const int d = dm.d;
+__global__ void __launch_bounds__(SUM_THREADS) summary_partial_kernel(FFBuffers buf, FFDims dm, int split) {
+  __shared__ float red[128];
+  const int j = blockIdx.x / split, piece = blockIdx.x % split, band = blockIdx.y, bh = blockIdx.z;
+  const int d = dm.d, vecs = d / 8;                // 8-channel vectors per row
   const BandView<ST> v = band_view<ST>(buf, dm, bh, band);
   const long long a = ((long long)j * v.n) / dm.m;
   long long e = ((long long)(j + 1) * v.n) / dm.m;
   if (e < a + 1) e = a + 1;
-  const int c = threadIdx.x % d, sub = threadIdx.x / d, nsub = blockDim.x / d;
-  float acc = 0.f;
-  for (long long p = a + sub; p < e; p += nsub)
-    acc += v.f32 ? v.f32[(size_t)p * d + c] : ldf<ST>(v.st + (size_t)p * d + c);
-  part[sub][c] = acc;
+  const long long chunk = (e - a + split - 1) / split;
+  const long long r0 = a + piece * chunk;
+  const long long r1 = r0 + chunk < e ? r0 + chunk : e;
+  const int vec = threadIdx.x % vecs, rsub = threadIdx.x / vecs, nrs = SUM_THREADS / vecs;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (rsub < nrs) {
+    for (long long p = r0 + rsub; p < r1; p += nrs) {
+      if (v.f32) {
+        const float4 x0 = *(const float4*)(v.f32 + (size_t)p * d + vec * 8);
+        const float4 x1 = *(const float4*)(v.f32 + (size_t)p * d + vec * 8 + 4);
+        acc[0] += x0.x; acc[1] += x0.y; acc[2] += x0.z; acc[3] += x0.w;
+        acc[4] += x1.x; acc[5] += x1.y; acc[6] += x1.z; acc[7] += x1.w;
+      } else if (sizeof(ST) == 4) {
+        const float4 x0 = *(const float4*)((const float*)v.st + (size_t)p * d + vec * 8);
+        const float4 x1 = *(const float4*)((const float*)v.st + (size_t)p * d + vec * 8 + 4);
+        acc[0] += x0.x; acc[1] += x0.y; acc[2] += x0.z; acc[3] += x0.w;
+        acc[4] += x1.x; acc[5] += x1.y; acc[6] += x1.z; acc[7] += x1.w;
+      } else {
+        const uint4 x = *(const uint4*)((const __nv_bfloat16*)v.st + (size_t)p * d + vec * 8);
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          acc[2 * i] += __uint_as_float(w[i] << 16);
+          acc[2 * i + 1] += __uint_as_float(w[i] & 0xffff0000u);
+        }
+      }
+    }
+  }
+  // combine the row groups: channel sums through shared-memory atomics, then one global atomic per channel
+  if (threadIdx.x < 128) red[threadIdx.x] = 0.f;
   __syncthreads();
-  if (sub == 0) {
-    for (int s2 = 1; s2 < nsub; ++s2) acc += part[s2][c];
-    pooled[c] = acc / (float)(e - a);
+  if (rsub < nrs) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) atomicAdd(&red[vec * 8 + i], acc[i]);
   }
   __syncthreads();
-  if (sub == 0) {
-    const float* Ul = U + ((size_t)band * d + c) * d;
-    float s = 0.f;
-    for (int i = 0; i < d; ++i) s = fmaf(Ul[i], pooled[i], s);
-    buf.summary[(((size_t)bh * 3 + band) * dm.m + j) * d + c] = s;
-  }
+  if (threadIdx.x < d && r0 < r1)
+    atomicAdd(buf.summary + (((size_t)bh * 3 + band) * dm.m + j) * d + threadIdx.x, red[threadIdx.x]);
+}
+
+template <typename ST>
+__global__ void summary_finalize_kernel(FFBuffers buf, const float* U, FFDims dm) {
+  __shared__ float pooled[128];
+  const int j = blockIdx.x, band = blockIdx.y, bh = blockIdx.z;
+  const int d = dm.d, c = threadIdx.x;
+  const BandView<ST> v = band_view<ST>(buf, dm, bh, band);
+  const long long a = ((long long)j * v.n) / dm.m;
+  long long e = ((long long)(j + 1) * v.n) / dm.m;
+  if (e < a + 1) e = a + 1;
+  float* S = buf.summary + (((size_t)bh * 3 + band) * dm.m + j) * d;
+  pooled[c] = S[c] / (float)(e - a);
+  __syncthreads();
+  const float* Ul = U + ((size_t)band * d + c) * d;
+  float s = 0.f;
+  for (int i = 0; i < d; ++i) s = fmaf(Ul[i], pooled[i], s);
+  S[c] = s;
 }
 
 // Exchange + recombination ("Cross-band residual exchange", "Reconstruction"): for every
@@ -560,11 +602,22 @@ cudaError_t ffk_attention_simt(ff_plan* p, int band_bits, cudaStream_t st) {
 
 cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st) {
   const FFDims& dm = p->dm;
-  dim3 grid((unsigned)dm.m, 3, (unsigned)dm.BH);
-  int nsub = 1024 / dm.d; if (nsub > 8) nsub = 8;
-  if (dm.fp32) summary_kernel<float><<<grid, nsub * dm.d, 0, st>>>(p->buf, p->U, dm);
-  else summary_kernel<__nv_bfloat16><<<grid, nsub * dm.d, 0, st>>>(p->buf, p->U, dm);
-  p->launches += 1;
+  cudaError_t e = cudaMemsetAsync(p->buf.summary, 0, (size_t)dm.BH * 3 * dm.m * dm.d * sizeof(float), st);
+  if (e != cudaSuccess) return e;
+  // split every segment so that each CTA reads about 256 rows of the longest band
+  long long longest = dm.Nhigh > dm.Nmid ? dm.Nhigh : dm.Nmid;
+  int split = (int)((longest / dm.m + 255) / 256);
+  if (split < 1) split = 1;
+  if (split > 64) split = 64;
+  dim3 pgrid((unsigned)(dm.m * split), 3, (unsigned)dm.BH), fgrid((unsigned)dm.m, 3, (unsigned)dm.BH);
+  if (dm.fp32) {
+    summary_partial_kernel<float><<<pgrid, SUM_THREADS, 0, st>>>(p->buf, dm, split);
+    summary_finalize_kernel<float><<<fgrid, dm.d, 0, st>>>(p->buf, p->U, dm);
+  } else {
+    summary_partial_kernel<__nv_bfloat16><<<pgrid, SUM_THREADS, 0, st>>>(p->buf, dm, split);
+    summary_finalize_kernel<__nv_bfloat16><<<fgrid, dm.d, 0, st>>>(p->buf, p->U, dm);
+  }
+  p->launches += 2;
   return cudaGetLastError();
 }
 
