@@ -64,10 +64,15 @@ struct DctTcParams {
   int* status;
 };
 
+constexpr int STG_PITCH = 80;                       // bytes per staged row piece (64 B of data, padded against bank conflicts)
+
 struct DctShared {
   uint64_t full[MAX_STAGE], empty[MAX_STAGE], acc_full[NACC], acc_empty[NACC], img_full;
   uint32_t tmem_base;
   int abort_flag;
+  // per epilogue warp: 32 rows x 64 bytes of hi and of lo, to turn one-row-per-thread registers
+  // into stores where four lanes cover a row's 64 contiguous bytes
+  alignas(16) uint8_t stage[4][2][32 * STG_PITCH];
 };
 
 // Grid coordinates (w, h, t) of the first position of tile `u` of a tensor-head.  A tile holds
@@ -253,6 +258,14 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
         if (P.mode != MODE_LAST) row_lo = P.dst_lo + o;
         if (P.mode == MODE_FIRST && a < dm.L[2]) row_f32 = P.side + ((((size_t)gi * dm.T + t) * dm.H + h + l) * dm.L[2] + a) * CH;
       }
+      // lane L stores for rows 8 i + L/4 of its warp: fetch those rows' destinations
+      __nv_bfloat16* dst_hi[4]; __nv_bfloat16* dst_lo[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int src = 8 * i + (lane >> 2);
+        dst_hi[i] = (__nv_bfloat16*)__shfl_sync(0xffffffffu, (unsigned long long)row_hi, src);
+        dst_lo[i] = (__nv_bfloat16*)__shfl_sync(0xffffffffu, (unsigned long long)row_lo, src);
+      }
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         uint32_t r[32];
@@ -287,7 +300,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
           }
           em[q] += sm_[0]; eh[q] += sh_[0];
         }
-        if (row_hi) {
+        {
           uint32_t hi[16], lo[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
@@ -297,12 +310,21 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
             const __nv_bfloat162 lp = __floats2bfloat162_rn(v0 - __uint_as_float(hi[i] << 16), v1 - __uint_as_float(hi[i] & 0xffff0000u));
             lo[i] = *(const uint32_t*)&lp;
           }
+          uint8_t* st_hi = sh.stage[quarter][0];
+          uint8_t* st_lo = sh.stage[quarter][1];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) *(uint4*)(row_hi + q * 32 + i * 8) = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
-          if (row_lo) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) *(uint4*)(row_lo + q * 32 + i * 8) = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
+          for (int i = 0; i < 4; ++i) {
+            *(uint4*)(st_hi + lane * STG_PITCH + i * 16) = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
+            *(uint4*)(st_lo + lane * STG_PITCH + i * 16) = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
           }
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int rr = 8 * i + (lane >> 2), piece = lane & 3;      // row of the warp, 16-byte piece of its 64 bytes
+            if (dst_hi[i]) *(uint4*)(dst_hi[i] + q * 32 + piece * 8) = *(const uint4*)(st_hi + rr * STG_PITCH + piece * 16);
+            if (dst_lo[i]) *(uint4*)(dst_lo[i] + q * 32 + piece * 8) = *(const uint4*)(st_lo + rr * STG_PITCH + piece * 16);
+          }
+          __syncwarp();
         }
       }
       tc_fence_before();
@@ -325,61 +347,71 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
   }
 }
 
-// Low band at full precision from the fp32 copy of the w-transformed columns k_w < L_w:
+// Low band at full precision from the fp32 copy of the w-transformed rows k_w < L_w:
 //   low[k_t][k_h][k_w][c] = sum_t C_T[k_t][t] sum_h C_H[k_h][h] side[t][h][k_w][c]
-// One CTA per (tensor-head, k_h, k_w); thread = (t group, channel); the t groups are combined through
-// shared memory.  Also accumulates the low band's energy.
-constexpr int LOW_MAX_LT = 16;
-constexpr int LOW_TG = 8;
+// One CTA per (tensor-head, k_w) computes every (k_t, k_h) of the low box, in chunks of 8 x 8, so the
+// side buffer is read once per chunk pair; thread = (t group, channel); the t groups are combined
+// through shared memory.  Also accumulates the low band's energy.
+constexpr int LOW_CH = 8;        // k_t and k_h chunk
+constexpr int LOW_TG = 4;
 
 __global__ void __launch_bounds__(CH * LOW_TG) low_band_kernel(const float* side, const float* CT, const float* CHm,
                                                                float* spec_low, double* energy, FFDims dm, int group_start) {
-  const int kw = blockIdx.x % dm.L[2], kh = blockIdx.x / dm.L[2];
+  const int kw = blockIdx.x;
   const int gi = blockIdx.y, th = group_start + gi;
   const int c = threadIdx.x % CH, tg = threadIdx.x / CH;
-  __shared__ float ch_row[128];
-  __shared__ float red[LOW_MAX_LT][CH];
-  for (int i = threadIdx.x; i < dm.H; i += CH * LOW_TG) ch_row[i] = CHm[(size_t)kh * dm.H + i];
+  __shared__ float ch_rows[LOW_CH][128];          // C_H rows of the current k_h chunk
+  __shared__ float red[LOW_CH * LOW_CH][CH];
   float e = 0.f;
-  for (int kt0 = 0; kt0 < dm.L[0]; kt0 += LOW_MAX_LT) {
-    for (int i = threadIdx.x; i < LOW_MAX_LT * CH; i += CH * LOW_TG) red[i / CH][i % CH] = 0.f;
+  for (int kh0 = 0; kh0 < dm.L[1]; kh0 += LOW_CH) {
     __syncthreads();
-    float acc[LOW_MAX_LT];
-#pragma unroll
-    for (int i = 0; i < LOW_MAX_LT; ++i) acc[i] = 0.f;
-    for (int t = tg; t < dm.T; t += LOW_TG) {
-      const float* col = side + ((((size_t)gi * dm.T + t) * dm.H) * dm.L[2] + kw) * CH + c;
-      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-      int h = 0;
-      for (; h + 3 < dm.H; h += 4) {
-        s0 = fmaf(ch_row[h], col[(size_t)h * dm.L[2] * CH], s0);
-        s1 = fmaf(ch_row[h + 1], col[(size_t)(h + 1) * dm.L[2] * CH], s1);
-        s2 = fmaf(ch_row[h + 2], col[(size_t)(h + 2) * dm.L[2] * CH], s2);
-        s3 = fmaf(ch_row[h + 3], col[(size_t)(h + 3) * dm.L[2] * CH], s3);
-      }
-      for (; h < dm.H; ++h) s0 = fmaf(ch_row[h], col[(size_t)h * dm.L[2] * CH], s0);
-      const float sh_ = (s0 + s1) + (s2 + s3);
-#pragma unroll
-      for (int i = 0; i < LOW_MAX_LT; ++i)
-        if (kt0 + i < dm.L[0]) acc[i] = fmaf(CT[(size_t)(kt0 + i) * dm.T + t], sh_, acc[i]);
+    for (int i = threadIdx.x; i < LOW_CH * dm.H; i += CH * LOW_TG) {
+      const int q = i / dm.H, h = i % dm.H;
+      ch_rows[q][h] = kh0 + q < dm.L[1] ? CHm[(size_t)(kh0 + q) * dm.H + h] : 0.f;
     }
+    for (int kt0 = 0; kt0 < dm.L[0]; kt0 += LOW_CH) {
+      for (int i = threadIdx.x; i < LOW_CH * LOW_CH * CH; i += CH * LOW_TG) red[i / CH][i % CH] = 0.f;
+      __syncthreads();
+      float acc[LOW_CH][LOW_CH];                    // [k_t][k_h]
 #pragma unroll
-    for (int i = 0; i < LOW_MAX_LT; ++i)
-      if (kt0 + i < dm.L[0]) atomicAdd(&red[i][c], acc[i]);
-    __syncthreads();
-    if (tg == 0) {
+      for (int i = 0; i < LOW_CH; ++i)
 #pragma unroll
-      for (int i = 0; i < LOW_MAX_LT; ++i) {
-        if (kt0 + i >= dm.L[0]) break;
-        const long long rank = ((long long)(kt0 + i) * dm.L[1] + kh) * dm.L[2] + kw;
-        const float v = red[i][c];
+        for (int q = 0; q < LOW_CH; ++q) acc[i][q] = 0.f;
+      for (int t = tg; t < dm.T; t += LOW_TG) {
+        const float* col = side + ((((size_t)gi * dm.T + t) * dm.H) * dm.L[2] + kw) * CH + c;
+        float s[LOW_CH];
+#pragma unroll
+        for (int q = 0; q < LOW_CH; ++q) s[q] = 0.f;
+        for (int h = 0; h < dm.H; ++h) {
+          const float x = col[(size_t)h * dm.L[2] * CH];
+#pragma unroll
+          for (int q = 0; q < LOW_CH; ++q) s[q] = fmaf(ch_rows[q][h], x, s[q]);
+        }
+#pragma unroll
+        for (int i = 0; i < LOW_CH; ++i) {
+          const float ct = kt0 + i < dm.L[0] ? CT[(size_t)(kt0 + i) * dm.T + t] : 0.f;
+#pragma unroll
+          for (int q = 0; q < LOW_CH; ++q) acc[i][q] = fmaf(ct, s[q], acc[i][q]);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < LOW_CH; ++i)
+#pragma unroll
+        for (int q = 0; q < LOW_CH; ++q)
+          if (kt0 + i < dm.L[0] && kh0 + q < dm.L[1]) atomicAdd(&red[i * LOW_CH + q][c], acc[i][q]);
+      __syncthreads();
+      for (int o = tg; o < LOW_CH * LOW_CH; o += LOW_TG) {
+        const int i = o / LOW_CH, q = o % LOW_CH;
+        if (kt0 + i >= dm.L[0] || kh0 + q >= dm.L[1]) continue;
+        const long long rank = ((long long)(kt0 + i) * dm.L[1] + kh0 + q) * dm.L[2] + kw;
+        const float v = red[o][c];
         spec_low[((size_t)th * dm.Nlow + rank) * CH + c] = v;
         e = fmaf(v, v, e);
       }
+      __syncthreads();
     }
-    __syncthreads();
   }
-  if (energy && tg == 0) atomicAdd(energy + ((size_t)((th % dm.BH) / dm.heads) * 3) * CH + c, (double)e);
+  if (energy) atomicAdd(energy + ((size_t)((th % dm.BH) / dm.heads) * 3) * CH + c, (double)e);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -518,7 +550,7 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
     P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 0 + 0) * TILE_BYTES; P.dst = nullptr;
     e = launch_pass(p, m2h, m2l, m2l, P, st);
     if (e != cudaSuccess) return e;
-    dim3 lgrid((unsigned)(dm.L[1] * dm.L[2]), (unsigned)g);
+    dim3 lgrid((unsigned)dm.L[2], (unsigned)g);
     low_band_kernel<<<lgrid, CH * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
     p->launches += 1;
     e = cudaGetLastError();
