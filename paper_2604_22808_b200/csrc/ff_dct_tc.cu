@@ -277,28 +277,42 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
             *(uint4*)(row_f32 + q * 32 + i * 4) = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
         }
         if (P.mode == MODE_SPLIT && P.energy) {
-          // channel energies of this 32-channel chunk, summed over the warp's 32 rows with a
-          // halving butterfly: afterwards lane k holds the sum for channel 32 q + k
-          float sm_[32], sh_[32];
+          // Channel energies of this 32-channel chunk, summed over the warp's 32 rows with a halving
+          // butterfly (afterwards lane k holds the sum for channel 32 q + k): one butterfly for the
+          // mid + high rows together, a second one for the mid rows only where the warp has any;
+          // the high band's energy is the difference.
+          const bool any_mid = __any_sync(0xffffffffu, band == 1);
+          float sa[32], sm_[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             const float v = __uint_as_float(r[i]);
             const float v2 = v * v;
+            sa[i] = band != 0 ? v2 : 0.f;
             sm_[i] = band == 1 ? v2 : 0.f;
-            sh_[i] = band == 2 ? v2 : 0.f;
           }
 #pragma unroll
           for (int step = 16; step >= 1; step >>= 1) {
             const bool upper = lane & step;
 #pragma unroll
             for (int i = 0; i < step; ++i) {
-              const float keep_m = upper ? sm_[i + step] : sm_[i], send_m = upper ? sm_[i] : sm_[i + step];
-              const float keep_h = upper ? sh_[i + step] : sh_[i], send_h = upper ? sh_[i] : sh_[i + step];
-              sm_[i] = keep_m + __shfl_xor_sync(0xffffffffu, send_m, step);
-              sh_[i] = keep_h + __shfl_xor_sync(0xffffffffu, send_h, step);
+              const float keep = upper ? sa[i + step] : sa[i], send = upper ? sa[i] : sa[i + step];
+              sa[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
             }
           }
-          em[q] += sm_[0]; eh[q] += sh_[0];
+          if (any_mid) {
+#pragma unroll
+            for (int step = 16; step >= 1; step >>= 1) {
+              const bool upper = lane & step;
+#pragma unroll
+              for (int i = 0; i < step; ++i) {
+                const float keep = upper ? sm_[i + step] : sm_[i], send = upper ? sm_[i] : sm_[i + step];
+                sm_[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
+              }
+            }
+            em[q] += sm_[0]; eh[q] += sa[0] - sm_[0];
+          } else {
+            eh[q] += sa[0];
+          }
         }
         {
           uint32_t hi[16], lo[16];

@@ -4,7 +4,9 @@
 // written to the coefficient grid at the position of band rank p (a table built at plan creation).
 //
 // A CTA owns a contiguous run of (head, band, 128-rank tile) items, so the summary tokens of a head
-// are re-staged only a few times per CTA.  Per tile:
+// are re-staged only a few times per CTA.
+// Two CTAs share an SM (256 tensor-memory columns each), which overlaps one tile's softmax and
+// stores with the other's MMAs and loads.  Per tile:
 //   TMA     the 128 band tokens (operator output where the head's mask has the band, V~ otherwise)
 //   MMA 1   S[128 x 3m] = Y Z^T against all 3m summaries of the head (own band masked in the softmax)
 //   softmax one token per thread (row = TMEM lane); normalised P written back to TMEM as bf16 hi + lo
@@ -27,7 +29,6 @@ constexpr int XD = 128;                 // head_dim
 constexpr int X_TILE_BYTES = XT * XD * 2;
 constexpr int X_HALF = X_TILE_BYTES / 2;
 constexpr int X_THREADS = 192;
-constexpr int MAX_KEYS = 96;            // 3m rounded up to 16, m <= 32
 
 struct XParams {
   FFDims dm;
@@ -39,6 +40,7 @@ struct XParams {
   __nv_bfloat16* grid_lo;
   int h0, g;                  // heads [h0, h0+g)
   int nkeys;                  // 3m rounded up to a multiple of 16
+  int ybufs;                  // token-tile buffers in shared memory (1 or 2)
   int* status;
 };
 
@@ -50,6 +52,12 @@ struct XShared {
 
 struct XItem { int bh, band, tile; };
 
+__device__ __forceinline__ float ex2f_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __device__ __forceinline__ XItem x_decode(const FFDims& dm, int h0, int it, int tm, int th) {
   XItem x;
   const int per = tm + th;
@@ -60,16 +68,16 @@ __device__ __forceinline__ XItem x_decode(const FFDims& dm, int h0, int it, int 
   return x;
 }
 
-__global__ void __launch_bounds__(X_THREADS, 1)
+__global__ void __launch_bounds__(X_THREADS, 2)
 exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_constant__ CUtensorMap map_v_mid,
                    const __grid_constant__ CUtensorMap map_y_high, const __grid_constant__ CUtensorMap map_v_high,
                    const XParams P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* sY = smem;                                    // 2 x 32 KB
-  uint8_t* sZhi = smem + 2 * X_TILE_BYTES;               // [2 halves][nkeys rows][128 B]
-  uint8_t* sZlo = sZhi + 2 * MAX_KEYS * 128;
-  XShared& sh = *(XShared*)(sZlo + 2 * MAX_KEYS * 128);
+  uint8_t* sY = smem;                                    // ybufs x 32 KB
+  uint8_t* sZhi = smem + P.ybufs * X_TILE_BYTES;         // [2 halves][nkeys rows][128 B]
+  uint8_t* sZlo = sZhi + 2 * P.nkeys * 128;
+  XShared& sh = *(XShared*)(sZlo + 2 * P.nkeys * 128);
   const FFDims& dm = P.dm;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m = dm.m, nk = P.nkeys;
@@ -86,13 +94,14 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
     sh.abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 1) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc(&sh.tmem_base, 256); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sh.tmem_base;
   volatile int* abort_flag = &sh.abort_flag;
-  // tensor-memory columns: S [0,96)  P_hi [128,176)  P_lo [192,240)  D [256,384)
+  // tensor-memory columns: S [0,96), overwritten by P_hi [0,48) and P_lo [48,96);  D [128,256)
+  const int YB = P.ybufs;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -103,8 +112,8 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         const bool exec = P.alloc[x.bh] & (1 << x.band);
         const CUtensorMap* map = x.band == 1 ? (exec ? &map_y_mid : &map_v_mid) : (exec ? &map_y_high : &map_v_high);
         const int slice = exec ? x.bh : 2 * dm.BH + x.bh;
-        const int slot = n & 1;
-        if (n >= 2) ok = mbar_wait(&sh.y_empty[slot], ((n >> 1) - 1) & 1, abort_flag);
+        const int slot = n % YB;
+        if (n >= YB) ok = mbar_wait(&sh.y_empty[slot], ((n / YB) - 1) & 1, abort_flag);
         if (!ok) break;
         mbar_arrive_expect_tx(&sh.y_full[slot], X_TILE_BYTES);
         tma_load_3d(sY + slot * X_TILE_BYTES, map, &sh.y_full[slot], 0, x.tile * XT, slice);
@@ -125,8 +134,8 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
           ok = mbar_wait(&sh.z_ready, zc & 1, abort_flag); ++zc; prev_bh = x.bh;
           if (!ok) break;
         }
-        const int slot = n & 1;
-        ok = mbar_wait(&sh.y_full[slot], (n >> 1) & 1, abort_flag);
+        const int slot = n % YB;
+        ok = mbar_wait(&sh.y_full[slot], (n / YB) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
         const uint32_t ybase = smem_u32(sY + slot * X_TILE_BYTES);
@@ -144,9 +153,9 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         tc_fence_after();
         for (int k = 0; k < nk / 16; ++k) {               // D = (Phi + Plo) (Zhi + Zlo) without lo*lo, K = keys
           const uint64_t bh_ = smem_desc_sw128(zhi + k * 2048, zhalf, 1024);
-          umma_ts(tmem + 256, tmem + 128 + k * 8, bh_, idesc2, k > 0 ? 1u : 0u);
-          umma_ts(tmem + 256, tmem + 128 + k * 8, smem_desc_sw128(zlo + k * 2048, zhalf, 1024), idesc2, 1u);
-          umma_ts(tmem + 256, tmem + 192 + k * 8, bh_, idesc2, 1u);
+          umma_ts(tmem + 128, tmem + k * 8, bh_, idesc2, k > 0 ? 1u : 0u);
+          umma_ts(tmem + 128, tmem + k * 8, smem_desc_sw128(zlo + k * 2048, zhalf, 1024), idesc2, 1u);
+          umma_ts(tmem + 128, tmem + 48 + k * 8, bh_, idesc2, 1u);
         }
         umma_commit(&sh.d_full);
       }
@@ -180,7 +189,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         fence_proxy_async();
         mbar_arrive(&sh.z_ready);
       }
-      const int slot = n & 1;
+      const int slot = n % YB;
       const long long n_band = x.band == 1 ? dm.Nmid : dm.Nhigh;
       const long long p = (long long)x.tile * XT + row;
       // ---- softmax over the 2m summaries of the other bands
@@ -188,49 +197,46 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       if (!ok) break;
       tc_fence_after();
       const int own0 = x.band * m, own1 = own0 + m;       // this band's own summaries are not attended
-      float mx = -INFINITY;
-      uint32_t r[32];
-      for (int c0 = 0; c0 < nk; c0 += 32) {               // nk is 48 or 96: the last chunk may read stale columns
-        tmem_ld32(tmem + lane_addr + c0, r);
-        tmem_wait_ld();
+      // all scores of the row into registers (they are overwritten by P below)
+      uint32_t sc[96];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int j = c0 + i;
-          if (j < 3 * m && (j < own0 || j >= own1)) mx = fmaxf(mx, __uint_as_float(r[i]));
+      for (int c3 = 0; c3 < 3; ++c3) {
+        if (c3 * 32 < nk) {
+          uint32_t r[32];
+          tmem_ld32(tmem + lane_addr + c3 * 32, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) sc[c3 * 32 + i] = r[i];
         }
       }
-      float den = 0.f;
-      for (int c0 = 0; c0 < nk; c0 += 32) {
-        tmem_ld32(tmem + lane_addr + c0, r);
-        tmem_wait_ld();
+      float mx = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int j = c0 + i;
-          if (j < 3 * m && (j < own0 || j >= own1)) den += exp2f((__uint_as_float(r[i]) - mx) * sl2);
-        }
+      for (int j = 0; j < 96; ++j)
+        if (j < 3 * m && (j < own0 || j >= own1)) mx = fmaxf(mx, __uint_as_float(sc[j]));
+      const float mb = mx * sl2;
+      float den = 0.f;
+#pragma unroll
+      for (int j = 0; j < 96; ++j) {
+        float pv = 0.f;
+        if (j < 3 * m && (j < own0 || j >= own1)) pv = ex2f_approx(fmaf(__uint_as_float(sc[j]), sl2, -mb));
+        den += pv;
+        sc[j] = __float_as_uint(pv);
       }
       const float inv = 1.f / den;
-      for (int c0 = 0; c0 < nk; c0 += 32) {
-        tmem_ld32(tmem + lane_addr + c0, r);
-        tmem_wait_ld();
-        uint32_t ph[16], pl[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float pv[2];
+      for (int c3 = 0; c3 < 3; ++c3) {
+        if (c3 * 32 < nk) {
+          uint32_t ph[16], pl[16];
 #pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int j = c0 + 2 * i + e;
-            pv[e] = (j < 3 * m && (j < own0 || j >= own1)) ? exp2f((__uint_as_float(r[2 * i + e]) - mx) * sl2) * inv : 0.f;
+          for (int i = 0; i < 16; ++i) {
+            const float p0 = __uint_as_float(sc[c3 * 32 + 2 * i]) * inv, p1 = __uint_as_float(sc[c3 * 32 + 2 * i + 1]) * inv;
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+            ph[i] = *(const uint32_t*)&h2;
+            const __nv_bfloat162 l2 = __floats2bfloat162_rn(p0 - __uint_as_float(ph[i] << 16), p1 - __uint_as_float(ph[i] & 0xffff0000u));
+            pl[i] = *(const uint32_t*)&l2;
           }
-          const __nv_bfloat162 h2 = __floats2bfloat162_rn(pv[0], pv[1]);
-          ph[i] = *(const uint32_t*)&h2;
-          const __nv_bfloat162 l2 = __floats2bfloat162_rn(pv[0] - __uint_as_float(ph[i] << 16),
-                                                          pv[1] - __uint_as_float(ph[i] & 0xffff0000u));
-          pl[i] = *(const uint32_t*)&l2;
-        }
-        if (c0 + 32 <= nk || true) {
-          tmem_st16(tmem + lane_addr + 128 + (c0 >> 1), ph);
-          tmem_st16(tmem + lane_addr + 192 + (c0 >> 1), pl);
+          tmem_st16(tmem + lane_addr + c3 * 16, ph);
+          tmem_st16(tmem + lane_addr + 48 + c3 * 16, pl);
         }
       }
       tmem_wait_st();
@@ -246,7 +252,8 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       const uint8_t* yrow = sY + slot * X_TILE_BYTES + row * 128;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        tmem_ld32(tmem + lane_addr + 256 + q * 32, r);
+        uint32_t r[32];
+        tmem_ld32(tmem + lane_addr + 128 + q * 32, r);
         tmem_wait_ld();
         if (valid) {
 #pragma unroll
@@ -286,7 +293,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
   }
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem, 512);
+    tmem_dealloc(tmem, 256);
   }
 }
 
@@ -351,11 +358,13 @@ cudaError_t ffk_exchange_tc(ff_plan* p, int h0, int g, void* grid_hi, void* grid
   P.pos_mid = p->pos_table; P.pos_high = p->pos_table + dm.Nmid;
   P.grid_hi = (__nv_bfloat16*)grid_hi; P.grid_lo = (__nv_bfloat16*)grid_lo;
   P.h0 = h0; P.g = g; P.nkeys = (3 * dm.m + 15) / 16 * 16; P.status = p->buf.status;
-  const size_t smem = 2 * X_TILE_BYTES + 4 * MAX_KEYS * 128 + sizeof(XShared) + 1024;
+  // two CTAs per SM: double-buffer the token tile only if both still fit in shared memory
+  P.ybufs = (2 * X_TILE_BYTES + 4 * P.nkeys * 128 + sizeof(XShared) + 2048) * 2 <= 227 * 1024 ? 2 : 1;
+  const size_t smem = P.ybufs * X_TILE_BYTES + 4 * P.nkeys * 128 + sizeof(XShared) + 1024;
   cudaError_t e = cudaFuncSetAttribute(exchange_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const long long tiles = (long long)g * ((dm.Nmid + XT - 1) / XT + (dm.Nhigh + XT - 1) / XT);
-  const int grid = tiles < p->sm_count ? (int)tiles : p->sm_count;
+  const int grid = tiles < 2 * p->sm_count ? (int)tiles : 2 * p->sm_count;
   exchange_tc_kernel<<<grid, X_THREADS, smem, st>>>(*(const CUtensorMap*)p->tmap_x[0], *(const CUtensorMap*)p->tmap_x[1],
                                                    *(const CUtensorMap*)p->tmap_x[2], *(const CUtensorMap*)p->tmap_x[3], P);
   p->launches += 1;
