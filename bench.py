@@ -249,7 +249,8 @@ def run_cuda(args, cfg):
     clocks = sampler.stop()
     ms_step = reduce_max(ev[0].elapsed_time(ev[-1]) / args.steps)
     launches = plan.last_launches()
-    assert plan.device_status() == 0
+    if plan.device_status() != 0:
+        raise RuntimeError(B.library().ff_last_error(plan.handle).decode())
     alloc = plan.tap(B.TAP_ALLOC).cpu().numpy().tolist()
     pi = plan.tap(B.TAP_PI).cpu().numpy().tolist()
 

@@ -212,6 +212,7 @@ extern "C" ff_status_t ff_plan_create(const ff_config_t* c, const ff_weights_t* 
   }
   if (s == FF_OK) {
     std::vector<float> U(3 * d * d, 0.f);
+    p->identity_u = !(w && w->U);
     if (w && w->U) memcpy(U.data(), w->U, U.size() * sizeof(float));
     else for (size_t l = 0; l < 3; ++l) for (size_t i = 0; i < d; ++i) U[(l * d + i) * d + i] = 1.f;
     s = upload(p, &p->U, U.data(), U.size());
@@ -294,7 +295,7 @@ extern "C" ff_status_t ff_plan_device_status(ff_plan_t* p, void* stream) {
   FF_CUDA(p, cudaStreamSynchronize(st));
   if (word != 0) {
     FF_CUDA(p, cudaMemsetAsync(p->buf.status, 0, sizeof(int), st));
-    return fail(p, (ff_status_t)word, "device status word reports an error%s (code %lld)", "", word);
+    return fail(p, (ff_status_t)(word & 0xff), "device status word reports an error%s (status %lld, kernel %lld)", "", word & 0xff, word >> 8);
   }
   return FF_OK;
 }

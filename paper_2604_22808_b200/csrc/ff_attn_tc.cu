@@ -308,60 +308,63 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full[sb], (g >> 1) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
-        // pass 1: row maximum of the raw scores
-        float tmax = -INFINITY;
-        uint32_t r[32];
+        // the row's 128 raw scores into registers (P will overwrite them in tensor memory)
+        uint32_t sc[128];
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
           tmem_ld32(s_addr + c * 32, r);
           tmem_wait_ld();
-          if (full) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, __uint_as_float(r[i]));
-          } else {
+          for (int i = 0; i < 32; ++i) sc[c * 32 + i] = r[i];
+        }
+        float tmax = -INFINITY;
+        if (full) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const int col = c * 32 + i;
-              if (col >= clo && col <= chi) tmax = fmaxf(tmax, __uint_as_float(r[i]));
-            }
-          }
+          for (int i = 0; i < 128; ++i) tmax = fmaxf(tmax, __uint_as_float(sc[i]));
+        } else {
+#pragma unroll
+          for (int i = 0; i < 128; ++i)
+            if (i >= clo && i <= chi) tmax = fmaxf(tmax, __uint_as_float(sc[i]));
         }
         const float m_new = fmaxf(m_ref, tmax);
         const bool need = (m_new - m_ref) * sl2 > LAZY_LOG2;
         const float alpha = need ? ex2((m_ref - m_new) * sl2) : 1.f;
-        if (j > 0) {
-          // PV of the previous key tile must have landed before O may be touched
+        // Completion j-1 of this buffer's barrier (the PV of the previous key tile) is normally
+        // awaited at the end of this tile, just before P is published, when it has long happened; only a row maximum that grew
+        // past the lazy threshold needs it now, because O is then rescaled in place.  Every phase of
+        // the barrier is awaited exactly once, in order (parity waits must not skip phases).
+        bool waited_prev = false;
+        if (j > 0 && __any_sync(0xffffffffu, need)) {
           ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[ob], ocount[ob] & 1, abort_flag));
           ++ocount[ob];
+          waited_prev = true;
           if (!ok) break;
           tc_fence_after();
-          if (__any_sync(0xffffffffu, need)) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              tmem_ld32(o_addr + c * 32, r);
-              tmem_wait_ld();
+          for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tmem_ld32(o_addr + c * 32, r);
+            tmem_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-              tmem_st32(o_addr + c * 32, r);
-            }
-            tmem_wait_st();
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+            tmem_st32(o_addr + c * 32, r);
           }
+          tmem_wait_st();
         }
         if (need) { l *= alpha; m_ref = m_new; }
-        // pass 2: P = 2^(s*scale*log2e - m) as bf16 over the scores, row sum
+        // P = 2^(s*scale*log2e - m) as bf16 over the scores, row sum
         const float mb = m_ref * sl2;
         float sum = 0.f;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          tmem_ld32(s_addr + c * 32, r);
-          tmem_wait_ld();
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            float p0 = ex2(fmaf(__uint_as_float(r[2 * i]), sl2, -mb));
-            float p1 = ex2(fmaf(__uint_as_float(r[2 * i + 1]), sl2, -mb));
+            const int col = c * 32 + 2 * i;
+            float p0 = ex2(fmaf(__uint_as_float(sc[col]), sl2, -mb));
+            float p1 = ex2(fmaf(__uint_as_float(sc[col + 1]), sl2, -mb));
             if (!full) {
-              const int col = c * 32 + 2 * i;
               if (col < clo || col > chi) p0 = 0.f;
               if (col + 1 < clo || col + 1 > chi) p1 = 0.f;
             }
@@ -373,11 +376,18 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         }
         l += sum;
         tmem_wait_st();
+        // (this wait has to precede the arrival below: PV j may not be issued, let alone complete,
+        // before this thread has consumed the phase of PV j-1)
+        if (j > 0 && !waited_prev) {
+          ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[ob], ocount[ob] & 1, abort_flag));
+          ++ocount[ob];
+          if (!ok) break;
+        }
         tc_fence_before();
         mbar_arrive(&sh.p_full[sb]);
       }
       if (!ok) break;
-      // epilogue: O / l -> Y
+      // epilogue: O / l -> Y, once the item's last PV has landed
       ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[ob], ocount[ob] & 1, abort_flag));
       ++ocount[ob];
       if (!ok) break;
@@ -413,7 +423,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
   tc_fence_before();
   __syncthreads();
   if (sh.abort_flag) {
-    if (threadIdx.x == 0) atomicExch(P.status, FF_ERR_TIMEOUT);
+    if (threadIdx.x == 0) atomicExch(P.status, FF_ERR_TIMEOUT | 0x100);   // low byte: status, next byte: which kernel
     // let copies that were already issued land before the shared memory is released
     const long long t0 = clock64();
     while (clock64() - t0 < 2000000) { }

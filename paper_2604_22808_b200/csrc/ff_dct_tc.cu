@@ -350,7 +350,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
   tc_fence_before();
   __syncthreads();
   if (sh.abort_flag) {
-    if (threadIdx.x == 0) atomicExch(P.status, FF_ERR_TIMEOUT);
+    if (threadIdx.x == 0) atomicExch(P.status, FF_ERR_TIMEOUT | 0x200);   // low byte: status, next byte: which kernel
     const long long t0 = clock64();
     while (clock64() - t0 < 2000000) { }
     __syncthreads();

@@ -286,7 +286,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
   tc_fence_before();
   __syncthreads();
   if (sh.abort_flag) {
-    if (threadIdx.x == 0) atomicExch(P.status, FF_ERR_TIMEOUT);
+    if (threadIdx.x == 0) atomicExch(P.status, FF_ERR_TIMEOUT | 0x300);   // low byte: status, next byte: which kernel
     const long long t0 = clock64();
     while (clock64() - t0 < 2000000) { }
     __syncthreads();

@@ -86,6 +86,7 @@ struct ff_plan {
   float* basis_t[3];  // transposes
   float* W1; float* b1; float* W2; float* b2; float* U;
   bool has_router;
+  int identity_u;     // no summary projections were given: U_l = I
   // workspace
   void* ws; size_t ws_bytes;
   FFBuffers buf;

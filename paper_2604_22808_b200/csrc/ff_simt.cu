@@ -384,7 +384,26 @@ __global__ void __launch_bounds__(SUM_THREADS) summary_partial_kernel(FFBuffers 
   const int vec = threadIdx.x % vecs, rsub = threadIdx.x / vecs, nrs = SUM_THREADS / vecs;
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   if (rsub < nrs) {
-    for (long long p = r0 + rsub; p < r1; p += nrs) {
+    long long p = r0 + rsub;
+    if (!v.f32 && sizeof(ST) == 2) {
+      // bf16 rows, four rows in flight per thread
+      const __nv_bfloat16* base = (const __nv_bfloat16*)v.st + vec * 8;
+      for (; p + 3 * nrs < r1; p += 4 * nrs) {
+        uint4 x[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) x[u] = *(const uint4*)(base + (size_t)(p + u * nrs) * d);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const uint32_t w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            acc[2 * i] += __uint_as_float(w[i] << 16);
+            acc[2 * i + 1] += __uint_as_float(w[i] & 0xffff0000u);
+          }
+        }
+      }
+    }
+    for (; p < r1; p += nrs) {
       if (v.f32) {
         const float4 x0 = *(const float4*)(v.f32 + (size_t)p * d + vec * 8);
         const float4 x1 = *(const float4*)(v.f32 + (size_t)p * d + vec * 8 + 4);
@@ -419,7 +438,7 @@ __global__ void __launch_bounds__(SUM_THREADS) summary_partial_kernel(FFBuffers 
 }
 
 template <typename ST>
-__global__ void summary_finalize_kernel(FFBuffers buf, const float* U, FFDims dm) {
+__global__ void summary_finalize_kernel(FFBuffers buf, const float* U, FFDims dm, int identity_u) {
   __shared__ float pooled[128];
   const int j = blockIdx.x, band = blockIdx.y, bh = blockIdx.z;
   const int d = dm.d, c = threadIdx.x;
@@ -429,6 +448,7 @@ __global__ void summary_finalize_kernel(FFBuffers buf, const float* U, FFDims dm
   if (e < a + 1) e = a + 1;
   float* S = buf.summary + (((size_t)bh * 3 + band) * dm.m + j) * d;
   pooled[c] = S[c] / (float)(e - a);
+  if (identity_u) { S[c] = pooled[c]; return; }
   __syncthreads();
   const float* Ul = U + ((size_t)band * d + c) * d;
   float s = 0.f;
@@ -612,10 +632,10 @@ cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st) {
   dim3 pgrid((unsigned)(dm.m * split), 3, (unsigned)dm.BH), fgrid((unsigned)dm.m, 3, (unsigned)dm.BH);
   if (dm.fp32) {
     summary_partial_kernel<float><<<pgrid, SUM_THREADS, 0, st>>>(p->buf, dm, split);
-    summary_finalize_kernel<float><<<fgrid, dm.d, 0, st>>>(p->buf, p->U, dm);
+    summary_finalize_kernel<float><<<fgrid, dm.d, 0, st>>>(p->buf, p->U, dm, p->identity_u);
   } else {
     summary_partial_kernel<__nv_bfloat16><<<pgrid, SUM_THREADS, 0, st>>>(p->buf, dm, split);
-    summary_finalize_kernel<__nv_bfloat16><<<fgrid, dm.d, 0, st>>>(p->buf, p->U, dm);
+    summary_finalize_kernel<__nv_bfloat16><<<fgrid, dm.d, 0, st>>>(p->buf, p->U, dm, p->identity_u);
   }
   p->launches += 2;
   return cudaGetLastError();
