@@ -8,7 +8,7 @@
 //   warp 0      TMA producer: Q tile (double buffered), K and V tiles (two stages each)
 //   warp 1      tcgen05.mma issuer: S = Q K^T (A, B from shared memory), O += P V (A = P from
 //               tensor memory, B = V as an MN-major operand); owns the tensor-memory allocation
-//   warps 2..5  softmax: one query row per thread (row = TMEM lane), scores read with tcgen05.ld,
+//   warps 2..9  softmax: two threads per query row (row = TMEM lane, 64 key columns each), scores read with tcgen05.ld,
 //               key masks generated in registers from the row's band rank, P written back to
 //               tensor memory as bf16 over the scores it came from; O is accumulated in tensor
 //               memory and rescaled only when a row's running maximum grows by more than 2^8
@@ -29,7 +29,7 @@ constexpr int HD = 128;              // head_dim
 constexpr int TILE_BYTES = TILE * HD * 2;
 constexpr int HALF_BYTES = TILE_BYTES / 2;
 constexpr int MAX_UNITS = 1024;
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 320;         // TMA warp, MMA warp, 8 softmax warps
 constexpr float LAZY_LOG2 = 8.0f;    // rescale O only when the running max grows by more than this (log2 units)
 
 struct TcParams {
@@ -86,6 +86,9 @@ struct Shared {
   int n_units, total;
   int offsets[MAX_UNITS + 1];
   int desc[MAX_UNITS];
+  // hand-shake slots of the two threads of a row: (sequence number << 32) | float bits
+  unsigned long long xmax[2][2][128];
+  unsigned long long xsum[2][2][128];
 };
 
 __device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, int it) {
@@ -136,6 +139,20 @@ __device__ __forceinline__ void load_tile(uint8_t* dst, const CUtensorMap* map, 
   }
 }
 
+// The two softmax threads of a row swap one float: each publishes (seq, value) in its slot and
+// waits, bounded, until the partner's slot carries the same sequence number.
+__device__ __forceinline__ bool pair_exchange(unsigned long long* mine, unsigned long long* theirs, unsigned seq, float v,
+                                              float& other, volatile int* abort_flag) {
+  *(volatile unsigned long long*)mine = ((unsigned long long)seq << 32) | __float_as_uint(v);
+  const long long t0 = clock64();
+  while (true) {
+    const unsigned long long w = *(volatile unsigned long long*)theirs;
+    if ((unsigned)(w >> 32) == seq) { other = __uint_as_float((unsigned)w); return true; }
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return false; }
+  }
+}
+
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -163,8 +180,8 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
       mbar_init(&sh.q_full[i], 1); mbar_init(&sh.q_empty[i], 1);
       mbar_init(&sh.k_full[i], 1); mbar_init(&sh.k_empty[i], 1);
       mbar_init(&sh.v_full[i], 1); mbar_init(&sh.v_empty[i], 1);
-      mbar_init(&sh.s_full[i], 1); mbar_init(&sh.p_full[i], 128);
-      mbar_init(&sh.o_full[i], 1); mbar_init(&sh.o_empty[i], 128);
+      mbar_init(&sh.s_full[i], 1); mbar_init(&sh.p_full[i], 256);
+      mbar_init(&sh.o_full[i], 1); mbar_init(&sh.o_empty[i], 256);
     }
     sh.abort_flag = 0;
     sh.n_units = P.work[0];
@@ -172,6 +189,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
     fence_mbar_init();
   }
   __syncthreads();
+  for (int i = threadIdx.x; i < 2 * 2 * 128; i += TC_THREADS) { (&sh.xmax[0][0][0])[i] = 0ull; (&sh.xsum[0][0][0])[i] = 0ull; }
   for (int i = threadIdx.x; i <= sh.n_units; i += TC_THREADS) {
     sh.offsets[i] = P.work[2 + i];
     if (i < sh.n_units) sh.desc[i] = P.work[2 + MAX_UNITS + 1 + i];
@@ -263,9 +281,15 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
       if (ok && have_prev) issue_pv();
     }
   } else {
-    // ------------------------------------------------------------------ softmax, one row per thread
+    // ------------------------------------------------------------------ softmax, two threads per row
+    // Warps 2..5 take key columns 0..63 of their 32 rows, warps 6..9 columns 64..127 of the same
+    // rows (a warp reaches the TMEM lanes 32*(warp%4)..+31), so every scheduler has two softmax warps
+    // to interleave.  The two threads of a row agree on the row maximum through shared memory and a
+    // bounded hand-shake; each keeps the partial row sum of its own columns.
     const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;
     const int row = quarter * 32 + lane;
+    const int col0 = half * 64;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const float sl2 = rsqrtf((float)HD) * 1.4426950408889634f;
     int iter = 0; unsigned g = 0;
@@ -274,7 +298,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
     for (int it = blockIdx.x; it < total && ok; it += gridDim.x, ++iter) {
       const Item x = decode_item(sh, dm, it);
       const int ob = iter & 1;
-      const uint32_t o_addr = tm + lane_addr + 256 + ob * 128;
+      const uint32_t o_addr = tm + lane_addr + 256 + ob * 128 + col0;      // this thread's 64 output columns
       // band rank of this thread's query row
       const long long u_q = (long long)x.tile * TILE + row;
       const long long p = x.band == 1 ? mid_rank(dm, x.c, u_q) : u_q;
@@ -308,12 +332,12 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full[sb], (g >> 1) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
-        // the row's 128 raw scores into registers (P will overwrite them in tensor memory)
-        uint32_t sc[128];
+        // this thread's 64 raw scores into registers (P will overwrite them in tensor memory)
+        uint32_t sc[64];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 2; ++c) {
           uint32_t r[32];
-          tmem_ld32(s_addr + c * 32, r);
+          tmem_ld32(s_addr + col0 + c * 32, r);
           tmem_wait_ld();
 #pragma unroll
           for (int i = 0; i < 32; ++i) sc[c * 32 + i] = r[i];
@@ -321,19 +345,29 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         float tmax = -INFINITY;
         if (full) {
 #pragma unroll
-          for (int i = 0; i < 128; ++i) tmax = fmaxf(tmax, __uint_as_float(sc[i]));
+          for (int i = 0; i < 64; ++i) tmax = fmaxf(tmax, __uint_as_float(sc[i]));
         } else {
 #pragma unroll
-          for (int i = 0; i < 128; ++i)
-            if (i >= clo && i <= chi) tmax = fmaxf(tmax, __uint_as_float(sc[i]));
+          for (int i = 0; i < 64; ++i)
+            if (col0 + i >= clo && col0 + i <= chi) tmax = fmaxf(tmax, __uint_as_float(sc[i]));
+        }
+        // row maximum over both halves (slots alternate with the tile parity, so the partner's
+        // read of this tile cannot meet this thread's write of the next)
+        {
+          float other;
+          ok = __all_sync(0xffffffffu, pair_exchange(&sh.xmax[g & 1][half][row], &sh.xmax[g & 1][half ^ 1][row], g + 1, tmax,
+                                                     other, abort_flag));
+          if (!ok) break;
+          tmax = fmaxf(tmax, other);
         }
         const float m_new = fmaxf(m_ref, tmax);
         const bool need = (m_new - m_ref) * sl2 > LAZY_LOG2;
         const float alpha = need ? ex2((m_ref - m_new) * sl2) : 1.f;
         // Completion j-1 of this buffer's barrier (the PV of the previous key tile) is normally
-        // awaited at the end of this tile, just before P is published, when it has long happened; only a row maximum that grew
-        // past the lazy threshold needs it now, because O is then rescaled in place.  Every phase of
-        // the barrier is awaited exactly once, in order (parity waits must not skip phases).
+        // awaited at the end of this tile, just before P is published, when it has long happened;
+        // only a row maximum that grew past the lazy threshold needs it now, because O is then
+        // rescaled in place.  Every phase of the barrier is awaited exactly once, in order (parity
+        // waits must not skip phases).  Both threads of a row see the same `need`.
         bool waited_prev = false;
         if (j > 0 && __any_sync(0xffffffffu, need)) {
           ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[ob], ocount[ob] & 1, abort_flag));
@@ -342,7 +376,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < 2; ++c) {
             uint32_t r[32];
             tmem_ld32(o_addr + c * 32, r);
             tmem_wait_ld();
@@ -353,17 +387,17 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
           tmem_wait_st();
         }
         if (need) { l *= alpha; m_ref = m_new; }
-        // P = 2^(s*scale*log2e - m) as bf16 over the scores, row sum
+        // P = 2^(s*scale*log2e - m) as bf16 over the scores, partial row sum
         const float mb = m_ref * sl2;
         float sum = 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 2; ++c) {
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const int col = c * 32 + 2 * i;
-            float p0 = ex2(fmaf(__uint_as_float(sc[col]), sl2, -mb));
-            float p1 = ex2(fmaf(__uint_as_float(sc[col + 1]), sl2, -mb));
+            const int k = c * 32 + 2 * i, col = col0 + k;
+            float p0 = ex2(fmaf(__uint_as_float(sc[k]), sl2, -mb));
+            float p1 = ex2(fmaf(__uint_as_float(sc[k + 1]), sl2, -mb));
             if (!full) {
               if (col < clo || col > chi) p0 = 0.f;
               if (col + 1 < clo || col + 1 > chi) p1 = 0.f;
@@ -372,7 +406,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
             const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
             pk[i] = *(const uint32_t*)&v;
           }
-          tmem_st16(s_addr + c * 16, pk);
+          tmem_st16(s_addr + (col0 >> 1) + c * 16, pk);
         }
         l += sum;
         tmem_wait_st();
@@ -387,17 +421,24 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         mbar_arrive(&sh.p_full[sb]);
       }
       if (!ok) break;
-      // epilogue: O / l -> Y, once the item's last PV has landed
+      // epilogue: O / l -> Y, once the item's last PV has landed; l = the two partial row sums
+      {
+        float other;
+        ok = __all_sync(0xffffffffu, pair_exchange(&sh.xsum[iter & 1][half][row], &sh.xsum[iter & 1][half ^ 1][row],
+                                                   (unsigned)iter + 1, l, other, abort_flag));
+        if (!ok) break;
+        l += other;
+      }
       ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[ob], ocount[ob] & 1, abort_flag));
       ++ocount[ob];
       if (!ok) break;
       tc_fence_after();
       const float inv = 1.f / l;
-      const bool store = p < x.n && (x.band != 1 || u_q < (long long)x.nk * TILE);
-      __nv_bfloat16* y = (x.band == 1 ? P.y_mid : P.y_high) + ((size_t)x.bh * x.n + (store ? p : 0)) * HD;
-      uint32_t r[32];
+      const bool store = p < x.n;
+      __nv_bfloat16* y = (x.band == 1 ? P.y_mid : P.y_high) + ((size_t)x.bh * x.n + (store ? p : 0)) * HD + col0;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
         tmem_ld32(o_addr + c * 32, r);
         tmem_wait_ld();
         if (store) {
