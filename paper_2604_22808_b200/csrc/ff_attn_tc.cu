@@ -117,8 +117,11 @@ __device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, 
 }
 
 // Band rank of class-local position u of residue class c (mid band).
+// (32-bit arithmetic: positions and ranks stay below 2^32 for every supported size.)
 __device__ __forceinline__ long long mid_rank(const FFDims& dm, int c, long long u) {
-  return ((long long)c + (u / dm.b) * dm.s) * dm.b + (u % dm.b);
+  const unsigned uu = (unsigned)u, b = (unsigned)dm.b;
+  const unsigned blk = uu / b;
+  return (long long)(((unsigned)c + blk * (unsigned)dm.s) * b + (uu - blk * b));
 }
 
 // Issues the TMA loads of one 128-row tile (two 64-column halves) into `dst`.
