@@ -28,6 +28,11 @@ from paper_2604_22808_b200 import inputs as I           # noqa: E402
 
 METRIC = "freqformer_attn_layer_tokens_per_s"
 
+# dram__bytes_read.sum + dram__bytes_write.sum of the transform kernels per token and head, from the ncu
+# capture summarised in profiles/dct_tc_kernel_64k_6heads.md (forward: three passes over Q, K and V;
+# inverse: three passes over one tensor).
+NCU_DRAM_BYTES_PER_TOKEN_HEAD = {"transform": 7490.0, "inverse": 2960.0}
+
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -271,19 +276,27 @@ def run_cuda(args, cfg):
         peaks = measured_peaks()
         tokens = cfg.batch * cfg.N * world
         work = layer_work(cfg, alloc)
-        # roofline of the dominant stage
+        # roofline of the dominant stage (achieved and traffic are per launch of the stage's kernel)
         top = max(stage_ms, key=stage_ms.get)
+        n_launch = max(1, stage_launches.get(top) or 1)
+        heads_total = cfg.batch * cfg.heads
         if top == "attention":
             achieved = work["attn_flops"] / (stage_ms[top] * 1e-3) / 1e12
             roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                    "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None}
+                    "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
+                    "kernel": "attention_tc_kernel"}
         else:
             nbytes = work["bytes_transform"] if top == "transform" else work["bytes_inverse"]
             achieved = nbytes / (stage_ms[top] * 1e-3) / 1e9
+            # DRAM bytes per token-head and stage from the ncu capture of the 6-head 64K case
+            # (profiles/dct_tc_kernel_64k_6heads.md); traffic is proportional to tokens x heads.
+            per_token_head = NCU_DRAM_BYTES_PER_TOKEN_HEAD[top]
             roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": None}
-        roof.update({"kernel": top, "launches_per_step": stage_launches.get(top), "ms_per_step": stage_ms[top],
-                     "peak_source": peaks["source"]})
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": per_token_head * cfg.N * heads_total / n_launch,
+                    "kernel": "dct_tc_kernel (%s stage)" % top,
+                    "algorithmic_bytes_per_launch": nbytes / n_launch}
+        roof.update({"stage": top, "launches_per_step": stage_launches.get(top), "ms_per_step": stage_ms[top],
+                     "ms_per_launch": stage_ms[top] / n_launch, "peak_source": peaks["source"]})
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
             v_cpu, spent, cores, text = oracle_sample_time(cfg, alloc)

@@ -275,7 +275,7 @@ extern "C" const char* ff_last_error(const ff_plan_t* p) { return p ? p->err : g
 
 extern "C" ff_status_t ff_plan_set_attention_impl(ff_plan_t* p, int32_t impl) {
   if (!p) return fail(nullptr, FF_ERR_INVALID_ARG, "plan is NULL%s");
-  if (impl < 0 || impl > 3) return fail(p, FF_ERR_INVALID_ARG, "impl must be in [0, 3]%s");
+  if (impl < 0 || impl > 7) return fail(p, FF_ERR_INVALID_ARG, "impl must be in [0, 7]%s");
   p->attn_impl = impl;
   return FF_OK;
 }

@@ -42,7 +42,7 @@ constexpr int TILE_BYTES = TILE_ROWS * CH * 2;     // 32 KB: 128 rows of bf16
 constexpr int HALF_BYTES = TILE_BYTES / 2;
 constexpr int MAX_STAGE = 4;
 constexpr int NACC = 4;
-constexpr int DCT_TC_THREADS = 192;
+constexpr int DCT_TC_THREADS = 320;        // TMA warp, MMA warp, 8 epilogue warps
 
 enum { MODE_FIRST = 0, MODE_MIDDLE = 1, MODE_SPLIT = 2, MODE_LAST = 3 };
 
@@ -64,7 +64,7 @@ struct DctTcParams {
   int* status;
 };
 
-constexpr int STG_PITCH = 80;                       // bytes per staged row piece (64 B of data, padded against bank conflicts)
+constexpr int STG_PITCH = 64;                       // bytes per staged row piece; the 16-byte chunks are rotated by row/2 against bank conflicts
 
 struct DctShared {
   uint64_t full[MAX_STAGE], empty[MAX_STAGE], acc_full[NACC], acc_empty[NACC], img_full;
@@ -72,7 +72,7 @@ struct DctShared {
   int abort_flag;
   // per epilogue warp: 32 rows x 64 bytes of hi and of lo, to turn one-row-per-thread registers
   // into stores where four lanes cover a row's 64 contiguous bytes
-  alignas(16) uint8_t stage[4][2][32 * STG_PITCH];
+  alignas(16) uint8_t stage[8][2][32 * STG_PITCH];
 };
 
 // Grid coordinates (w, h, t) of the first position of tile `u` of a tensor-head.  A tile holds
@@ -121,7 +121,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NSTAGE; ++i) { mbar_init(&sh.full[i], 1); mbar_init(&sh.empty[i], 1); }
-    for (int i = 0; i < NACC; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 128); }
+    for (int i = 0; i < NACC; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 256); }
     mbar_init(&sh.img_full, 1);
     sh.abort_flag = 0;
     fence_mbar_init();
@@ -199,6 +199,8 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     const int a = seq ? j & (n - 1) : j >> lkf;           // output index along the axis
     const int l = seq ? j >> ln : j & (kf - 1);           // line of the tile
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const int ew = warp - 2;                              // epilogue warp 0..7: warps 0-3 take channels 0..63, 4-7 channels 64..127
+    const int q_lo = (ew >> 2) * 2;
     const long long N_d = dm.N * CH;
     const long long axis_stride = (P.axis == 2 ? 1LL : (P.axis == 1 ? (long long)dm.W : (long long)dm.W * dm.H)) * CH;
     const long long line_stride = (P.axis == 2 ? (long long)dm.W : 1LL) * CH;   // between the lines of a tile
@@ -212,7 +214,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     auto flush_energy = [&]() {
       if (e_sample >= 0 && P.energy) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = q_lo; q < q_lo + 2; ++q) {
           atomicAdd(P.energy + ((size_t)e_sample * 3 + 1) * CH + q * 32 + lane, (double)em[q]);
           atomicAdd(P.energy + ((size_t)e_sample * 3 + 2) * CH + q * 32 + lane, (double)eh[q]);
           em[q] = eh[q] = 0.f;
@@ -267,7 +269,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
         dst_lo[i] = (__nv_bfloat16*)__shfl_sync(0xffffffffu, (unsigned long long)row_lo, src);
       }
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+      for (int q = q_lo; q < q_lo + 2; ++q) {
         uint32_t r[32];
         tmem_ld32(tm + lane_addr + ab * 128 + q * 32, r);
         tmem_wait_ld();
@@ -324,19 +326,19 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
             const __nv_bfloat162 lp = __floats2bfloat162_rn(v0 - __uint_as_float(hi[i] << 16), v1 - __uint_as_float(hi[i] & 0xffff0000u));
             lo[i] = *(const uint32_t*)&lp;
           }
-          uint8_t* st_hi = sh.stage[quarter][0];
-          uint8_t* st_lo = sh.stage[quarter][1];
+          uint8_t* st_hi = sh.stage[ew][0];
+          uint8_t* st_lo = sh.stage[ew][1];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            *(uint4*)(st_hi + lane * STG_PITCH + i * 16) = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
-            *(uint4*)(st_lo + lane * STG_PITCH + i * 16) = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
+            *(uint4*)(st_hi + lane * STG_PITCH + (((i + (lane >> 1)) & 3) << 4)) = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
+            *(uint4*)(st_lo + lane * STG_PITCH + (((i + (lane >> 1)) & 3) << 4)) = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
           }
           __syncwarp();
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int rr = 8 * i + (lane >> 2), piece = lane & 3;      // row of the warp, 16-byte piece of its 64 bytes
-            if (dst_hi[i]) *(uint4*)(dst_hi[i] + q * 32 + piece * 8) = *(const uint4*)(st_hi + rr * STG_PITCH + piece * 16);
-            if (dst_lo[i]) *(uint4*)(dst_lo[i] + q * 32 + piece * 8) = *(const uint4*)(st_lo + rr * STG_PITCH + piece * 16);
+            if (dst_hi[i]) *(uint4*)(dst_hi[i] + q * 32 + piece * 8) = *(const uint4*)(st_hi + rr * STG_PITCH + (((piece + (rr >> 1)) & 3) << 4));
+            if (dst_lo[i]) *(uint4*)(dst_lo[i] + q * 32 + piece * 8) = *(const uint4*)(st_lo + rr * STG_PITCH + (((piece + (rr >> 1)) & 3) << 4));
           }
           __syncwarp();
         }
@@ -460,7 +462,7 @@ cudaError_t launch_pass(ff_plan* p, const CUtensorMap& m0, const CUtensorMap& m1
   const size_t img = TILE_BYTES;
   const size_t stage = P.in_split ? 2 * TILE_BYTES : TILE_BYTES;
   const size_t fixed = 2 * img + sizeof(DctShared) + 1024;
-  int nstage = (int)((220 * 1024 - fixed) / stage);
+  int nstage = (int)((232448 - 256 - fixed) / stage);   // 227 KB of shared memory per CTA
   if (nstage > MAX_STAGE) nstage = MAX_STAGE;
   P.nstage = nstage;
   const size_t smem = nstage * stage + fixed;
@@ -517,11 +519,12 @@ bool ffk_dct_tc_build_image(ff_plan* p, int axis, int inverse, const float* mat,
 size_t ffk_dct_tc_scratch_bytes(const FFDims& dm, int group) {
   const size_t grid = (size_t)group * dm.N * CH * 2;
   const size_t side = (size_t)group * dm.T * dm.H * dm.L[2] * CH * 4;
-  return 4 * ((grid + 255) / 256 * 256) + (side + 255) / 256 * 256;
+  const size_t ring = ffk_dct_wh_supported(dm) ? ffk_dct_wh_scratch_bytes(dm, group) : 0;
+  return 4 * ((grid + 255) / 256 * 256) + (side + 255) / 256 * 256 + (ring + 255) / 256 * 256;
 }
 
 namespace {
-struct Scratch { __nv_bfloat16 *a_hi, *a_lo, *b_hi, *b_lo; float* side; };
+struct Scratch { __nv_bfloat16 *a_hi, *a_lo, *b_hi, *b_lo; float* side; void* ring; };
 Scratch carve(ff_plan* p) {
   const size_t grid_bytes = ((size_t)p->dct_group * p->dm.N * CH * 2 + 255) / 256 * 256;
   char* base = (char*)p->buf.scratchA;
@@ -529,6 +532,8 @@ Scratch carve(ff_plan* p) {
   s.a_hi = (__nv_bfloat16*)base; s.a_lo = (__nv_bfloat16*)(base + grid_bytes);
   s.b_hi = (__nv_bfloat16*)(base + 2 * grid_bytes); s.b_lo = (__nv_bfloat16*)(base + 3 * grid_bytes);
   s.side = (float*)(base + 4 * grid_bytes);
+  const size_t side_bytes = ((size_t)p->dct_group * p->dm.T * p->dm.H * p->dm.L[2] * CH * 4 + 255) / 256 * 256;
+  s.ring = base + 4 * grid_bytes + side_bytes;
   return s;
 }
 }  // namespace
@@ -546,6 +551,7 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
       !encode_grid_map(&m2l, sc.b_lo, dm, G, 0))
     return cudaErrorInvalidValue;
   const int total = 3 * dm.BH;
+  const bool fused = ffk_dct_wh_supported(dm) && !(p->attn_impl & 4);
   DctTcParams P{};
   P.dm = dm; P.status = p->buf.status;
   P.spec_mid = (__nv_bfloat16*)p->buf.spec_mid; P.spec_high = (__nv_bfloat16*)p->buf.spec_high;
@@ -553,14 +559,22 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
   for (int g0 = 0; g0 < total; g0 += G) {
     const int g = total - g0 < G ? total - g0 : G;
     P.group = g; P.group_start = g0;
-    P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 2 + 0) * TILE_BYTES;
-    P.dst = sc.a_hi; P.dst_lo = sc.a_lo; P.side = side;
-    cudaError_t e = launch_pass(p, mq, mk, mv, P, st);
-    if (e != cudaSuccess) return e;
-    P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 1 + 0) * TILE_BYTES;
-    P.dst = sc.b_hi; P.dst_lo = sc.b_lo;
-    e = launch_pass(p, m1h, m1l, m1l, P, st);
-    if (e != cudaSuccess) return e;
+    cudaError_t e;
+    if (fused) {
+      // w and h passes in one launch, the intermediate staying in L2
+      e = ffk_dct_wh_launch(p, 1, Q, K, V, g0, g, sc.ring, sc.b_hi, sc.b_lo, side, st);
+      if (e != cudaSuccess) return e;
+    } else {
+      P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 2 + 0) * TILE_BYTES;
+      P.dst = sc.a_hi; P.dst_lo = sc.a_lo; P.side = side;
+      e = launch_pass(p, mq, mk, mv, P, st);
+      if (e != cudaSuccess) return e;
+      P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 1 + 0) * TILE_BYTES;
+      P.dst = sc.b_hi; P.dst_lo = sc.b_lo;
+      e = launch_pass(p, m1h, m1l, m1l, P, st);
+      if (e != cudaSuccess) return e;
+    }
+    P.in_split = 1;
     P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 0 + 0) * TILE_BYTES; P.dst = nullptr;
     e = launch_pass(p, m2h, m2l, m2l, P, st);
     if (e != cudaSuccess) return e;
@@ -590,6 +604,8 @@ cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaS
   P.dst = sc.b_hi; P.dst_lo = sc.b_lo;
   cudaError_t e = launch_pass(p, m_in, m_inl, m_inl, P, st);
   if (e != cudaSuccess) return e;
+  if (ffk_dct_wh_supported(dm) && !(p->attn_impl & 4))
+    return ffk_dct_wh_launch(p, 0, sc.b_hi, sc.b_lo, nullptr, h0, g, sc.ring, out, nullptr, nullptr, st);
   P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 4 + 0) * TILE_BYTES;
   P.dst = sc.a_hi; P.dst_lo = sc.a_lo;
   e = launch_pass(p, mbh, mbl, mbl, P, st);

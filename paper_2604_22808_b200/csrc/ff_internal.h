@@ -138,5 +138,10 @@ size_t ffk_dct_tc_scratch_bytes(const FFDims& dm, int group);
 cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, const void* V, bool want_energy,
                                      cudaStream_t st);
 cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaStream_t st);
+// ---- fused w/h passes (ff_dct_wh.cu) ---------------------------------------------------------------
+bool ffk_dct_wh_supported(const FFDims& dm);
+size_t ffk_dct_wh_scratch_bytes(const FFDims& dm, int group);
+cudaError_t ffk_dct_wh_launch(ff_plan* p, int forward, const void* src0, const void* src1, const void* src2, int g0, int g,
+                              void* ring, void* out_hi, void* out_lo, float* side, cudaStream_t st);
 cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st);
 cudaError_t ffk_exchange_inverse(ff_plan* p, void* out, cudaStream_t st);
