@@ -198,8 +198,10 @@ enum {
 };
 ff_status_t ff_get_tap(const ff_plan_t *plan, int32_t which, const void **dev_ptr, size_t *bytes);
 
-/* Selects the attention implementation: 0 = automatic (tensor-core kernel where it applies),
- * 1 = force the generic SIMT kernel.  For tests. */
+/* Kernel selection, a bit mask (0 = the defaults): 1 = generic SIMT attention instead of the
+ * tensor-core kernel, 2 = generic SIMT transform instead of the tensor-core passes, 4 = w and h
+ * passes fused in one launch with the intermediate kept in L2 (measured slower than separate passes
+ * on B200; kept for experiments).  For tests and benchmarks. */
 ff_status_t ff_plan_set_attention_impl(ff_plan_t *plan, int32_t impl);
 
 /* ---- for callers that cannot allocate device memory ---------------------------------------------

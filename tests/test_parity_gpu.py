@@ -128,6 +128,15 @@ def test_replica_simt_attention_matches_too():
     _run(C.R64K, alloc=[2, 4, 1, 7, 4, 2], impl=1)
 
 
+def test_replica_fused_wh_passes_match_too():
+    _run(C.R64K, alloc=[2, 4, 1, 7, 4, 2], impl=4)
+    _run(C.R1M, alloc=[7, 2, 4, 1], impl=4)
+
+
+def test_replica_generic_transform_matches_too():
+    _run(C.R64K, alloc=[2, 4, 1, 7, 4, 2], impl=2)
+
+
 def test_route_entry_point():
     import torch
     from paper_2604_22808_b200 import binding as B
