@@ -194,6 +194,30 @@ def run_reference(args, cfg):
 
 
 # ---------------------------------------------------------------------------------------------
+# Multi-rank plumbing (replicas only: no data-path collective; used with NCCL on GPUs, gloo in tests)
+# ---------------------------------------------------------------------------------------------
+def replica_config(cfg, rank: int):
+    """Every rank runs its own replica of the batch: same workload, its own seeded inputs."""
+    return cfg.scaled(cfg.name, seed=cfg.seed + 1000 * rank) if rank else cfg
+
+
+def reduce_max(x: float, world: int, device) -> float:
+    """Slowest rank's value (the timing every rank reports)."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tokens_per_s(cfg, world: int, ms_step_max: float) -> float:
+    """Whole-job throughput: the tokens all ranks processed over the slowest rank's step time."""
+    return cfg.batch * cfg.N * world / (ms_step_max * 1e-3)
+
+
+# ---------------------------------------------------------------------------------------------
 # The CUDA arm
 # ---------------------------------------------------------------------------------------------
 def run_cuda(args, cfg):
@@ -210,7 +234,7 @@ def run_cuda(args, cfg):
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     dt = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
-    cfg_r = cfg.scaled(cfg.name, seed=cfg.seed + 1000 * rank) if rank else cfg       # each rank its own replica
+    cfg_r = replica_config(cfg, rank)
     host = [torch.from_numpy(I.qkv_full(cfg_r, t)).to(dt).pin_memory() for t in range(3)]
     q, k, v = (x.to(dev, non_blocking=True) for x in host)
     out = torch.empty_like(q)
@@ -228,12 +252,8 @@ def run_cuda(args, cfg):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def reduce_max(x):
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    def reduce_max_(x):
+        return reduce_max(x, world, dev)
 
     # device-resident timing
     for _ in range(args.warmup):
@@ -253,7 +273,7 @@ def run_cuda(args, cfg):
             stage_launches[name] = n
     barrier()
     clocks = sampler.stop()
-    ms_step = reduce_max(ev[0].elapsed_time(ev[-1]) / args.steps)
+    ms_step = reduce_max_(ev[0].elapsed_time(ev[-1]) / args.steps)
     launches = plan.last_launches()
     if plan.device_status() != 0:
         raise RuntimeError(B.library().ff_last_error(plan.handle).decode())
@@ -270,7 +290,7 @@ def run_cuda(args, cfg):
         t0 = time.perf_counter()
         for _ in range(e2e_steps):
             plan.forward_host(host[0], host[1], host[2], out_host, timesteps=ts)      # synchronises the stream
-        e2e_ms = reduce_max((time.perf_counter() - t0) * 1e3 / e2e_steps)
+        e2e_ms = reduce_max_((time.perf_counter() - t0) * 1e3 / e2e_steps)
         barrier()
 
     if rank == 0:
@@ -305,7 +325,7 @@ def run_cuda(args, cfg):
                    "seconds": spent}
         io_bytes = q.numel() * q.element_size()
         line = {
-            "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
+            "metric": METRIC, "value": aggregate_tokens_per_s(cfg, world, ms_step), "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
             "config": {"workload": cfg.name, "grid": list(cfg.grid), "batch": cfg.batch, "heads": cfg.heads,
