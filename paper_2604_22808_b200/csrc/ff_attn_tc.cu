@@ -29,7 +29,9 @@ constexpr int HD = 128;              // head_dim
 constexpr int TILE_BYTES = TILE * HD * 2;
 constexpr int HALF_BYTES = TILE_BYTES / 2;
 constexpr int MAX_UNITS = 1024;
-constexpr int TC_THREADS = 320;         // TMA warp, MMA warp, 8 softmax warps
+constexpr int NSPLIT = 4;                // softmax threads per query row
+constexpr int SCOLS = TILE / NSPLIT;     // key (and output) columns per softmax thread
+constexpr int TC_THREADS = 64 + 128 * NSPLIT;   // TMA warp, MMA warp, 4 * NSPLIT softmax warps
 constexpr float LAZY_LOG2 = 8.0f;    // rescale O only when the running max grows by more than this (log2 units)
 
 struct TcParams {
@@ -87,8 +89,8 @@ struct Shared {
   int offsets[MAX_UNITS + 1];
   int desc[MAX_UNITS];
   // hand-shake slots of the two threads of a row: (sequence number << 32) | float bits
-  unsigned long long xmax[2][2][128];
-  unsigned long long xsum[2][2][128];
+  unsigned long long xmax[2][NSPLIT][128];
+  unsigned long long xsum[2][NSPLIT][128];
 };
 
 __device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, int it) {
@@ -142,18 +144,31 @@ __device__ __forceinline__ void load_tile(uint8_t* dst, const CUtensorMap* map, 
   }
 }
 
-// The two softmax threads of a row swap one float: each publishes (seq, value) in its slot and
-// waits, bounded, until the partner's slot carries the same sequence number.
-__device__ __forceinline__ bool pair_exchange(unsigned long long* mine, unsigned long long* theirs, unsigned seq, float v,
-                                              float& other, volatile int* abort_flag) {
-  *(volatile unsigned long long*)mine = ((unsigned long long)seq << 32) | __float_as_uint(v);
-  const long long t0 = clock64();
-  while (true) {
-    const unsigned long long w = *(volatile unsigned long long*)theirs;
-    if ((unsigned)(w >> 32) == seq) { other = __uint_as_float((unsigned)w); return true; }
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return false; }
+// The NSPLIT softmax threads of a row share one float each: a thread publishes (seq, value) in its
+// slot and reads the others' slots, waiting (bounded) until they carry the same sequence number.
+// `slots` points at [NSPLIT][128] entries of one parity; MAX selects max, otherwise sum.
+template <bool MAX>
+__device__ __forceinline__ bool row_exchange(unsigned long long* slots, int part, int row, unsigned seq, float& v,
+                                             volatile int* abort_flag) {
+  *(volatile unsigned long long*)(slots + part * 128 + row) = ((unsigned long long)seq << 32) | __float_as_uint(v);
+  float acc = v;
+#pragma unroll
+  for (int o = 1; o < NSPLIT; ++o) {
+    const volatile unsigned long long* theirs = slots + ((part + o) % NSPLIT) * 128 + row;
+    const long long t0 = clock64();
+    while (true) {
+      const unsigned long long w = *theirs;
+      if ((unsigned)(w >> 32) == seq) {
+        const float x = __uint_as_float((unsigned)w);
+        acc = MAX ? fmaxf(acc, x) : acc + x;
+        break;
+      }
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return false; }
+    }
   }
+  v = acc;
+  return true;
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -183,8 +198,8 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
       mbar_init(&sh.q_full[i], 1); mbar_init(&sh.q_empty[i], 1);
       mbar_init(&sh.k_full[i], 1); mbar_init(&sh.k_empty[i], 1);
       mbar_init(&sh.v_full[i], 1); mbar_init(&sh.v_empty[i], 1);
-      mbar_init(&sh.s_full[i], 1); mbar_init(&sh.p_full[i], 256);
-      mbar_init(&sh.o_full[i], 1); mbar_init(&sh.o_empty[i], 256);
+      mbar_init(&sh.s_full[i], 1); mbar_init(&sh.p_full[i], 128 * NSPLIT);
+      mbar_init(&sh.o_full[i], 1); mbar_init(&sh.o_empty[i], 128 * NSPLIT);
     }
     sh.abort_flag = 0;
     sh.n_units = P.work[0];
@@ -192,7 +207,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
     fence_mbar_init();
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < 2 * 2 * 128; i += TC_THREADS) { (&sh.xmax[0][0][0])[i] = 0ull; (&sh.xsum[0][0][0])[i] = 0ull; }
+  for (int i = threadIdx.x; i < 2 * NSPLIT * 128; i += TC_THREADS) { (&sh.xmax[0][0][0])[i] = 0ull; (&sh.xsum[0][0][0])[i] = 0ull; }
   for (int i = threadIdx.x; i <= sh.n_units; i += TC_THREADS) {
     sh.offsets[i] = P.work[2 + i];
     if (i < sh.n_units) sh.desc[i] = P.work[2 + MAX_UNITS + 1 + i];
@@ -290,9 +305,9 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
     // to interleave.  The two threads of a row agree on the row maximum through shared memory and a
     // bounded hand-shake; each keeps the partial row sum of its own columns.
     const int quarter = warp & 3;
-    const int half = (warp - 2) >> 2;
+    const int part = (warp - 2) >> 2;                      // which SCOLS-wide column slice of the row
     const int row = quarter * 32 + lane;
-    const int col0 = half * 64;
+    const int col0 = part * SCOLS;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const float sl2 = rsqrtf((float)HD) * 1.4426950408889634f;
     int iter = 0; unsigned g = 0;
@@ -336,9 +351,9 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         if (!ok) break;
         tc_fence_after();
         // this thread's 64 raw scores into registers (P will overwrite them in tensor memory)
-        uint32_t sc[64];
+        uint32_t sc[SCOLS];
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        for (int c = 0; c < SCOLS / 32; ++c) {
           uint32_t r[32];
           tmem_ld32(s_addr + col0 + c * 32, r);
           tmem_wait_ld();
@@ -348,21 +363,16 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         float tmax = -INFINITY;
         if (full) {
 #pragma unroll
-          for (int i = 0; i < 64; ++i) tmax = fmaxf(tmax, __uint_as_float(sc[i]));
+          for (int i = 0; i < SCOLS; ++i) tmax = fmaxf(tmax, __uint_as_float(sc[i]));
         } else {
 #pragma unroll
-          for (int i = 0; i < 64; ++i)
+          for (int i = 0; i < SCOLS; ++i)
             if (col0 + i >= clo && col0 + i <= chi) tmax = fmaxf(tmax, __uint_as_float(sc[i]));
         }
         // row maximum over both halves (slots alternate with the tile parity, so the partner's
         // read of this tile cannot meet this thread's write of the next)
-        {
-          float other;
-          ok = __all_sync(0xffffffffu, pair_exchange(&sh.xmax[g & 1][half][row], &sh.xmax[g & 1][half ^ 1][row], g + 1, tmax,
-                                                     other, abort_flag));
-          if (!ok) break;
-          tmax = fmaxf(tmax, other);
-        }
+        ok = __all_sync(0xffffffffu, row_exchange<true>(&sh.xmax[g & 1][0][0], part, row, g + 1, tmax, abort_flag));
+        if (!ok) break;
         const float m_new = fmaxf(m_ref, tmax);
         const bool need = (m_new - m_ref) * sl2 > LAZY_LOG2;
         const float alpha = need ? ex2((m_ref - m_new) * sl2) : 1.f;
@@ -379,7 +389,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {
+          for (int c = 0; c < SCOLS / 32; ++c) {
             uint32_t r[32];
             tmem_ld32(o_addr + c * 32, r);
             tmem_wait_ld();
@@ -394,7 +404,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         const float mb = m_ref * sl2;
         float sum = 0.f;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        for (int c = 0; c < SCOLS / 32; ++c) {
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
@@ -425,13 +435,8 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
       }
       if (!ok) break;
       // epilogue: O / l -> Y, once the item's last PV has landed; l = the two partial row sums
-      {
-        float other;
-        ok = __all_sync(0xffffffffu, pair_exchange(&sh.xsum[iter & 1][half][row], &sh.xsum[iter & 1][half ^ 1][row],
-                                                   (unsigned)iter + 1, l, other, abort_flag));
-        if (!ok) break;
-        l += other;
-      }
+      ok = __all_sync(0xffffffffu, row_exchange<false>(&sh.xsum[iter & 1][0][0], part, row, (unsigned)iter + 1, l, abort_flag));
+      if (!ok) break;
       ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[ob], ocount[ob] & 1, abort_flag));
       ++ocount[ob];
       if (!ok) break;
@@ -440,7 +445,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
       const bool store = p < x.n;
       __nv_bfloat16* y = (x.band == 1 ? P.y_mid : P.y_high) + ((size_t)x.bh * x.n + (store ? p : 0)) * HD + col0;
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      for (int c = 0; c < SCOLS / 32; ++c) {
         uint32_t r[32];
         tmem_ld32(o_addr + c * 32, r);
         tmem_wait_ld();
