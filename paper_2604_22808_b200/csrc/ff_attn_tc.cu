@@ -2,19 +2,24 @@
 // attention": strided block-sparse attention on the mid band, sliding-window attention on the high
 // band), bf16 operands, fp32 accumulation, head_dim 128.
 //
-// One persistent launch runs both branches from a worklist of (head, band, query tile) items that
-// is rebuilt from the head-to-band allocation before every launch.  A CTA owns every gridDim-th
-// item.  Per CTA:
-//   warp 0      TMA producer: Q tile (double buffered), K and V tiles (two stages each)
-//   warp 1      tcgen05.mma issuer: S = Q K^T (A, B from shared memory), O += P V (A = P from
-//               tensor memory, B = V as an MN-major operand); owns the tensor-memory allocation
-//   warps 2..9  softmax: two threads per query row (row = TMEM lane, 64 key columns each), scores read with tcgen05.ld,
-//               key masks generated in registers from the row's band rank, P written back to
-//               tensor memory as bf16 over the scores it came from; O is accumulated in tensor
-//               memory and rescaled only when a row's running maximum grows by more than 2^8
-// Tensor memory (512 columns): S/P buffer 0, S/P buffer 1, O buffer 0, O buffer 1.
-// Every mbarrier wait is bounded; when one runs out the CTA raises FF_ERR_TIMEOUT in the plan's
-// status word, stops taking work, lets its copies drain, frees its tensor memory and returns.
+// One persistent launch runs both branches from a worklist of (head, band, pair of query tiles)
+// items that is rebuilt from the head-to-band allocation before every launch.  A CTA owns every
+// gridDim-th item.  An item is two neighbouring 128-row query tiles ("streams" A and B) that walk
+// one sequence of 128-key tiles together: both streams of a mid-band item see every key tile of
+// their residue class; in the high band the union of the two windows is 2 + 2R/128 key tiles of
+// which each stream takes part in 1 + 2R/128.  K and V tiles are therefore fetched once for two
+// query tiles, and while the softmax warps of one stream work the tensor core runs the other's MMAs.
+//   warp 0       TMA producer: the two Q tiles, K and V tiles (two stages each)
+//   warp 1       tcgen05.mma issuer: S_x = Q_x K^T (operands from shared memory), O_x += P_x V
+//                (A = P from tensor memory, B = V as an MN-major operand), issue order
+//                PV_A[j], QK_A[j+1], PV_B[j], QK_B[j+1]; owns the tensor-memory allocation
+//   warps 2..17  softmax: per stream two threads per query row (row = TMEM lane, 64 key columns
+//                each); scores read with tcgen05.ld, key masks generated in registers from the row's
+//                band rank, P written back to tensor memory as bf16 over the thread's own scores; O
+//                accumulates in tensor memory and is rescaled only when a row maximum grows by > 2^8
+// Tensor memory (512 columns): S/P of stream A, S/P of stream B, O of stream A, O of stream B.
+// Every wait is bounded; when one runs out the CTA raises FF_ERR_TIMEOUT in the plan's status
+// word, stops taking work, lets its copies drain, frees its tensor memory and returns.
 #include <cuda.h>
 
 #include "ff_internal.h"
@@ -24,14 +29,14 @@ using namespace sm100;
 
 namespace {
 
-constexpr int TILE = 128;            // query rows per item = key rows per tile
+constexpr int TILE = 128;            // query rows per stream = key rows per tile
 constexpr int HD = 128;              // head_dim
 constexpr int TILE_BYTES = TILE * HD * 2;
 constexpr int HALF_BYTES = TILE_BYTES / 2;
 constexpr int MAX_UNITS = 1024;
-constexpr int NSPLIT = 4;                // softmax threads per query row
+constexpr int NSPLIT = 2;                // softmax threads per query row
 constexpr int SCOLS = TILE / NSPLIT;     // key (and output) columns per softmax thread
-constexpr int TC_THREADS = 64 + 128 * NSPLIT;   // TMA warp, MMA warp, 4 * NSPLIT softmax warps
+constexpr int TC_THREADS = 64 + 2 * 128 * NSPLIT;   // TMA warp, MMA warp, 2 streams x 4 NSPLIT softmax warps
 constexpr float LAZY_LOG2 = 8.0f;    // rescale O only when the running max grows by more than this (log2 units)
 
 struct TcParams {
@@ -45,7 +50,7 @@ struct TcParams {
 };
 
 // Worklist: one unit per (head, mid residue class) and per (head, high band) that the allocation
-// executes; mid units first (their items are the long ones).
+// executes; mid units first (their items are the long ones).  An item is a pair of query tiles.
 __global__ void build_worklist_kernel(TcParams P) {
   if (threadIdx.x != 0 || blockIdx.x != 0) return;
   const FFDims& dm = P.dm;
@@ -60,14 +65,14 @@ __global__ void build_worklist_kernel(TcParams P) {
       const long long nblk = (dm.nb - c + dm.s - 1) / dm.s;
       const int nt = (int)((nblk * dm.b + TILE - 1) / TILE);
       offsets[nu] = total; desc[nu] = (bh << 12) | (1 << 10) | c; tiles[nu] = nt;
-      total += nt; ++nu;
+      total += (nt + 1) / 2; ++nu;
     }
   }
   for (int bh = 0; bh < dm.BH && nu < MAX_UNITS; ++bh) {
     if (!(P.alloc[bh] & FF_BAND_HIGH)) continue;
     const int nt = (int)((dm.Nhigh + TILE - 1) / TILE);
     offsets[nu] = total; desc[nu] = (bh << 12) | (2 << 10); tiles[nu] = nt;
-    total += nt; ++nu;
+    total += (nt + 1) / 2; ++nu;
   }
   offsets[nu] = total;
   P.work[0] = nu;
@@ -75,22 +80,26 @@ __global__ void build_worklist_kernel(TcParams P) {
 }
 
 struct Item {
-  int band, bh, c, tile, nk;
+  int band, bh, c;
+  int tile_a;         // query tile of stream A; stream B takes tile_a + 1
+  int has_b;          // stream B exists
+  int nk;             // key tiles of the item
   long long n;        // band length
   long long ks;       // high: first key rank of key tile 0
 };
 
 struct Shared {
-  uint64_t q_full[2], q_empty[2], k_full[2], k_empty[2], v_full[2], v_empty[2];
-  uint64_t s_full[2], p_full[2], o_full[2], o_empty[2];
+  uint64_t q_full, q_empty, k_full[2], k_empty[2], v_full[2], v_empty[2];
+  uint64_t s_full[2], p_full[2], o_full[2], o_empty[2];      // per stream
   uint32_t tmem_base;
   int abort_flag;
   int n_units, total;
   int offsets[MAX_UNITS + 1];
   int desc[MAX_UNITS];
-  // hand-shake slots of the two threads of a row: (sequence number << 32) | float bits
-  unsigned long long xmax[2][NSPLIT][128];
-  unsigned long long xsum[2][NSPLIT][128];
+  int ntile[MAX_UNITS];
+  // hand-shake slots of the threads of a row: (sequence number << 32) | float bits
+  unsigned long long xmax[2][2][NSPLIT][128];     // [parity][stream][part][row]
+  unsigned long long xsum[2][2][NSPLIT][128];
 };
 
 __device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, int it) {
@@ -102,20 +111,31 @@ __device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, 
   Item x;
   const int dsc = sh.desc[lo];
   x.bh = dsc >> 12; x.band = (dsc >> 10) & 3; x.c = dsc & 1023;
-  x.tile = it - sh.offsets[lo];
+  x.tile_a = 2 * (it - sh.offsets[lo]);
+  x.has_b = x.tile_a + 1 < sh.ntile[lo];
   if (x.band == 1) {
     x.n = dm.Nmid;
-    x.nk = sh.offsets[lo + 1] - sh.offsets[lo];     // every query tile of a class sees all its key tiles
+    x.nk = sh.ntile[lo];                  // every query tile of a class sees all its key tiles
     x.ks = 0;
   } else {
     x.n = dm.Nhigh;
-    const long long q0 = (long long)x.tile * TILE;
+    const long long q0 = (long long)x.tile_a * TILE;
     x.ks = q0 - dm.R > 0 ? q0 - dm.R : 0;
-    long long ke = q0 + TILE + dm.R;
+    long long ke = q0 + (x.has_b ? 2 : 1) * TILE + dm.R;
     if (ke > x.n) ke = x.n;
     x.nk = (int)((ke - x.ks + TILE - 1) / TILE);
   }
   return x;
+}
+
+// Does stream `sx` (0 = A, 1 = B) take part in key tile j of the item?  Mid band: always.  High
+// band: when the tile meets the window of the stream's 128 query rows.
+__device__ __forceinline__ bool stream_active(const Item& x, const FFDims& dm, int sx, int j) {
+  if (sx == 1 && !x.has_b) return false;
+  if (x.band == 1) return true;
+  const long long t0 = x.ks + (long long)j * TILE;
+  const long long q0 = (long long)(x.tile_a + sx) * TILE;
+  return t0 <= q0 + TILE - 1 + dm.R && t0 + TILE - 1 >= q0 - dm.R && t0 < x.n;
 }
 
 // Band rank of class-local position u of residue class c (mid band).
@@ -126,10 +146,10 @@ __device__ __forceinline__ long long mid_rank(const FFDims& dm, int c, long long
   return (long long)(((unsigned)c + blk * (unsigned)dm.s) * b + (uu - blk * b));
 }
 
-// Issues the TMA loads of one 128-row tile (two 64-column halves) into `dst`.
+// Issues the TMA loads of one 128-row tile (two 64-column halves) into `dst`; the caller has
+// already announced the bytes on `bar`.  `first` = class-local position (mid) or band rank (high).
 __device__ __forceinline__ void load_tile(uint8_t* dst, const CUtensorMap* map, uint64_t* bar, const FFDims& dm,
                                           const Item& x, int slice, long long first, int rb) {
-  mbar_arrive_expect_tx(bar, TILE_BYTES);
   if (x.band == 2) {
     tma_load_3d(dst, map, bar, 0, (int)first, slice);
     tma_load_3d(dst + HALF_BYTES, map, bar, 64, (int)first, slice);
@@ -146,7 +166,7 @@ __device__ __forceinline__ void load_tile(uint8_t* dst, const CUtensorMap* map, 
 
 // The NSPLIT softmax threads of a row share one float each: a thread publishes (seq, value) in its
 // slot and reads the others' slots, waiting (bounded) until they carry the same sequence number.
-// `slots` points at [NSPLIT][128] entries of one parity; MAX selects max, otherwise sum.
+// `slots` points at [NSPLIT][128] entries; MAX selects max, otherwise sum.
 template <bool MAX>
 __device__ __forceinline__ bool row_exchange(unsigned long long* slots, int part, int row, unsigned seq, float& v,
                                              volatile int* abort_flag) {
@@ -159,8 +179,8 @@ __device__ __forceinline__ bool row_exchange(unsigned long long* slots, int part
     while (true) {
       const unsigned long long w = *theirs;
       if ((unsigned)(w >> 32) == seq) {
-        const float x = __uint_as_float((unsigned)w);
-        acc = MAX ? fmaxf(acc, x) : acc + x;
+        const float xv = __uint_as_float((unsigned)w);
+        acc = MAX ? fmaxf(acc, xv) : acc + xv;
         break;
       }
       if (*abort_flag) return false;
@@ -186,16 +206,16 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
                                                   const CUtensorMap& map_c, const TcParams& P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* sQ = smem;                       // 2 x 32 KB
-  uint8_t* sK = smem + 2 * TILE_BYTES;      // 2 x 32 KB
-  uint8_t* sV = smem + 4 * TILE_BYTES;      // 2 x 32 KB
+  uint8_t* sQ = smem;                       // stream A, stream B: 2 x 32 KB
+  uint8_t* sK = smem + 2 * TILE_BYTES;      // 2 stages x 32 KB
+  uint8_t* sV = smem + 4 * TILE_BYTES;      // 2 stages x 32 KB
   Shared& sh = *(Shared*)(smem + 6 * TILE_BYTES);
   const FFDims& dm = P.dm;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
+    mbar_init(&sh.q_full, 1); mbar_init(&sh.q_empty, 1);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&sh.q_full[i], 1); mbar_init(&sh.q_empty[i], 1);
       mbar_init(&sh.k_full[i], 1); mbar_init(&sh.k_empty[i], 1);
       mbar_init(&sh.v_full[i], 1); mbar_init(&sh.v_empty[i], 1);
       mbar_init(&sh.s_full[i], 1); mbar_init(&sh.p_full[i], 128 * NSPLIT);
@@ -207,10 +227,16 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
     fence_mbar_init();
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < 2 * NSPLIT * 128; i += TC_THREADS) { (&sh.xmax[0][0][0])[i] = 0ull; (&sh.xsum[0][0][0])[i] = 0ull; }
+  for (int i = threadIdx.x; i < 2 * 2 * NSPLIT * 128; i += TC_THREADS) {
+    (&sh.xmax[0][0][0][0])[i] = 0ull;
+    (&sh.xsum[0][0][0][0])[i] = 0ull;
+  }
   for (int i = threadIdx.x; i <= sh.n_units; i += TC_THREADS) {
     sh.offsets[i] = P.work[2 + i];
-    if (i < sh.n_units) sh.desc[i] = P.work[2 + MAX_UNITS + 1 + i];
+    if (i < sh.n_units) {
+      sh.desc[i] = P.work[2 + MAX_UNITS + 1 + i];
+      sh.ntile[i] = P.work[2 + MAX_UNITS + 1 + MAX_UNITS + i];
+    }
   }
   if (warp == 1) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
   tc_fence_before();
@@ -234,18 +260,21 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         const CUtensorMap* mapv = QKV_MAPS ? &map_c : map;
         const int slice_k = QKV_MAPS ? x.bh : dm.BH + x.bh, slice_v = QKV_MAPS ? x.bh : 2 * dm.BH + x.bh;
         const int rb = x.band == 1 ? P.rb_mid : TILE;
-        const int qb = iter & 1;
-        if (iter >= 2) ok = mbar_wait(&sh.q_empty[qb], ((iter >> 1) - 1) & 1, abort_flag);
+        if (iter >= 1) ok = mbar_wait(&sh.q_empty, (iter - 1) & 1, abort_flag);
         if (!ok) break;
-        load_tile(sQ + qb * TILE_BYTES, mapq, &sh.q_full[qb], dm, x, x.bh, (long long)x.tile * TILE, rb);
+        mbar_arrive_expect_tx(&sh.q_full, x.has_b ? 2 * TILE_BYTES : TILE_BYTES);
+        load_tile(sQ, mapq, &sh.q_full, dm, x, x.bh, (long long)x.tile_a * TILE, rb);
+        if (x.has_b) load_tile(sQ + TILE_BYTES, mapq, &sh.q_full, dm, x, x.bh, (long long)(x.tile_a + 1) * TILE, rb);
         for (int j = 0; j < x.nk && ok; ++j, ++g) {
           const int st = g & 1;
           const long long first = x.band == 1 ? (long long)j * TILE : x.ks + (long long)j * TILE;
           if (g >= 2) ok = mbar_wait(&sh.k_empty[st], ((g >> 1) - 1) & 1, abort_flag);
           if (!ok) break;
+          mbar_arrive_expect_tx(&sh.k_full[st], TILE_BYTES);
           load_tile(sK + st * TILE_BYTES, mapk, &sh.k_full[st], dm, x, slice_k, first, rb);
           if (g >= 2) ok = mbar_wait(&sh.v_empty[st], ((g >> 1) - 1) & 1, abort_flag);
           if (!ok) break;
+          mbar_arrive_expect_tx(&sh.v_full[st], TILE_BYTES);
           load_tile(sV + st * TILE_BYTES, mapv, &sh.v_full[st], dm, x, slice_v, first, rb);
         }
       }
@@ -256,74 +285,114 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
       const uint32_t idesc_qk = idesc_bf16_f32(TILE, TILE, false, false);
       const uint32_t idesc_pv = idesc_bf16_f32(TILE, HD, false, true);
       int iter = 0; unsigned g = 0;
-      bool ok = true, have_prev = false;
-      unsigned pg = 0; int pob = 0, piter = 0; bool pfirst = false;
-      auto issue_pv = [&]() -> bool {
-        const int sb = pg & 1, st = pg & 1;
-        if (!mbar_wait(&sh.p_full[sb], (pg >> 1) & 1, abort_flag)) return false;
-        if (!mbar_wait(&sh.v_full[st], (pg >> 1) & 1, abort_flag)) return false;
-        if (pfirst && piter >= 2 && !mbar_wait(&sh.o_empty[pob], ((piter >> 1) - 1) & 1, abort_flag)) return false;
+      unsigned cp[2] = {0, 0};          // P phases consumed per stream
+      unsigned ce[2] = {0, 0};          // items seen per stream (for the O buffer hand-back)
+      bool ok = true;
+      // S_x = Q_x K[tile]^T; `last` = no further QK uses this K stage
+      auto issue_qk = [&](int sx, unsigned gt, bool last, bool release_q) {
+        const int st = gt & 1;
+        const uint32_t qbase = smem_u32(sQ + sx * TILE_BYTES), kbase = smem_u32(sK + st * TILE_BYTES);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint32_t off = (k >> 2) * HALF_BYTES + (k & 3) * 32;
+          umma_ss(tm + sx * 128, smem_desc_sw128(qbase + off, 16, 1024), smem_desc_sw128(kbase + off, 16, 1024),
+                  idesc_qk, k > 0 ? 1u : 0u);
+        }
+        umma_commit(&sh.s_full[sx]);
+        if (last) umma_commit(&sh.k_empty[st]);
+        if (release_q) umma_commit(&sh.q_empty);
+      };
+      // O_x (+)= P_x V[tile]
+      auto issue_pv = [&](int sx, unsigned gt, bool first_of_item, bool last) -> bool {
+        const int st = gt & 1;
+        if (!mbar_wait(&sh.p_full[sx], cp[sx] & 1, abort_flag)) return false;
+        ++cp[sx];
+        if (first_of_item && ce[sx] >= 1 && !mbar_wait(&sh.o_empty[sx], (ce[sx] - 1) & 1, abort_flag)) return false;
         tc_fence_after();
         const uint32_t vbase = smem_u32(sV + st * TILE_BYTES);
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-          umma_ts(tm + 256 + pob * 128, tm + sb * 128 + k * 8, smem_desc_sw128(vbase + k * 2048, HALF_BYTES, 1024),
-                  idesc_pv, (pfirst && k == 0) ? 0u : 1u);
-        umma_commit(&sh.v_empty[st]);
-        umma_commit(&sh.o_full[pob]);
+        for (int k = 0; k < 8; ++k) {
+          // P of keys 16k..16k+15 sits at the start of the score columns of the thread that owns them
+          const uint32_t pcol = ((16 * k) / SCOLS) * SCOLS + ((16 * k) % SCOLS) / 2;
+          umma_ts(tm + 256 + sx * 128, tm + sx * 128 + pcol, smem_desc_sw128(vbase + k * 2048, HALF_BYTES, 1024),
+                  idesc_pv, (first_of_item && k == 0) ? 0u : 1u);
+        }
+        umma_commit(&sh.o_full[sx]);
+        if (last) umma_commit(&sh.v_empty[st]);
         return true;
       };
       for (int it = blockIdx.x; it < total && ok; it += gridDim.x, ++iter) {
         const Item x = decode_item(sh, dm, it);
-        const int qb = iter & 1;
-        ok = mbar_wait(&sh.q_full[qb], (iter >> 1) & 1, abort_flag);
-        for (int j = 0; j < x.nk && ok; ++j, ++g) {
-          const int st = g & 1, sb = g & 1;
-          ok = mbar_wait(&sh.k_full[st], (g >> 1) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t qbase = smem_u32(sQ + qb * TILE_BYTES), kbase = smem_u32(sK + st * TILE_BYTES);
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const uint32_t off = (k >> 2) * HALF_BYTES + (k & 3) * 32;
-            umma_ss(tm + sb * 128, smem_desc_sw128(qbase + off, 16, 1024), smem_desc_sw128(kbase + off, 16, 1024),
-                    idesc_qk, k > 0 ? 1u : 0u);
-          }
-          umma_commit(&sh.k_empty[st]);
-          umma_commit(&sh.s_full[sb]);
-          if (j == x.nk - 1) umma_commit(&sh.q_empty[qb]);
-          if (have_prev) ok = issue_pv();
-          pg = g; pob = iter & 1; piter = iter; pfirst = (j == 0); have_prev = true;
+        ok = mbar_wait(&sh.q_full, iter & 1, abort_flag);
+        if (!ok) break;
+        const unsigned g0 = g;
+        bool started[2] = {false, false};
+        // key tile 0: QK of both streams
+        ok = mbar_wait(&sh.k_full[g0 & 1], (g0 >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        {
+          const bool a0 = stream_active(x, dm, 0, 0), b0 = stream_active(x, dm, 1, 0);
+          if (a0) issue_qk(0, g0, !b0, x.nk == 1 && !b0);
+          if (b0) issue_qk(1, g0, true, x.nk == 1);
         }
+        for (int j = 0; j < x.nk && ok; ++j) {
+          const unsigned gt = g0 + j;
+          const bool aj = stream_active(x, dm, 0, j), bj = stream_active(x, dm, 1, j);
+          const bool more = j + 1 < x.nk;
+          const bool an = more && stream_active(x, dm, 0, j + 1), bn = more && stream_active(x, dm, 1, j + 1);
+          bool v_ready = false, k_ready = false;
+          for (int sx = 0; sx < 2 && ok; ++sx) {
+            const bool act = sx ? bj : aj, nxt = sx ? bn : an;
+            if (act) {
+              if (!v_ready) { ok = mbar_wait(&sh.v_full[gt & 1], (gt >> 1) & 1, abort_flag); v_ready = true; if (!ok) break; }
+              const bool last_pv = sx == 1 || !bj;
+              ok = issue_pv(sx, gt, !started[sx], last_pv);
+              started[sx] = true;
+              if (!ok) break;
+            }
+            if (nxt) {
+              if (!k_ready) { ok = mbar_wait(&sh.k_full[(gt + 1) & 1], ((gt + 1) >> 1) & 1, abort_flag); k_ready = true; if (!ok) break; tc_fence_after(); }
+              const bool last_qk = sx == 1 || !bn;
+              issue_qk(sx, gt + 1, last_qk, last_qk && j + 2 == x.nk);
+            }
+          }
+        }
+        g = g0 + x.nk;
+        ce[0] += 1;
+        if (x.has_b) ce[1] += 1;
       }
-      if (ok && have_prev) issue_pv();
     }
   } else {
-    // ------------------------------------------------------------------ softmax, two threads per row
-    // Warps 2..5 take key columns 0..63 of their 32 rows, warps 6..9 columns 64..127 of the same
-    // rows (a warp reaches the TMEM lanes 32*(warp%4)..+31), so every scheduler has two softmax warps
-    // to interleave.  The two threads of a row agree on the row maximum through shared memory and a
-    // bounded hand-shake; each keeps the partial row sum of its own columns.
+    // ------------------------------------------------------------------ softmax
+    // Warps 2..9 serve stream A, 10..17 stream B.  Inside a stream the first four warps take key
+    // columns 0..63 of their 32 rows, the next four columns 64..127 (a warp reaches the TMEM lanes
+    // 32*(warp%4)..+31).  The threads of a row agree on the row maximum through a bounded
+    // hand-shake in shared memory; each keeps the partial row sum of its own columns.
     const int quarter = warp & 3;
-    const int part = (warp - 2) >> 2;                      // which SCOLS-wide column slice of the row
+    const int sx = (warp - 2) / (4 * NSPLIT);
+    const int part = ((warp - 2) >> 2) % NSPLIT;
     const int row = quarter * 32 + lane;
     const int col0 = part * SCOLS;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const uint32_t s_addr = tm + lane_addr + sx * 128;
+    const uint32_t o_addr = tm + lane_addr + 256 + sx * 128 + col0;      // this thread's output columns
     const float sl2 = rsqrtf((float)HD) * 1.4426950408889634f;
-    int iter = 0; unsigned g = 0;
-    unsigned ocount[2] = {0, 0};
+    unsigned cs = 0;                  // key tiles this stream has processed (phases of s_full / p_full)
+    unsigned co = 0;                  // phases of o_full consumed
+    unsigned ci = 0;                  // items this stream has processed
     bool ok = true;
-    for (int it = blockIdx.x; it < total && ok; it += gridDim.x, ++iter) {
+    for (int it = blockIdx.x; it < total && ok; it += gridDim.x) {
       const Item x = decode_item(sh, dm, it);
-      const int ob = iter & 1;
-      const uint32_t o_addr = tm + lane_addr + 256 + ob * 128 + col0;      // this thread's 64 output columns
+      if (sx == 1 && !x.has_b) continue;
+      const int tile = x.tile_a + sx;
       // band rank of this thread's query row
-      const long long u_q = (long long)x.tile * TILE + row;
+      const long long u_q = (long long)tile * TILE + row;
       const long long p = x.band == 1 ? mid_rank(dm, x.c, u_q) : u_q;
       float m_ref = -1e30f, l = 0.f;
-      for (int j = 0; j < x.nk && ok; ++j, ++g) {
-        const int sb = g & 1;
-        const uint32_t s_addr = tm + lane_addr + sb * 128;
+      bool first = true;
+      for (int j = 0; j < x.nk && ok; ++j) {
+        if (!stream_active(x, dm, sx, j)) continue;
         // valid key columns [clo, chi] of this row in this tile
         int clo = 0, chi = TILE - 1;
         bool full;
@@ -339,7 +408,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
           }
         } else {
           const long long t0 = x.ks + (long long)j * TILE;
-          const long long q0 = (long long)x.tile * TILE;
+          const long long q0 = (long long)tile * TILE;
           full = (t0 >= q0 + TILE - 1 - dm.R) && (t0 + TILE - 1 <= q0 + dm.R) && (t0 + TILE <= x.n);
           if (!full) {
             const long long lo = p - dm.R - t0, hi = (p + dm.R < x.n - 1 ? p + dm.R : x.n - 1) - t0;
@@ -347,44 +416,41 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
             chi = hi < TILE - 1 ? (int)(hi < -1 ? -1 : hi) : TILE - 1;
           }
         }
-        ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full[sb], (g >> 1) & 1, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full[sx], cs & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
-        // this thread's 64 raw scores into registers (P will overwrite them in tensor memory)
-        uint32_t sc[SCOLS];
+        // first sweep over this thread's raw scores: the row maximum of its columns
+        float tmax = -INFINITY;
 #pragma unroll
         for (int c = 0; c < SCOLS / 32; ++c) {
           uint32_t r[32];
           tmem_ld32(s_addr + col0 + c * 32, r);
           tmem_wait_ld();
+          if (full) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) sc[c * 32 + i] = r[i];
+            for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, __uint_as_float(r[i]));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (col0 + c * 32 + i >= clo && col0 + c * 32 + i <= chi) tmax = fmaxf(tmax, __uint_as_float(r[i]));
+          }
         }
-        float tmax = -INFINITY;
-        if (full) {
-#pragma unroll
-          for (int i = 0; i < SCOLS; ++i) tmax = fmaxf(tmax, __uint_as_float(sc[i]));
-        } else {
-#pragma unroll
-          for (int i = 0; i < SCOLS; ++i)
-            if (col0 + i >= clo && col0 + i <= chi) tmax = fmaxf(tmax, __uint_as_float(sc[i]));
-        }
-        // row maximum over both halves (slots alternate with the tile parity, so the partner's
+        // row maximum over the row's threads (slots alternate with the tile parity, so a partner's
         // read of this tile cannot meet this thread's write of the next)
-        ok = __all_sync(0xffffffffu, row_exchange<true>(&sh.xmax[g & 1][0][0], part, row, g + 1, tmax, abort_flag));
+        ok = __all_sync(0xffffffffu, row_exchange<true>(&sh.xmax[cs & 1][sx][0][0], part, row, cs + 1, tmax, abort_flag));
         if (!ok) break;
         const float m_new = fmaxf(m_ref, tmax);
         const bool need = (m_new - m_ref) * sl2 > LAZY_LOG2;
         const float alpha = need ? ex2((m_ref - m_new) * sl2) : 1.f;
-        // Completion j-1 of this buffer's barrier (the PV of the previous key tile) is normally
-        // awaited at the end of this tile, just before P is published, when it has long happened;
-        // only a row maximum that grew past the lazy threshold needs it now, because O is then
-        // rescaled in place.  Every phase of the barrier is awaited exactly once, in order (parity
-        // waits must not skip phases).  Both threads of a row see the same `need`.
+        // The phase of the previous PV of this stream is normally consumed at the end of this tile,
+        // just before P is published, when it has long completed; only a row maximum that grew past
+        // the lazy threshold needs it now, because O is then rescaled in place.  Every phase of the
+        // barrier is awaited exactly once, in order (parity waits must not skip phases), and before
+        // the arrival that lets the next PV be issued.  All threads of a row see the same `need`.
         bool waited_prev = false;
-        if (j > 0 && __any_sync(0xffffffffu, need)) {
-          ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[ob], ocount[ob] & 1, abort_flag));
-          ++ocount[ob];
+        if (!first && __any_sync(0xffffffffu, need)) {
+          ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[sx], co & 1, abort_flag));
+          ++co;
           waited_prev = true;
           if (!ok) break;
           tc_fence_after();
@@ -405,12 +471,17 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         float sum = 0.f;
 #pragma unroll
         for (int c = 0; c < SCOLS / 32; ++c) {
+          // second sweep: the scores again (tensor-memory reads are cheap; keeping them in registers
+          // is not, with 576 threads per CTA), P written over them
+          uint32_t r[32];
+          tmem_ld32(s_addr + col0 + c * 32, r);
+          tmem_wait_ld();
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const int k = c * 32 + 2 * i, col = col0 + k;
-            float p0 = ex2(fmaf(__uint_as_float(sc[k]), sl2, -mb));
-            float p1 = ex2(fmaf(__uint_as_float(sc[k + 1]), sl2, -mb));
+            const int col = col0 + c * 32 + 2 * i;
+            float p0 = ex2(fmaf(__uint_as_float(r[2 * i]), sl2, -mb));
+            float p1 = ex2(fmaf(__uint_as_float(r[2 * i + 1]), sl2, -mb));
             if (!full) {
               if (col < clo || col > chi) p0 = 0.f;
               if (col + 1 < clo || col + 1 > chi) p1 = 0.f;
@@ -419,26 +490,26 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
             const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
             pk[i] = *(const uint32_t*)&v;
           }
-          tmem_st16(s_addr + (col0 >> 1) + c * 16, pk);
+          tmem_st16(s_addr + col0 + c * 16, pk);      // inside this thread's own score columns
         }
         l += sum;
         tmem_wait_st();
-        // (this wait has to precede the arrival below: PV j may not be issued, let alone complete,
-        // before this thread has consumed the phase of PV j-1)
-        if (j > 0 && !waited_prev) {
-          ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[ob], ocount[ob] & 1, abort_flag));
-          ++ocount[ob];
+        if (!first && !waited_prev) {
+          ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[sx], co & 1, abort_flag));
+          ++co;
           if (!ok) break;
         }
         tc_fence_before();
-        mbar_arrive(&sh.p_full[sb]);
+        mbar_arrive(&sh.p_full[sx]);
+        first = false;
+        ++cs;
       }
       if (!ok) break;
-      // epilogue: O / l -> Y, once the item's last PV has landed; l = the two partial row sums
-      ok = __all_sync(0xffffffffu, row_exchange<false>(&sh.xsum[iter & 1][0][0], part, row, (unsigned)iter + 1, l, abort_flag));
+      // epilogue: O / l -> Y, once the item's last PV has landed; l = the partial row sums together
+      ok = __all_sync(0xffffffffu, row_exchange<false>(&sh.xsum[ci & 1][sx][0][0], part, row, ci + 1, l, abort_flag));
       if (!ok) break;
-      ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[ob], ocount[ob] & 1, abort_flag));
-      ++ocount[ob];
+      ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[sx], co & 1, abort_flag));
+      ++co;
       if (!ok) break;
       tc_fence_after();
       const float inv = 1.f / l;
@@ -464,7 +535,8 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         }
       }
       tc_fence_before();
-      mbar_arrive(&sh.o_empty[ob]);
+      mbar_arrive(&sh.o_empty[sx]);
+      ++ci;
     }
   }
 
