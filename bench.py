@@ -212,6 +212,17 @@ def reduce_max(x: float, world: int, device) -> float:
     return float(t.item())
 
 
+def forced_allocation(cfg, text):
+    """'L,M,H' (heads per band, summing to the head count) -> band masks of every (batch, head);
+    heads [0,L) run the low band, the next M the mid band, the rest the high band."""
+    if not text:
+        return None
+    n = [int(x) for x in text.split(",")]
+    if len(n) != 3 or min(n) < 0 or sum(n) != cfg.heads:
+        raise SystemExit(f"--alloc wants L,M,H summing to {cfg.heads} heads")
+    return ([1] * n[0] + [2] * n[1] + [4] * n[2]) * cfg.batch
+
+
 def aggregate_tokens_per_s(cfg, world: int, ms_step_max: float) -> float:
     """Whole-job throughput: the tokens all ranks processed over the slowest rank's step time."""
     return cfg.batch * cfg.N * world / (ms_step_max * 1e-3)
@@ -244,6 +255,9 @@ def run_cuda(args, cfg):
     plan.set_profiling(True)
     plan.set_attention_impl(args.kernel_select)
     ts = [cfg.timesteps[args.timestep_index]] * cfg.batch
+    forced = forced_allocation(cfg, args.alloc)
+    alloc_dev = None if forced is None else torch.tensor(forced, dtype=torch.uint8, device=dev)
+    alloc_np = None if forced is None else np.asarray(forced, np.uint8)
     torch.cuda.synchronize()
 
     def barrier():
@@ -257,7 +271,7 @@ def run_cuda(args, cfg):
 
     # device-resident timing
     for _ in range(args.warmup):
-        plan.forward(q, k, v, out, timesteps=ts)
+        plan.forward(q, k, v, out, alloc=alloc_dev, timesteps=ts)
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
@@ -266,7 +280,7 @@ def run_cuda(args, cfg):
     stage_launches = {}
     ev[0].record()
     for i in range(args.steps):
-        plan.forward(q, k, v, out, timesteps=ts)
+        plan.forward(q, k, v, out, alloc=alloc_dev, timesteps=ts)
         ev[i + 1].record()
         for name, (ms, n) in plan.stage_times().items():       # waits for this step's last event
             stage_ms[name] += ms / args.steps
@@ -277,19 +291,19 @@ def run_cuda(args, cfg):
     launches = plan.last_launches()
     if plan.device_status() != 0:
         raise RuntimeError(B.library().ff_last_error(plan.handle).decode())
-    alloc = plan.tap(B.TAP_ALLOC).cpu().numpy().tolist()
-    pi = plan.tap(B.TAP_PI).cpu().numpy().tolist()
+    alloc = forced if forced is not None else plan.tap(B.TAP_ALLOC).cpu().numpy().tolist()
+    pi = [None] if forced is not None else plan.tap(B.TAP_PI).cpu().numpy().tolist()
 
     # end to end through the host-buffer entry point (pinned host memory, copies inside the call)
     e2e_ms = float("nan")
     if not args.no_e2e:
         for _ in range(min(2, args.warmup)):
-            plan.forward_host(host[0], host[1], host[2], out_host, timesteps=ts)
+            plan.forward_host(host[0], host[1], host[2], out_host, alloc_host=alloc_np, timesteps=ts)
         barrier()
         e2e_steps = max(1, min(args.steps, 5))
         t0 = time.perf_counter()
         for _ in range(e2e_steps):
-            plan.forward_host(host[0], host[1], host[2], out_host, timesteps=ts)      # synchronises the stream
+            plan.forward_host(host[0], host[1], host[2], out_host, alloc_host=alloc_np, timesteps=ts)      # synchronises the stream
         e2e_ms = reduce_max_((time.perf_counter() - t0) * 1e3 / e2e_steps)
         barrier()
 
@@ -329,7 +343,7 @@ def run_cuda(args, cfg):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
             "config": {"workload": cfg.name, "grid": list(cfg.grid), "batch": cfg.batch, "heads": cfg.heads,
-                       "head_dim": cfg.head_dim, "timestep": ts[0], "allocation": "router",
+                       "head_dim": cfg.head_dim, "timestep": ts[0], "allocation": "router" if forced is None else "forced",
                        "heads_per_band": [alloc.count(1), alloc.count(2), alloc.count(4)], "pi": pi[0],
                        "l2": "inputs (%.0f MB) larger than L2" % (3 * io_bytes / 1e6)},
             "roofline": roof,
@@ -359,6 +373,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="64k")
     ap.add_argument("--timestep-index", type=int, default=0)
+    ap.add_argument("--alloc", default="", help="forced heads per band 'L,M,H' instead of the router's allocation")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--heads", type=int, default=0, help="override the number of heads (profiling on a small case)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling)")

@@ -18,7 +18,12 @@
 //
 //   warp 0      TMA producer (ring of 2-4 stages, as many as fit beside the matrix images)
 //   warp 1      tcgen05.mma issuer, 4 accumulator buffers of 128 TMEM columns
-//   warps 2..5  epilogue: tcgen05.ld, convert, store
+//   warps 2..9  epilogue: tcgen05.ld, convert to hi/lo bf16, store; a thread owns one output position
+// Output path (FIRST, MIDDLE, LAST): an epilogue warp's 32 rows are 32 grid positions that form a
+// box of the grid, so the warp writes 32 channels of them (64 bytes per row, 64-byte swizzle, no
+// bank conflicts) into its own staging area and one lane sends them out with a tensor store; the
+// area is reused when that store has read it.  SPLIT scatters rows to band positions: staged the
+// same way, then stored by all lanes with four lanes per 64-byte row piece.
 // Modes: FIRST  caller's Q/K/V -> hi/lo intermediate, plus an fp32 copy of the rows k_w < L_w
 //               from which the low band is computed at full precision
 //        MIDDLE hi/lo intermediate -> hi/lo intermediate
@@ -72,7 +77,7 @@ struct DctShared {
   int abort_flag;
   // per epilogue warp: 32 rows x 64 bytes of hi and of lo, to turn one-row-per-thread registers
   // into stores where four lanes cover a row's 64 contiguous bytes
-  alignas(16) uint8_t stage[8][2][32 * STG_PITCH];
+  alignas(1024) uint8_t stage[8][2][32 * STG_PITCH];
 };
 
 // Grid coordinates (w, h, t) of the first position of tile `u` of a tensor-head.  A tile holds
@@ -91,6 +96,16 @@ __device__ __forceinline__ void tma_load_5d(void* smem_dst, const CUtensorMap* m
       : "memory");
 }
 
+__device__ __forceinline__ void tma_store_5d(const void* smem_src, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                             int c4) {
+  asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
+               ::"l"((uint64_t)map), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(smem_u32(smem_dst)), "l"((uint64_t)gsrc), "r"(bytes), "r"(smem_u32(bar))
@@ -98,9 +113,12 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
 }
 
 // Three source maps (Q, K, V) in MODE_FIRST; otherwise map0 (= hi) and, for split input, map1 (= lo).
+// map_oh / map_ol: destination hi / lo grids with the box of one epilogue warp (32 positions x 32
+// channels), all modes but SPLIT; MODE_LAST has no lo grid.
 __global__ void __launch_bounds__(DCT_TC_THREADS, 1)
 dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
-              const __grid_constant__ CUtensorMap map2, const DctTcParams P) {
+              const __grid_constant__ CUtensorMap map2, const __grid_constant__ CUtensorMap map_oh,
+              const __grid_constant__ CUtensorMap map_ol, const DctTcParams P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const FFDims& dm = P.dm;
@@ -110,6 +128,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
   const int ln = 31 - __clz(n);
   const bool seq = P.axis == 2;                           // lines follow one another (w axis) or interleave
   const int NSTAGE = P.nstage;
+  const bool tma_out = P.mode != MODE_SPLIT;
   const int STAGE_BYTES = P.in_split ? 2 * TILE_BYTES : TILE_BYTES;
   uint8_t* sData = smem;                                  // NSTAGE x STAGE_BYTES
   uint8_t* sHi = smem + NSTAGE * STAGE_BYTES;             // matrix hi: [K half][128 rows][128 B], swizzled
@@ -201,10 +220,11 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const int ew = warp - 2;                              // epilogue warp 0..7: warps 0-3 take channels 0..63, 4-7 channels 64..127
     const int q_lo = (ew >> 2) * 2;
-    const long long N_d = dm.N * CH;
-    const long long axis_stride = (P.axis == 2 ? 1LL : (P.axis == 1 ? (long long)dm.W : (long long)dm.W * dm.H)) * CH;
-    const long long line_stride = (P.axis == 2 ? (long long)dm.W : 1LL) * CH;   // between the lines of a tile
-    const long long row_off = (long long)a * axis_stride + (long long)l * line_stride;
+    // Grid offset of the warp's first row (tile row 32 quarter) from the tile origin: the warp's 32
+    // rows are the box [32 channels] x [these offsets .. + the extents the store map was built with]
+    const int j0 = quarter * 32;
+    const int a0 = seq ? j0 & (n - 1) : j0 >> lkf, l0 = seq ? j0 >> ln : j0 & (kf - 1);
+    const int dw = P.axis == 2 ? a0 : l0, dh = P.axis == 2 ? l0 : (P.axis == 1 ? a0 : 0), dt = P.axis == 0 ? a0 : 0;
     const int Lhw = dm.L[1] * dm.L[2], Mhw = dm.M[1] * dm.M[2];
     // lane k of a warp accumulates the energies of channels 32 q + k over the warp's rows
     float em[4] = {0.f, 0.f, 0.f, 0.f}, eh[4] = {0.f, 0.f, 0.f, 0.f};
@@ -228,11 +248,10 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
       tc_fence_after();
       const int gi = s / tiles_per_th, u = s % tiles_per_th;
       int w, h, t; tile_origin(dm, P.axis, kf, u, w, h, t);
-      const long long pos0 = (((long long)t * dm.H + h) * dm.W + w) * CH;           // first position of the tile
       const int th = P.group_start + gi;
       const int tensor = th / dm.BH, bh = th % dm.BH;
       // where this thread's row goes
-      __nv_bfloat16* row_hi = nullptr; __nv_bfloat16* row_lo = nullptr; float* row_f32 = nullptr;
+      __nv_bfloat16* row_hi = nullptr; float* row_f32 = nullptr;
       int band = -1;
       if (P.mode == MODE_SPLIT) {
         const int sample = bh / dm.heads;
@@ -254,20 +273,17 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
           band = 2;
           row_hi = P.spec_high + (((size_t)tensor * dm.BH + bh) * dm.Nhigh + ((((long long)kt * dm.H + h) * dm.W + ww) - cm)) * CH;
         }
-      } else {
-        const size_t o = (size_t)(P.mode == MODE_LAST ? th : gi) * N_d + pos0 + row_off;
-        row_hi = P.dst + o;
-        if (P.mode != MODE_LAST) row_lo = P.dst_lo + o;
-        if (P.mode == MODE_FIRST && a < dm.L[2]) row_f32 = P.side + ((((size_t)gi * dm.T + t) * dm.H + h + l) * dm.L[2] + a) * CH;
+      } else if (P.mode == MODE_FIRST && a < dm.L[2]) {
+        row_f32 = P.side + ((((size_t)gi * dm.T + t) * dm.H + h + l) * dm.L[2] + a) * CH;
       }
-      // lane L stores for rows 8 i + L/4 of its warp: fetch those rows' destinations
-      __nv_bfloat16* dst_hi[4]; __nv_bfloat16* dst_lo[4];
+      // (SPLIT) lane L stores for rows 8 i + L/4 of its warp: fetch those rows' destinations
+      __nv_bfloat16* dst_hi[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int src = 8 * i + (lane >> 2);
         dst_hi[i] = (__nv_bfloat16*)__shfl_sync(0xffffffffu, (unsigned long long)row_hi, src);
-        dst_lo[i] = (__nv_bfloat16*)__shfl_sync(0xffffffffu, (unsigned long long)row_lo, src);
       }
+      const int out_slice = P.mode == MODE_LAST ? th : gi;
 #pragma unroll
       for (int q = q_lo; q < q_lo + 2; ++q) {
         uint32_t r[32];
@@ -317,36 +333,59 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
           }
         }
         {
+          const bool want_lo = P.mode == MODE_FIRST || P.mode == MODE_MIDDLE;
           uint32_t hi[16], lo[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float v0 = __uint_as_float(r[2 * i]), v1 = __uint_as_float(r[2 * i + 1]);
-            const __nv_bfloat162 hp = __floats2bfloat162_rn(v0, v1);
+            const __nv_bfloat162 hp = __floats2bfloat162_rn(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
             hi[i] = *(const uint32_t*)&hp;
-            const __nv_bfloat162 lp = __floats2bfloat162_rn(v0 - __uint_as_float(hi[i] << 16), v1 - __uint_as_float(hi[i] & 0xffff0000u));
-            lo[i] = *(const uint32_t*)&lp;
+          }
+          if (want_lo) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const __nv_bfloat162 lp = __floats2bfloat162_rn(__uint_as_float(r[2 * i]) - __uint_as_float(hi[i] << 16),
+                                                             __uint_as_float(r[2 * i + 1]) - __uint_as_float(hi[i] & 0xffff0000u));
+              lo[i] = *(const uint32_t*)&lp;
+            }
           }
           uint8_t* st_hi = sh.stage[ew][0];
           uint8_t* st_lo = sh.stage[ew][1];
+          if (tma_out) {
+            // the previous store of this warp must have read the staging area
+            if (lane == 0) bulk_wait_read0();
+            __syncwarp();
+          }
+          // 16-byte chunk i of row `lane` at chunk position i ^ (lane / 2 % 4): the 64-byte swizzle
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            *(uint4*)(st_hi + lane * STG_PITCH + (((i + (lane >> 1)) & 3) << 4)) = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
-            *(uint4*)(st_lo + lane * STG_PITCH + (((i + (lane >> 1)) & 3) << 4)) = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
+            *(uint4*)(st_hi + lane * STG_PITCH + ((i ^ ((lane >> 1) & 3)) << 4)) = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
+            if (want_lo)
+              *(uint4*)(st_lo + lane * STG_PITCH + ((i ^ ((lane >> 1) & 3)) << 4)) = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
           }
-          __syncwarp();
+          if (tma_out) {
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_5d(st_hi, &map_oh, q * 32, w + dw, h + dh, t + dt, out_slice);
+              if (want_lo) tma_store_5d(st_lo, &map_ol, q * 32, w + dw, h + dh, t + dt, out_slice);
+              bulk_commit();
+            }
+          } else {
+            __syncwarp();
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int rr = 8 * i + (lane >> 2), piece = lane & 3;      // row of the warp, 16-byte piece of its 64 bytes
-            if (dst_hi[i]) *(uint4*)(dst_hi[i] + q * 32 + piece * 8) = *(const uint4*)(st_hi + rr * STG_PITCH + (((piece + (rr >> 1)) & 3) << 4));
-            if (dst_lo[i]) *(uint4*)(dst_lo[i] + q * 32 + piece * 8) = *(const uint4*)(st_lo + rr * STG_PITCH + (((piece + (rr >> 1)) & 3) << 4));
+            for (int i = 0; i < 4; ++i) {
+              const int rr = 8 * i + (lane >> 2), piece = lane & 3;      // row of the warp, 16-byte piece of its 64 bytes
+              if (dst_hi[i]) *(uint4*)(dst_hi[i] + q * 32 + piece * 8) = *(const uint4*)(st_hi + rr * STG_PITCH + ((piece ^ ((rr >> 1) & 3)) << 4));
+            }
+            __syncwarp();
           }
-          __syncwarp();
         }
       }
       tc_fence_before();
       mbar_arrive(&sh.acc_empty[ab]);
     }
     if (P.mode == MODE_SPLIT) flush_energy();
+    if (tma_out && lane == 0) bulk_wait0();
   }
 
   tc_fence_before();
@@ -457,8 +496,36 @@ bool encode_grid_map(CUtensorMap* map, const void* base, const FFDims& dm, int s
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-cudaError_t launch_pass(ff_plan* p, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& m2, DctTcParams& P,
-                        cudaStream_t st) {
+// Store map over the same kind of grid: the box is what one epilogue warp holds, 32 channels of the
+// 32 positions of a quarter tile (tile rows 32 q .. 32 q + 31 of a pass along `axis`), 64-byte swizzle.
+bool encode_store_map(CUtensorMap* map, const void* base, const FFDims& dm, int slices, int axis) {
+  static EncodeTiledFn enc = nullptr;
+  if (!enc) {
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", (void**)&enc, cudaEnableDefault, &qr) != cudaSuccess || !enc)
+      return false;
+  }
+  cuuint64_t dims[5] = {(cuuint64_t)CH, (cuuint64_t)dm.W, (cuuint64_t)dm.H, (cuuint64_t)dm.T, (cuuint64_t)slices};
+  cuuint64_t strides[4] = {(cuuint64_t)CH * 2, (cuuint64_t)dm.W * CH * 2, (cuuint64_t)dm.H * dm.W * CH * 2,
+                           (cuuint64_t)dm.N * CH * 2};
+  const int n = axis == 2 ? dm.W : (axis == 1 ? dm.H : dm.T);
+  const int kf = TILE_ROWS / n;
+  cuuint32_t box[5] = {32, 1, 1, 1, 1};
+  if (axis == 2) {                       // rows = line * n + a: 32 consecutive rows
+    box[1] = (cuuint32_t)(n < 32 ? n : 32);
+    box[2] = (cuuint32_t)(n < 32 ? 32 / n : 1);
+  } else {                               // rows = a * kf + line: 32 consecutive rows
+    box[1] = (cuuint32_t)(kf < 32 ? kf : 32);
+    box[1 + (2 - axis)] = (cuuint32_t)(kf < 32 ? 32 / kf : 1);
+  }
+  cuuint32_t es[5] = {1, 1, 1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, es,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+cudaError_t launch_pass(ff_plan* p, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& m2,
+                        const CUtensorMap& moh, const CUtensorMap& mol, DctTcParams& P, cudaStream_t st) {
   const size_t img = TILE_BYTES;
   const size_t stage = P.in_split ? 2 * TILE_BYTES : TILE_BYTES;
   const size_t fixed = 2 * img + sizeof(DctShared) + 1024;
@@ -470,7 +537,7 @@ cudaError_t launch_pass(ff_plan* p, const CUtensorMap& m0, const CUtensorMap& m1
   if (e != cudaSuccess) return e;
   const int stages = (int)(P.group * (P.dm.N / TILE_ROWS));
   const int grid = stages < p->sm_count ? stages : p->sm_count;
-  dct_tc_kernel<<<grid, DCT_TC_THREADS, smem, st>>>(m0, m1, m2, P);
+  dct_tc_kernel<<<grid, DCT_TC_THREADS, smem, st>>>(m0, m1, m2, moh, mol, P);
   p->launches += 1;
   return cudaGetLastError();
 }
@@ -544,11 +611,15 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
   const int G = p->dct_group;
   const Scratch sc = carve(p);
   float* side = sc.side;
-  CUtensorMap mq, mk, mv, m1h, m1l, m2h, m2l;
+  // mXh/mXl: load maps of a pass's input pair; oXh/oXl: store maps of a pass's output pair (the box
+  // follows the axis of the pass that uses the map)
+  CUtensorMap mq, mk, mv, m1h, m1l, m2h, m2l, o0h, o0l, o1h, o1l;
   if (!encode_grid_map(&mq, Q, dm, dm.BH, 2) || !encode_grid_map(&mk, K, dm, dm.BH, 2) ||
       !encode_grid_map(&mv, V, dm, dm.BH, 2) || !encode_grid_map(&m1h, sc.a_hi, dm, G, 1) ||
       !encode_grid_map(&m1l, sc.a_lo, dm, G, 1) || !encode_grid_map(&m2h, sc.b_hi, dm, G, 0) ||
-      !encode_grid_map(&m2l, sc.b_lo, dm, G, 0))
+      !encode_grid_map(&m2l, sc.b_lo, dm, G, 0) || !encode_store_map(&o0h, sc.a_hi, dm, G, 2) ||
+      !encode_store_map(&o0l, sc.a_lo, dm, G, 2) || !encode_store_map(&o1h, sc.b_hi, dm, G, 1) ||
+      !encode_store_map(&o1l, sc.b_lo, dm, G, 1))
     return cudaErrorInvalidValue;
   const int total = 3 * dm.BH;
   const bool fused = ffk_dct_wh_supported(dm) && (p->attn_impl & 4);   // opt-in: measured slower than separate passes
@@ -567,16 +638,16 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
     } else {
       P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 2 + 0) * TILE_BYTES;
       P.dst = sc.a_hi; P.dst_lo = sc.a_lo; P.side = side;
-      e = launch_pass(p, mq, mk, mv, P, st);
+      e = launch_pass(p, mq, mk, mv, o0h, o0l, P, st);
       if (e != cudaSuccess) return e;
       P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 1 + 0) * TILE_BYTES;
       P.dst = sc.b_hi; P.dst_lo = sc.b_lo;
-      e = launch_pass(p, m1h, m1l, m1l, P, st);
+      e = launch_pass(p, m1h, m1l, m1l, o1h, o1l, P, st);
       if (e != cudaSuccess) return e;
     }
     P.in_split = 1;
     P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 0 + 0) * TILE_BYTES; P.dst = nullptr;
-    e = launch_pass(p, m2h, m2l, m2l, P, st);
+    e = launch_pass(p, m2h, m2l, m2l, m2h, m2l, P, st);    // (no tensor stores in this mode)
     if (e != cudaSuccess) return e;
     dim3 lgrid((unsigned)dm.L[2], (unsigned)g);
     low_band_kernel<<<lgrid, CH * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
@@ -592,25 +663,27 @@ cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaS
   const FFDims& dm = p->dm;
   const int G = p->dct_group;
   const Scratch sc = carve(p);
-  CUtensorMap m_in, m_inl, mbh, mbl, mah, mal;
+  CUtensorMap m_in, m_inl, mbh, mbl, mah, mal, obh, obl, oah, oal, mout;
   if (!encode_grid_map(&m_in, sc.a_hi, dm, G, 0) || !encode_grid_map(&m_inl, sc.a_lo, dm, G, 0) ||
       !encode_grid_map(&mbh, sc.b_hi, dm, G, 1) ||
       !encode_grid_map(&mbl, sc.b_lo, dm, G, 1) || !encode_grid_map(&mah, sc.a_hi, dm, G, 2) ||
-      !encode_grid_map(&mal, sc.a_lo, dm, G, 2))
+      !encode_grid_map(&mal, sc.a_lo, dm, G, 2) || !encode_store_map(&obh, sc.b_hi, dm, G, 0) ||
+      !encode_store_map(&obl, sc.b_lo, dm, G, 0) || !encode_store_map(&oah, sc.a_hi, dm, G, 1) ||
+      !encode_store_map(&oal, sc.a_lo, dm, G, 1) || !encode_store_map(&mout, out, dm, dm.BH, 2))
     return cudaErrorInvalidValue;
   DctTcParams P{};
   P.dm = dm; P.status = p->buf.status; P.group = g; P.group_start = h0;
   P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 3 + 0) * TILE_BYTES;
   P.dst = sc.b_hi; P.dst_lo = sc.b_lo;
-  cudaError_t e = launch_pass(p, m_in, m_inl, m_inl, P, st);
+  cudaError_t e = launch_pass(p, m_in, m_inl, m_inl, obh, obl, P, st);
   if (e != cudaSuccess) return e;
   if (ffk_dct_wh_supported(dm) && (p->attn_impl & 4))
     return ffk_dct_wh_launch(p, 0, sc.b_hi, sc.b_lo, nullptr, h0, g, sc.ring, out, nullptr, nullptr, st);
   P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 4 + 0) * TILE_BYTES;
   P.dst = sc.a_hi; P.dst_lo = sc.a_lo;
-  e = launch_pass(p, mbh, mbl, mbl, P, st);
+  e = launch_pass(p, mbh, mbl, mbl, oah, oal, P, st);
   if (e != cudaSuccess) return e;
   P.mode = MODE_LAST; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 5 + 0) * TILE_BYTES;
   P.dst = (__nv_bfloat16*)out; P.dst_lo = nullptr;
-  return launch_pass(p, mah, mal, mal, P, st);
+  return launch_pass(p, mah, mal, mal, mout, mout, P, st);
 }
