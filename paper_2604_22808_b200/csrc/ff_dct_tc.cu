@@ -28,7 +28,7 @@
 //               from which the low band is computed at full precision
 //        MIDDLE hi/lo intermediate -> hi/lo intermediate
 //        SPLIT  intermediate -> band-major mid/high coefficient buffers (rank evaluated in
-//               registers) with the router's band energies accumulated from the fp32 accumulators
+//               registers) with the router's band energies accumulated from the stored (bf16) coefficients
 //        LAST   intermediate -> the caller's out tensor
 #include <cuda.h>
 
@@ -226,19 +226,23 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     const int a0 = seq ? j0 & (n - 1) : j0 >> lkf, l0 = seq ? j0 >> ln : j0 & (kf - 1);
     const int dw = P.axis == 2 ? a0 : l0, dh = P.axis == 2 ? l0 : (P.axis == 1 ? a0 : 0), dt = P.axis == 0 ? a0 : 0;
     const int Lhw = dm.L[1] * dm.L[2], Mhw = dm.M[1] * dm.M[2];
-    // lane k of a warp accumulates the energies of channels 32 q + k over the warp's rows
-    float em[4] = {0.f, 0.f, 0.f, 0.f}, eh[4] = {0.f, 0.f, 0.f, 0.f};
+    // (SPLIT) lane k of a warp accumulates the energies of channels 32 q + 2 (k % 16) + {0, 1} over the
+    // warp's rows of parity k / 16: ea = mid + high rows, em = mid rows
+    float ea[2][2] = {}, em[2][2] = {};                   // [chunk of the thread][channel of the pair]
     int e_sample = -1;
     unsigned it = 0;
     bool ok = true;
     auto flush_energy = [&]() {
       if (e_sample >= 0 && P.energy) {
 #pragma unroll
-        for (int q = q_lo; q < q_lo + 2; ++q) {
-          atomicAdd(P.energy + ((size_t)e_sample * 3 + 1) * CH + q * 32 + lane, (double)em[q]);
-          atomicAdd(P.energy + ((size_t)e_sample * 3 + 2) * CH + q * 32 + lane, (double)eh[q]);
-          em[q] = eh[q] = 0.f;
-        }
+        for (int qi = 0; qi < 2; ++qi)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int c = (q_lo + qi) * 32 + 2 * (lane & 15) + e;
+            atomicAdd(P.energy + ((size_t)e_sample * 3 + 1) * CH + c, (double)em[qi][e]);
+            atomicAdd(P.energy + ((size_t)e_sample * 3 + 2) * CH + c, (double)(ea[qi][e] - em[qi][e]));
+            ea[qi][e] = em[qi][e] = 0.f;
+          }
       }
     };
     for (int s = blockIdx.x; s < total_tiles && ok; s += gridDim.x, ++it) {
@@ -284,8 +288,10 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
         dst_hi[i] = (__nv_bfloat16*)__shfl_sync(0xffffffffu, (unsigned long long)row_hi, src);
       }
       const int out_slice = P.mode == MODE_LAST ? th : gi;
+      const unsigned nonlow_rows = __ballot_sync(0xffffffffu, band > 0), mid_rows = __ballot_sync(0xffffffffu, band == 1);
 #pragma unroll
-      for (int q = q_lo; q < q_lo + 2; ++q) {
+      for (int qi = 0; qi < 2; ++qi) {
+        const int q = q_lo + qi;
         uint32_t r[32];
         tmem_ld32(tm + lane_addr + ab * 128 + q * 32, r);
         tmem_wait_ld();
@@ -293,44 +299,6 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
 #pragma unroll
           for (int i = 0; i < 8; ++i)
             *(uint4*)(row_f32 + q * 32 + i * 4) = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
-        }
-        if (P.mode == MODE_SPLIT && P.energy) {
-          // Channel energies of this 32-channel chunk, summed over the warp's 32 rows with a halving
-          // butterfly (afterwards lane k holds the sum for channel 32 q + k): one butterfly for the
-          // mid + high rows together, a second one for the mid rows only where the warp has any;
-          // the high band's energy is the difference.
-          const bool any_mid = __any_sync(0xffffffffu, band == 1);
-          float sa[32], sm_[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float v = __uint_as_float(r[i]);
-            const float v2 = v * v;
-            sa[i] = band != 0 ? v2 : 0.f;
-            sm_[i] = band == 1 ? v2 : 0.f;
-          }
-#pragma unroll
-          for (int step = 16; step >= 1; step >>= 1) {
-            const bool upper = lane & step;
-#pragma unroll
-            for (int i = 0; i < step; ++i) {
-              const float keep = upper ? sa[i + step] : sa[i], send = upper ? sa[i] : sa[i + step];
-              sa[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
-            }
-          }
-          if (any_mid) {
-#pragma unroll
-            for (int step = 16; step >= 1; step >>= 1) {
-              const bool upper = lane & step;
-#pragma unroll
-              for (int i = 0; i < step; ++i) {
-                const float keep = upper ? sm_[i + step] : sm_[i], send = upper ? sm_[i] : sm_[i + step];
-                sm_[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
-              }
-            }
-            em[q] += sm_[0]; eh[q] += sa[0] - sm_[0];
-          } else {
-            eh[q] += sa[0];
-          }
         }
         {
           const bool want_lo = P.mode == MODE_FIRST || P.mode == MODE_MIDDLE;
@@ -372,6 +340,22 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
             }
           } else {
             __syncwarp();
+            if (P.energy) {
+              // Router statistics: channel energies of the staged (bf16) coefficients, summed down the
+              // columns of the warp's 32 x 32 block; a lane reads one channel pair of every other row.
+              const int par = lane >> 4, cp = lane & 15;
+              const unsigned nl = nonlow_rows >> par, md = mid_rows >> par;
+              float a0 = 0.f, a1 = 0.f, m0 = 0.f, m1 = 0.f;
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const uint32_t wd = *(const uint32_t*)(st_hi + (2 * i + par) * STG_PITCH + (((cp >> 2) ^ (i & 3)) << 4) + (cp & 3) * 4);
+                const float v0 = __uint_as_float(wd << 16), v1 = __uint_as_float(wd & 0xffff0000u);
+                const float s0 = v0 * v0, s1 = v1 * v1;
+                if ((nl >> (2 * i)) & 1) { a0 += s0; a1 += s1; }
+                if ((md >> (2 * i)) & 1) { m0 += s0; m1 += s1; }
+              }
+              ea[qi][0] += a0; ea[qi][1] += a1; em[qi][0] += m0; em[qi][1] += m1;
+            }
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const int rr = 8 * i + (lane >> 2), piece = lane & 3;      // row of the warp, 16-byte piece of its 64 bytes
