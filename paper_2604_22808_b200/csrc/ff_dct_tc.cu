@@ -289,12 +289,17 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
       }
       const int out_slice = P.mode == MODE_LAST ? th : gi;
       const unsigned nonlow_rows = __ballot_sync(0xffffffffu, band > 0), mid_rows = __ballot_sync(0xffffffffu, band == 1);
+      // both 32-channel chunks of the row at once; the accumulator buffer is free as soon as they are read
+      uint32_t rr2[2][32];
+      tmem_ld32(tm + lane_addr + ab * 128 + q_lo * 32, rr2[0]);
+      tmem_ld32(tm + lane_addr + ab * 128 + q_lo * 32 + 32, rr2[1]);
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(&sh.acc_empty[ab]);
 #pragma unroll
       for (int qi = 0; qi < 2; ++qi) {
         const int q = q_lo + qi;
-        uint32_t r[32];
-        tmem_ld32(tm + lane_addr + ab * 128 + q * 32, r);
-        tmem_wait_ld();
+        uint32_t (&r)[32] = rr2[qi];
         if (row_f32) {
 #pragma unroll
           for (int i = 0; i < 8; ++i)
@@ -365,8 +370,6 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
           }
         }
       }
-      tc_fence_before();
-      mbar_arrive(&sh.acc_empty[ab]);
     }
     if (P.mode == MODE_SPLIT) flush_energy();
     if (tma_out && lane == 0) bulk_wait0();
@@ -606,7 +609,6 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
       !encode_store_map(&o1l, sc.b_lo, dm, G, 1))
     return cudaErrorInvalidValue;
   const int total = 3 * dm.BH;
-  const bool fused = ffk_dct_wh_supported(dm) && (p->attn_impl & 4);   // opt-in: measured slower than separate passes
   DctTcParams P{};
   P.dm = dm; P.status = p->buf.status;
   P.spec_mid = (__nv_bfloat16*)p->buf.spec_mid; P.spec_high = (__nv_bfloat16*)p->buf.spec_high;
@@ -615,7 +617,7 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
     const int g = total - g0 < G ? total - g0 : G;
     P.group = g; P.group_start = g0;
     cudaError_t e;
-    if (fused) {
+    if ((p->attn_impl & 4) && ffk_dct_wh_usable(dm, g, p->sm_count)) {
       // w and h passes in one launch, the intermediate staying in L2
       e = ffk_dct_wh_launch(p, 1, Q, K, V, g0, g, sc.ring, sc.b_hi, sc.b_lo, side, st);
       if (e != cudaSuccess) return e;
@@ -661,7 +663,7 @@ cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaS
   P.dst = sc.b_hi; P.dst_lo = sc.b_lo;
   cudaError_t e = launch_pass(p, m_in, m_inl, m_inl, obh, obl, P, st);
   if (e != cudaSuccess) return e;
-  if (ffk_dct_wh_supported(dm) && (p->attn_impl & 4))
+  if ((p->attn_impl & 4) && ffk_dct_wh_usable(dm, g, p->sm_count))
     return ffk_dct_wh_launch(p, 0, sc.b_hi, sc.b_lo, nullptr, h0, g, sc.ring, out, nullptr, nullptr, st);
   P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 4 + 0) * TILE_BYTES;
   P.dst = sc.a_hi; P.dst_lo = sc.a_lo;

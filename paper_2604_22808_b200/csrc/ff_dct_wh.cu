@@ -12,6 +12,11 @@
 // ring slot it overwrites has been consumed; both conditions refer to earlier queue entries only,
 // so the earliest unfinished entry can always proceed.  Per-slab counters in global memory carry
 // the dependencies (one release per epilogue warp, acquire + cross-proxy fence before the TMA load).
+// An epilogue warp sends its rows out with tensor stores and releases a tile's counter only when
+// the stores have completed, which it checks after its next tile (so that the completion latency is
+// off the critical path); the launcher only fuses when no tile can depend on a release that is still
+// deferred in this way (lag * 2 * tiles-per-slab > grid + tiles-per-slab, lag not clamped).
+// Ring traffic carries an evict-last L2 policy, the streamed input and output evict-first.
 //
 // Tile math, precision (hi/lo split of matrix and intermediates) and the warp roles are those of
 // dct_tc_kernel: A = I kron Mat image (K-major), B = the TMA tile in place (MN-major), D in tensor
@@ -34,7 +39,7 @@ constexpr int STAGE_BYTES = 2 * TILE_BYTES;        // hi + lo
 constexpr int NSTAGE = 2;
 constexpr int NACC = 4;
 constexpr int WH_THREADS = 320;        // TMA warp, MMA warp, 8 epilogue warps
-constexpr int STG_PITCH = 64;                       // bytes per staged row piece; the 16-byte chunks are rotated by row/2 against bank conflicts
+constexpr int STG_PITCH = 64;                       // bytes per staged row piece (64-byte swizzle of the store maps)
 
 struct WhParams {
   FFDims dm;
@@ -57,7 +62,7 @@ struct WhShared {
   uint64_t full[NSTAGE], empty[NSTAGE], acc_full[NACC], acc_empty[NACC], img_full;
   uint32_t tmem_base;
   int abort_flag;
-  alignas(16) uint8_t stage[8][2][32 * STG_PITCH];
+  alignas(1024) uint8_t stage[8][2][32 * STG_PITCH];
 };
 
 struct WhTile {
@@ -82,11 +87,33 @@ __device__ __forceinline__ WhTile wh_decode(int idx, int tps, int S, int D) {
 }
 
 __device__ __forceinline__ void tma_load_5d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2,
-                                            int c3, int c4) {
+                                            int c3, int c4, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-      ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;"
+      ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(policy)
       : "memory");
+}
+
+__device__ __forceinline__ void tma_store_5d(const void* smem_src, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                             int c4, uint64_t policy) {
+  asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3, %4, %5, %6}], [%1], %7;"
+               ::"l"((uint64_t)map), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(policy)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait2() { asm volatile("cp.async.bulk.wait_group 2;" ::: "memory"); }
+
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
 }
 
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
@@ -112,10 +139,14 @@ __device__ __forceinline__ bool wait_counter(const int* cnt, int target, volatil
 
 // m0..m2: first-pass input (forward: Q, K, V; inverse: hi grid, lo grid, unused).
 // m3, m4: the ring (hi, lo) with the box of the second pass.
+// s_rh, s_rl: store maps of the ring (box of an epilogue warp of the first pass); s_oh, s_ol: store
+// maps of the result (box of an epilogue warp of the second pass; the inverse has no lo result).
 __global__ void __launch_bounds__(WH_THREADS, 1)
 dct_wh_kernel(const __grid_constant__ CUtensorMap m0, const __grid_constant__ CUtensorMap m1,
               const __grid_constant__ CUtensorMap m2, const __grid_constant__ CUtensorMap m3,
-              const __grid_constant__ CUtensorMap m4, const WhParams P) {
+              const __grid_constant__ CUtensorMap m4, const __grid_constant__ CUtensorMap s_rh,
+              const __grid_constant__ CUtensorMap s_rl, const __grid_constant__ CUtensorMap s_oh,
+              const __grid_constant__ CUtensorMap s_ol, const WhParams P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sData = smem;                                  // NSTAGE x 64 KB
@@ -148,6 +179,7 @@ dct_wh_kernel(const __grid_constant__ CUtensorMap m0, const __grid_constant__ CU
       mbar_arrive_expect_tx(&sh.img_full, 2 * TILE_BYTES);
       bulk_load(sHi, P.image, TILE_BYTES, &sh.img_full);
       bulk_load(sLo, P.image + TILE_BYTES, TILE_BYTES, &sh.img_full);
+      const uint64_t pol_ring = policy_evict_last(), pol_stream = policy_evict_first();
       unsigned it = 0;
       bool ok = true;
       for (int idx = blockIdx.x; idx < total && ok; idx += gridDim.x, ++it) {
@@ -155,6 +187,7 @@ dct_wh_kernel(const __grid_constant__ CUtensorMap m0, const __grid_constant__ CU
         const int gi = x.slab / dm.T, t = x.slab % dm.T, slot = x.slab % P.ring;
         const bool along_w = (x.second == 0) == (P.forward != 0);
         const bool split = x.second || !P.forward;
+        const uint64_t pol = x.second ? pol_ring : pol_stream;
         // dependencies: the slab's first pass is stored / the ring slot has been consumed
         if (x.second) ok = wait_counter(P.cnt_a + x.slab, 8 * tps, abort_flag);
         else if (x.slab >= P.ring) ok = wait_counter(P.cnt_b + x.slab - P.ring, 8 * tps, abort_flag);
@@ -173,21 +206,21 @@ dct_wh_kernel(const __grid_constant__ CUtensorMap m0, const __grid_constant__ CU
         mbar_arrive_expect_tx(&sh.full[st], split ? STAGE_BYTES : TILE_BYTES);
         if (along_w) {                                    // one box: kf whole lines along w
           const int h0 = x.u * kf;
-          tma_load_5d(dst, mhi, &sh.full[st], 0, 0, h0, tc, slice);
-          tma_load_5d(dst + HALF_BYTES, mhi, &sh.full[st], 64, 0, h0, tc, slice);
+          tma_load_5d(dst, mhi, &sh.full[st], 0, 0, h0, tc, slice, pol);
+          tma_load_5d(dst + HALF_BYTES, mhi, &sh.full[st], 64, 0, h0, tc, slice, pol);
           if (split) {
-            tma_load_5d(dst + TILE_BYTES, mlo, &sh.full[st], 0, 0, h0, tc, slice);
-            tma_load_5d(dst + TILE_BYTES + HALF_BYTES, mlo, &sh.full[st], 64, 0, h0, tc, slice);
+            tma_load_5d(dst + TILE_BYTES, mlo, &sh.full[st], 0, 0, h0, tc, slice, pol);
+            tma_load_5d(dst + TILE_BYTES + HALF_BYTES, mlo, &sh.full[st], 64, 0, h0, tc, slice, pol);
           }
         } else {                                          // kf boxes: one line along h each
           const int w0 = x.u * kf;
           for (int l = 0; l < kf; ++l) {
             const int o = l * n * 128;
-            tma_load_5d(dst + o, mhi, &sh.full[st], 0, w0 + l, 0, tc, slice);
-            tma_load_5d(dst + HALF_BYTES + o, mhi, &sh.full[st], 64, w0 + l, 0, tc, slice);
+            tma_load_5d(dst + o, mhi, &sh.full[st], 0, w0 + l, 0, tc, slice, pol);
+            tma_load_5d(dst + HALF_BYTES + o, mhi, &sh.full[st], 64, w0 + l, 0, tc, slice, pol);
             if (split) {
-              tma_load_5d(dst + TILE_BYTES + o, mlo, &sh.full[st], 0, w0 + l, 0, tc, slice);
-              tma_load_5d(dst + TILE_BYTES + HALF_BYTES + o, mlo, &sh.full[st], 64, w0 + l, 0, tc, slice);
+              tma_load_5d(dst + TILE_BYTES + o, mlo, &sh.full[st], 0, w0 + l, 0, tc, slice, pol);
+              tma_load_5d(dst + TILE_BYTES + HALF_BYTES + o, mlo, &sh.full[st], 64, w0 + l, 0, tc, slice, pol);
             }
           }
         }
@@ -229,6 +262,8 @@ dct_wh_kernel(const __grid_constant__ CUtensorMap m0, const __grid_constant__ CU
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const int ew = warp - 2;                              // epilogue warp 0..7: warps 0-3 take channels 0..63, 4-7 channels 64..127
     const int q_lo = (ew >> 2) * 2;
+    const uint64_t pol_ring = policy_evict_last(), pol_stream = policy_evict_first();
+    int* pending = nullptr;                               // counter of the tile whose stores are still in flight
     unsigned it = 0;
     bool ok = true;
     for (int idx = blockIdx.x; idx < total && ok; idx += gridDim.x, ++it) {
@@ -239,28 +274,20 @@ dct_wh_kernel(const __grid_constant__ CUtensorMap m0, const __grid_constant__ CU
       ok = __all_sync(0xffffffffu, mbar_wait(&sh.acc_full[ab], (it / NACC) & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
-      // grid position (h, w) of this thread's output row
+      // grid position (h, w) of this thread's output row (for the fp32 side rows) and of the warp's
+      // first row: the warp's 32 rows are 32 consecutive positions along the pass axis
       const int h = along_w ? x.u * kf + l : a;
-      const int w = along_w ? a : x.u * kf + l;
-      __nv_bfloat16* row_hi; __nv_bfloat16* row_lo = nullptr; float* row_f32 = nullptr;
-      if (!x.second) {                                     // first pass -> ring slot
-        const size_t o = (((size_t)slot * n + h) * n + w) * CH;
-        row_hi = P.ring_hi + o; row_lo = P.ring_lo + o;
-        if (P.forward && a < dm.L[2]) row_f32 = P.side + ((((size_t)gi * dm.T + t) * dm.H + h) * dm.L[2] + a) * CH;
-      } else if (P.forward) {                              // second pass -> hi/lo grid of the group
-        const size_t o = ((((size_t)gi * dm.T + t) * n + h) * n + w) * CH;
-        row_hi = P.out_hi + o; row_lo = P.out_lo + o;
-      } else {                                             // second pass of the inverse -> out tensor
-        row_hi = P.out_hi + (((((size_t)(P.group_start + gi)) * dm.T + t) * n + h) * n + w) * CH;
-      }
-      // lane L stores for rows 8 i + L/4 of its warp: fetch those rows' destinations
-      __nv_bfloat16* dst_hi[4]; __nv_bfloat16* dst_lo[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int src = 8 * i + (lane >> 2);
-        dst_hi[i] = (__nv_bfloat16*)__shfl_sync(0xffffffffu, (unsigned long long)row_hi, src);
-        dst_lo[i] = (__nv_bfloat16*)__shfl_sync(0xffffffffu, (unsigned long long)row_lo, src);
-      }
+      const int j0 = quarter * 32, a0 = j0 & (n - 1), l0 = j0 >> ln;
+      const int bh0 = along_w ? x.u * kf + l0 : a0, bw0 = along_w ? a0 : x.u * kf + l0;
+      float* row_f32 = nullptr;
+      if (!x.second && P.forward && a < dm.L[2]) row_f32 = P.side + ((((size_t)gi * dm.T + t) * dm.H + h) * dm.L[2] + a) * CH;
+      const CUtensorMap* mo_hi; const CUtensorMap* mo_lo;
+      int c3, c4;
+      uint64_t pol;
+      bool want_lo = true;
+      if (!x.second) { mo_hi = &s_rh; mo_lo = &s_rl; c3 = slot; c4 = 0; pol = pol_ring; }
+      else if (P.forward) { mo_hi = &s_oh; mo_lo = &s_ol; c3 = t; c4 = gi; pol = pol_stream; }
+      else { mo_hi = &s_oh; mo_lo = &s_ol; c3 = t; c4 = P.group_start + gi; pol = pol_stream; want_lo = false; }
 #pragma unroll
       for (int q = q_lo; q < q_lo + 2; ++q) {
         uint32_t r[32];
@@ -274,35 +301,57 @@ dct_wh_kernel(const __grid_constant__ CUtensorMap m0, const __grid_constant__ CU
         uint32_t hi[16], lo[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          const float v0 = __uint_as_float(r[2 * i]), v1 = __uint_as_float(r[2 * i + 1]);
-          const __nv_bfloat162 hp = __floats2bfloat162_rn(v0, v1);
+          const __nv_bfloat162 hp = __floats2bfloat162_rn(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
           hi[i] = *(const uint32_t*)&hp;
-          const __nv_bfloat162 lp = __floats2bfloat162_rn(v0 - __uint_as_float(hi[i] << 16), v1 - __uint_as_float(hi[i] & 0xffff0000u));
-          lo[i] = *(const uint32_t*)&lp;
+        }
+        if (want_lo) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const __nv_bfloat162 lp = __floats2bfloat162_rn(__uint_as_float(r[2 * i]) - __uint_as_float(hi[i] << 16),
+                                                           __uint_as_float(r[2 * i + 1]) - __uint_as_float(hi[i] & 0xffff0000u));
+            lo[i] = *(const uint32_t*)&lp;
+          }
         }
         uint8_t* st_hi = sh.stage[ew][0];
         uint8_t* st_lo = sh.stage[ew][1];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          *(uint4*)(st_hi + lane * STG_PITCH + (((i + (lane >> 1)) & 3) << 4)) = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
-          *(uint4*)(st_lo + lane * STG_PITCH + (((i + (lane >> 1)) & 3) << 4)) = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
-        }
+        // the previous store of this warp must have read the staging area
+        if (lane == 0) bulk_wait_read0();
         __syncwarp();
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int rr = 8 * i + (lane >> 2), piece = lane & 3;
-          *(uint4*)(dst_hi[i] + q * 32 + piece * 8) = *(const uint4*)(st_hi + rr * STG_PITCH + (((piece + (rr >> 1)) & 3) << 4));
-          if (dst_lo[i]) *(uint4*)(dst_lo[i] + q * 32 + piece * 8) = *(const uint4*)(st_lo + rr * STG_PITCH + (((piece + (rr >> 1)) & 3) << 4));
+          *(uint4*)(st_hi + lane * STG_PITCH + ((i ^ ((lane >> 1) & 3)) << 4)) = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
+          if (want_lo)
+            *(uint4*)(st_lo + lane * STG_PITCH + ((i ^ ((lane >> 1) & 3)) << 4)) = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
         }
+        fence_proxy_async();
         __syncwarp();
+        if (lane == 0) {
+          tma_store_5d(st_hi, mo_hi, q * 32, bw0, bh0, c3, c4, pol);
+          if (want_lo) tma_store_5d(st_lo, mo_lo, q * 32, bw0, bh0, c3, c4, pol);
+          bulk_commit();
+        }
       }
       tc_fence_before();
       mbar_arrive(&sh.acc_empty[ab]);
-      // publish: this warp's rows of the tile are stored (release after the whole warp's stores)
-      __syncwarp();
+      // publish the PREVIOUS tile of this warp: its two store groups are complete once at most this
+      // tile's two are pending (release after completion; the reader acquires the counter and fences
+      // towards the async proxy before its TMA load)
       if (lane == 0) {
+        if (pending) {
+          bulk_wait2();
+          asm volatile("fence.proxy.async;" ::: "memory");
+          __threadfence();
+          atomicAdd(pending, 1);
+        }
+        pending = (x.second ? P.cnt_b : P.cnt_a) + x.slab;
+      }
+    }
+    if (lane == 0) {
+      bulk_wait0();
+      if (pending) {
+        asm volatile("fence.proxy.async;" ::: "memory");
         __threadfence();
-        atomicAdd((x.second ? P.cnt_b : P.cnt_a) + x.slab, 1);
+        atomicAdd(pending, 1);
       }
     }
   }
@@ -345,12 +394,43 @@ bool encode_wh_map(CUtensorMap* map, const void* base, int n, int T, int slices,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Store map: the box of one epilogue warp, 32 channels of 32 consecutive positions along w
+// (along_w) or along h, 64-byte swizzle.
+bool encode_wh_store_map(CUtensorMap* map, const void* base, int n, int T, int slices, bool along_w) {
+  static EncodeTiledFn enc = nullptr;
+  if (!enc) {
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", (void**)&enc, cudaEnableDefault, &qr) != cudaSuccess || !enc)
+      return false;
+  }
+  cuuint64_t dims[5] = {(cuuint64_t)CH, (cuuint64_t)n, (cuuint64_t)n, (cuuint64_t)T, (cuuint64_t)slices};
+  cuuint64_t strides[4] = {(cuuint64_t)CH * 2, (cuuint64_t)n * CH * 2, (cuuint64_t)n * n * CH * 2,
+                           (cuuint64_t)T * n * n * CH * 2};
+  cuuint32_t box[5] = {32, 1, 1, 1, 1};
+  box[along_w ? 1 : 2] = 32;
+  cuuint32_t es[5] = {1, 1, 1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, es,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
-// bf16, head_dim 128, square h x w slabs whose side is a power of two in 16..128.
+// bf16, head_dim 128, square h x w slabs whose side is a power of two in 32..128 (an epilogue
+// warp's 32 rows must lie on one line).
 bool ffk_dct_wh_supported(const FFDims& dm) {
   const int n = dm.W;
-  return !dm.fp32 && dm.d == CH && dm.H == dm.W && (n == 16 || n == 32 || n == 64 || n == 128);
+  return !dm.fp32 && dm.d == CH && dm.H == dm.W && (n == 32 || n == 64 || n == 128);
+}
+
+// Can a group of `g` tensor-heads run fused on a grid of `sm_count` CTAs?  The second pass must
+// trail by the full lag, and no tile may wait for a counter whose release is deferred behind it.
+bool ffk_dct_wh_usable(const FFDims& dm, int g, int sm_count) {
+  if (!ffk_dct_wh_supported(dm)) return false;
+  int ring, lag;
+  ffk_dct_wh_shape(dm, &ring, &lag);
+  const int tps = dm.W * dm.W / TILE_ROWS;
+  return g * dm.T >= lag && (long long)lag * 2 * tps > sm_count + tps;
 }
 
 // Ring depth and lag: the second pass trails the first by about three rounds of the grid, and the
@@ -392,23 +472,28 @@ cudaError_t ffk_dct_wh_launch(ff_plan* p, int forward, const void* src0, const v
   P.image = p->dct_images + (size_t)(2 * ((forward ? 0 : 3) + 2)) * TILE_BYTES;
   cudaError_t e = cudaMemsetAsync(P.cnt_a, 0, (size_t)2 * S * sizeof(int), st);
   if (e != cudaSuccess) return e;
-  CUtensorMap m0, m1, m2, m3, m4;
+  if (!ffk_dct_wh_usable(dm, g, p->sm_count)) return cudaErrorInvalidValue;
+  CUtensorMap m0, m1, m2, m3, m4, s_rh, s_rl, s_oh, s_ol;
   bool ok;
   if (forward)
     ok = encode_wh_map(&m0, src0, n, dm.T, dm.BH, true) && encode_wh_map(&m1, src1, n, dm.T, dm.BH, true) &&
          encode_wh_map(&m2, src2, n, dm.T, dm.BH, true) && encode_wh_map(&m3, P.ring_hi, n, P.ring, 1, false) &&
-         encode_wh_map(&m4, P.ring_lo, n, P.ring, 1, false);
+         encode_wh_map(&m4, P.ring_lo, n, P.ring, 1, false) &&
+         encode_wh_store_map(&s_rh, P.ring_hi, n, P.ring, 1, true) && encode_wh_store_map(&s_rl, P.ring_lo, n, P.ring, 1, true) &&
+         encode_wh_store_map(&s_oh, out_hi, n, dm.T, g, false) && encode_wh_store_map(&s_ol, out_lo, n, dm.T, g, false);
   else
     ok = encode_wh_map(&m0, src0, n, dm.T, g, false) && encode_wh_map(&m1, src1, n, dm.T, g, false) &&
          encode_wh_map(&m2, src1, n, dm.T, g, false) && encode_wh_map(&m3, P.ring_hi, n, P.ring, 1, true) &&
-         encode_wh_map(&m4, P.ring_lo, n, P.ring, 1, true);
+         encode_wh_map(&m4, P.ring_lo, n, P.ring, 1, true) &&
+         encode_wh_store_map(&s_rh, P.ring_hi, n, P.ring, 1, false) && encode_wh_store_map(&s_rl, P.ring_lo, n, P.ring, 1, false) &&
+         encode_wh_store_map(&s_oh, out_hi, n, dm.T, dm.BH, true) && encode_wh_store_map(&s_ol, out_hi, n, dm.T, dm.BH, true);
   if (!ok) return cudaErrorInvalidValue;
   const size_t smem = NSTAGE * STAGE_BYTES + 2 * TILE_BYTES + sizeof(WhShared) + 1024;
   e = cudaFuncSetAttribute(dct_wh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int total = 2 * S * (n * n / TILE_ROWS);
   const int grid = total < p->sm_count ? total : p->sm_count;
-  dct_wh_kernel<<<grid, WH_THREADS, smem, st>>>(m0, m1, m2, m3, m4, P);
+  dct_wh_kernel<<<grid, WH_THREADS, smem, st>>>(m0, m1, m2, m3, m4, s_rh, s_rl, s_oh, s_ol, P);
   p->launches += 1;
   return cudaGetLastError();
 }

@@ -140,6 +140,8 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
 cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaStream_t st);
 // ---- fused w/h passes (ff_dct_wh.cu) ---------------------------------------------------------------
 bool ffk_dct_wh_supported(const FFDims& dm);
+void ffk_dct_wh_shape(const FFDims& dm, int* ring, int* lag);
+bool ffk_dct_wh_usable(const FFDims& dm, int g, int sm_count);
 size_t ffk_dct_wh_scratch_bytes(const FFDims& dm, int group);
 cudaError_t ffk_dct_wh_launch(ff_plan* p, int forward, const void* src0, const void* src1, const void* src2, int g0, int g,
                               void* ring, void* out_hi, void* out_lo, float* side, cudaStream_t st);
