@@ -394,16 +394,19 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
 // One CTA per (tensor-head, k_w) computes every (k_t, k_h) of the low box, in chunks of 8 x 8, so the
 // side buffer is read once per chunk pair; thread = (t group, channel); the t groups are combined
 // through shared memory.  Also accumulates the low band's energy.
-constexpr int LOW_CH = 8;        // k_t and k_h chunk
+constexpr int LOW_CH = 8;        // k_h chunk
 constexpr int LOW_TG = 4;
 
+// LOW_CT = k_t chunk: the smallest of 2, 4, 8 that covers L_t keeps the accumulators (and with them
+// the registers per thread) small, so that more CTAs are resident and more loads in flight.
+template <int LOW_CT>
 __global__ void __launch_bounds__(CH * LOW_TG) low_band_kernel(const float* side, const float* CT, const float* CHm,
                                                                float* spec_low, double* energy, FFDims dm, int group_start) {
   const int kw = blockIdx.x;
   const int gi = blockIdx.y, th = group_start + gi;
   const int c = threadIdx.x % CH, tg = threadIdx.x / CH;
   __shared__ float ch_rows[LOW_CH][128];          // C_H rows of the current k_h chunk
-  __shared__ float red[LOW_CH * LOW_CH][CH];
+  __shared__ float red[LOW_CT * LOW_CH][CH];
   float e = 0.f;
   for (int kh0 = 0; kh0 < dm.L[1]; kh0 += LOW_CH) {
     __syncthreads();
@@ -411,12 +414,12 @@ __global__ void __launch_bounds__(CH * LOW_TG) low_band_kernel(const float* side
       const int q = i / dm.H, h = i % dm.H;
       ch_rows[q][h] = kh0 + q < dm.L[1] ? CHm[(size_t)(kh0 + q) * dm.H + h] : 0.f;
     }
-    for (int kt0 = 0; kt0 < dm.L[0]; kt0 += LOW_CH) {
-      for (int i = threadIdx.x; i < LOW_CH * LOW_CH * CH; i += CH * LOW_TG) red[i / CH][i % CH] = 0.f;
+    for (int kt0 = 0; kt0 < dm.L[0]; kt0 += LOW_CT) {
+      for (int i = threadIdx.x; i < LOW_CT * LOW_CH * CH; i += CH * LOW_TG) red[i / CH][i % CH] = 0.f;
       __syncthreads();
-      float acc[LOW_CH][LOW_CH];                    // [k_t][k_h]
+      float acc[LOW_CT][LOW_CH];                    // [k_t][k_h]
 #pragma unroll
-      for (int i = 0; i < LOW_CH; ++i)
+      for (int i = 0; i < LOW_CT; ++i)
 #pragma unroll
         for (int q = 0; q < LOW_CH; ++q) acc[i][q] = 0.f;
       for (int t = tg; t < dm.T; t += LOW_TG) {
@@ -424,25 +427,31 @@ __global__ void __launch_bounds__(CH * LOW_TG) low_band_kernel(const float* side
         float s[LOW_CH];
 #pragma unroll
         for (int q = 0; q < LOW_CH; ++q) s[q] = 0.f;
-        for (int h = 0; h < dm.H; ++h) {
-          const float x = col[(size_t)h * dm.L[2] * CH];
+        const size_t hs = (size_t)dm.L[2] * CH;
+        constexpr int NB = LOW_CT <= 4 ? 16 : 8;      // loads in flight (axis lengths are multiples of 16)
+        for (int h0 = 0; h0 < dm.H; h0 += NB) {
+          float x[NB];
 #pragma unroll
-          for (int q = 0; q < LOW_CH; ++q) s[q] = fmaf(ch_rows[q][h], x, s[q]);
+          for (int u = 0; u < NB; ++u) x[u] = __ldg(col + (size_t)(h0 + u) * hs);
+#pragma unroll
+          for (int u = 0; u < NB; ++u)
+#pragma unroll
+            for (int q = 0; q < LOW_CH; ++q) s[q] = fmaf(ch_rows[q][h0 + u], x[u], s[q]);
         }
 #pragma unroll
-        for (int i = 0; i < LOW_CH; ++i) {
+        for (int i = 0; i < LOW_CT; ++i) {
           const float ct = kt0 + i < dm.L[0] ? CT[(size_t)(kt0 + i) * dm.T + t] : 0.f;
 #pragma unroll
           for (int q = 0; q < LOW_CH; ++q) acc[i][q] = fmaf(ct, s[q], acc[i][q]);
         }
       }
 #pragma unroll
-      for (int i = 0; i < LOW_CH; ++i)
+      for (int i = 0; i < LOW_CT; ++i)
 #pragma unroll
         for (int q = 0; q < LOW_CH; ++q)
           if (kt0 + i < dm.L[0] && kh0 + q < dm.L[1]) atomicAdd(&red[i * LOW_CH + q][c], acc[i][q]);
       __syncthreads();
-      for (int o = tg; o < LOW_CH * LOW_CH; o += LOW_TG) {
+      for (int o = tg; o < LOW_CT * LOW_CH; o += LOW_TG) {
         const int i = o / LOW_CH, q = o % LOW_CH;
         if (kt0 + i >= dm.L[0] || kh0 + q >= dm.L[1]) continue;
         const long long rank = ((long long)(kt0 + i) * dm.L[1] + kh0 + q) * dm.L[2] + kw;
@@ -636,7 +645,9 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
     e = launch_pass(p, m2h, m2l, m2l, m2h, m2l, P, st);    // (no tensor stores in this mode)
     if (e != cudaSuccess) return e;
     dim3 lgrid((unsigned)dm.L[2], (unsigned)g);
-    low_band_kernel<<<lgrid, CH * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
+    if (dm.L[0] <= 2) low_band_kernel<2><<<lgrid, CH * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
+    else if (dm.L[0] <= 4) low_band_kernel<4><<<lgrid, CH * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
+    else low_band_kernel<8><<<lgrid, CH * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
     p->launches += 1;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;

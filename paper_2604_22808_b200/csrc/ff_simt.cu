@@ -386,14 +386,14 @@ __global__ void __launch_bounds__(SUM_THREADS) summary_partial_kernel(FFBuffers 
   if (rsub < nrs) {
     long long p = r0 + rsub;
     if (!v.f32 && sizeof(ST) == 2) {
-      // bf16 rows, four rows in flight per thread
+      // bf16 rows, eight rows in flight per thread
       const __nv_bfloat16* base = (const __nv_bfloat16*)v.st + vec * 8;
-      for (; p + 3 * nrs < r1; p += 4 * nrs) {
-        uint4 x[4];
+      for (; p + 7 * nrs < r1; p += 8 * nrs) {
+        uint4 x[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) x[u] = *(const uint4*)(base + (size_t)(p + u * nrs) * d);
+        for (int u = 0; u < 8; ++u) x[u] = __ldcs((const uint4*)(base + (size_t)(p + u * nrs) * d));
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
           const uint32_t w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
@@ -624,9 +624,9 @@ cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st) {
   const FFDims& dm = p->dm;
   cudaError_t e = cudaMemsetAsync(p->buf.summary, 0, (size_t)dm.BH * 3 * dm.m * dm.d * sizeof(float), st);
   if (e != cudaSuccess) return e;
-  // split every segment so that each CTA reads about 256 rows of the longest band
+  // split every segment so that each CTA reads about 1024 rows of the longest band
   long long longest = dm.Nhigh > dm.Nmid ? dm.Nhigh : dm.Nmid;
-  int split = (int)((longest / dm.m + 255) / 256);
+  int split = (int)((longest / dm.m + 1023) / 1024);
   if (split < 1) split = 1;
   if (split > 64) split = 64;
   dim3 pgrid((unsigned)(dm.m * split), 3, (unsigned)dm.BH), fgrid((unsigned)dm.m, 3, (unsigned)dm.BH);
