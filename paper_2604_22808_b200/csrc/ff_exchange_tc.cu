@@ -5,13 +5,14 @@
 //
 // A CTA owns a contiguous run of (head, band, 128-rank tile) items, so the summary tokens of a head
 // are re-staged only a few times per CTA.
-// Two CTAs share an SM (256 tensor-memory columns each), which overlaps one tile's softmax and
-// stores with the other's MMAs and loads.  Per tile:
+// Two CTAs share an SM (256 tensor-memory columns each).  Inside a CTA the softmax warps work on
+// tile n + 1 while the store warps finish tile n.  Per tile:
 //   TMA     the 128 band tokens (operator output where the head's mask has the band, V~ otherwise)
 //   MMA 1   S[128 x 3m] = Y Z^T against all 3m summaries of the head (own band masked in the softmax)
 //   softmax one token per thread (row = TMEM lane); normalised P written back to TMEM as bf16 hi + lo
 //   MMA 2   D[128 x 128] = P Z  (A = P from tensor memory, B = the same Z image read MN-major)
-//   store   Y + D as a bf16 hi/lo pair, one 256-byte grid row per thread
+//   store   Y + D as a bf16 hi/lo pair; a thread owns a token, the warp stages 32 channels of its 32
+//           tokens in shared memory and four lanes then write a token's 64 contiguous bytes
 // Z and P are split into bf16 hi + lo parts (Y is exact bf16), so the logits and the update carry
 // about 16 bits: the summary logits of a band with large low-frequency content reach O(100).
 // The low band (fp32, a few hundred tokens) is handled by the generic kernel.
@@ -28,7 +29,7 @@ constexpr int XT = 128;                 // tokens per tile
 constexpr int XD = 128;                 // head_dim
 constexpr int X_TILE_BYTES = XT * XD * 2;
 constexpr int X_HALF = X_TILE_BYTES / 2;
-constexpr int X_THREADS = 192;
+constexpr int X_THREADS = 320;           // TMA warp, MMA warp, 4 softmax warps, 4 store warps
 
 struct XParams {
   FFDims dm;
@@ -44,10 +45,14 @@ struct XParams {
   int* status;
 };
 
+constexpr int X_STG_PITCH = 64;         // bytes per staged row piece (32 channels)
+
 struct XShared {
   uint64_t y_full[2], y_empty[2], z_ready, s_full, p_full, d_full, d_empty;
   uint32_t tmem_base;
   int abort_flag;
+  // per softmax warp: 32 rows x 64 bytes of hi and of lo (16-byte chunks XOR-swizzled with row / 2)
+  alignas(16) uint8_t stage[4][2][32 * X_STG_PITCH];
 };
 
 struct XItem { int bh, band, tile; };
@@ -68,6 +73,8 @@ __device__ __forceinline__ XItem x_decode(const FFDims& dm, int h0, int it, int 
   return x;
 }
 
+// NK32 = 32-key chunks of the score row that are in use (3m <= 32 NK32).
+template <int NK32>
 __global__ void __launch_bounds__(X_THREADS, 2)
 exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_constant__ CUtensorMap map_v_mid,
                    const __grid_constant__ CUtensorMap map_y_high, const __grid_constant__ CUtensorMap map_v_high,
@@ -160,7 +167,8 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         umma_commit(&sh.d_full);
       }
     }
-  } else {
+  } else if (warp < 6) {
+    // ------------------------------------------------------------------ softmax warps
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const int tid = row;                                  // 0..127 among the softmax threads
@@ -173,8 +181,12 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       if (x.bh != prev_bh) {
         // Stage the head's 3m summaries as two bf16 images (hi, lo) in the operand layout: row = key,
         // 64 channels per 128-byte row, 16-byte chunks XOR-swizzled with the row.  Rows >= 3m are zero.
-        // Every MMA of the previous tile has completed (its D was read before this point).
+        // The MMAs of the previous tile, which read the old images, must have completed.
         prev_bh = x.bh;
+        if (n >= 1) {
+          ok = __all_sync(0xffffffffu, mbar_wait(&sh.d_full, (n - 1) & 1, abort_flag));
+          if (!ok) break;
+        }
         const float* S = P.summary + (size_t)x.bh * 3 * m * XD;
         for (int idx = tid; idx < nk * XD; idx += 128) {
           const int j = idx >> 7, c = idx & 127;
@@ -189,42 +201,37 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         fence_proxy_async();
         mbar_arrive(&sh.z_ready);
       }
-      const int slot = n % YB;
-      const long long n_band = x.band == 1 ? dm.Nmid : dm.Nhigh;
-      const long long p = (long long)x.tile * XT + row;
       // ---- softmax over the 2m summaries of the other bands
       ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full, n & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
       const int own0 = x.band * m, own1 = own0 + m;       // this band's own summaries are not attended
       // all scores of the row into registers (they are overwritten by P below)
-      uint32_t sc[96];
+      uint32_t sc[NK32 * 32];
 #pragma unroll
-      for (int c3 = 0; c3 < 3; ++c3) {
-        if (c3 * 32 < nk) {
-          uint32_t r[32];
-          tmem_ld32(tmem + lane_addr + c3 * 32, r);
-          tmem_wait_ld();
+      for (int c3 = 0; c3 < NK32; ++c3) {
+        uint32_t r[32];
+        tmem_ld32(tmem + lane_addr + c3 * 32, r);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) sc[c3 * 32 + i] = r[i];
-        }
+        for (int i = 0; i < 32; ++i) sc[c3 * 32 + i] = r[i];
       }
-      float mx = -INFINITY;
+      tmem_wait_ld();
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int j = 0; j < 96; ++j)
-        if (j < 3 * m && (j < own0 || j >= own1)) mx = fmaxf(mx, __uint_as_float(sc[j]));
-      const float mb = mx * sl2;
-      float den = 0.f;
+      for (int j = 0; j < NK32 * 32; ++j)
+        if (j < 3 * m && (j < own0 || j >= own1)) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(sc[j]));
+      const float mb = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
+      float den4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int j = 0; j < 96; ++j) {
+      for (int j = 0; j < NK32 * 32; ++j) {
         float pv = 0.f;
         if (j < 3 * m && (j < own0 || j >= own1)) pv = ex2f_approx(fmaf(__uint_as_float(sc[j]), sl2, -mb));
-        den += pv;
+        den4[j & 3] += pv;
         sc[j] = __float_as_uint(pv);
       }
-      const float inv = 1.f / den;
+      const float inv = 1.f / ((den4[0] + den4[1]) + (den4[2] + den4[3]));
 #pragma unroll
-      for (int c3 = 0; c3 < 3; ++c3) {
+      for (int c3 = 0; c3 < NK32; ++c3) {
         if (c3 * 32 < nk) {
           uint32_t ph[16], pl[16];
 #pragma unroll
@@ -242,40 +249,70 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&sh.p_full);
+    }
+  } else {
+    // ------------------------------------------------------------------ store warps
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    bool ok = true;
+    int n = 0;
+    for (int it = it0; it < it1 && ok; ++it, ++n) {
+      const XItem x = x_decode(dm, P.h0, it, tm_tiles, th_tiles);
+      const int slot = n % YB;
+      const long long n_band = x.band == 1 ? dm.Nmid : dm.Nhigh;
+      const long long p = (long long)x.tile * XT + row;
       // ---- residual add and store
       ok = __all_sync(0xffffffffu, mbar_wait(&sh.d_full, n & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
       const bool valid = p < n_band;
-      const int f = valid ? (x.band == 1 ? P.pos_mid[p] : P.pos_high[p]) : 0;
-      const size_t o = ((size_t)(x.bh - P.h0) * dm.N + f) * XD;
+      const int f = valid ? (x.band == 1 ? P.pos_mid[p] : P.pos_high[p]) : -1;
+      // lane L stores for rows 8 i + L/4 of its warp: fetch those rows' grid positions
+      int fpos[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) fpos[i] = __shfl_sync(0xffffffffu, f, 8 * i + (lane >> 2));
+      const size_t obase = (size_t)(x.bh - P.h0) * dm.N * XD;
       const uint8_t* yrow = sY + slot * X_TILE_BYTES + row * 128;
+      uint8_t* st_hi = sh.stage[quarter][0];
+      uint8_t* st_lo = sh.stage[quarter][1];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         uint32_t r[32];
         tmem_ld32(tmem + lane_addr + 128 + q * 32, r);
         tmem_wait_ld();
-        if (valid) {
 #pragma unroll
-          for (int v4 = 0; v4 < 4; ++v4) {
-            // channels 32q + 8v4 .. +7 of this token: one 16-byte chunk of the swizzled Y tile
-            const int cch = q * 4 + v4;                    // 16-byte chunk index along the row, 0..15
-            const uint4 yv = *(const uint4*)(yrow + (cch >> 3) * X_HALF + (((cch & 7) ^ (row & 7)) << 4));
-            const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
-            uint32_t hi[4], lo[4];
+        for (int v4 = 0; v4 < 4; ++v4) {
+          // channels 32q + 8v4 .. +7 of this token: one 16-byte chunk of the swizzled Y tile
+          const int cch = q * 4 + v4;                    // 16-byte chunk index along the row, 0..15
+          const uint4 yv = *(const uint4*)(yrow + (cch >> 3) * X_HALF + (((cch & 7) ^ (row & 7)) << 4));
+          const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
+          uint32_t hi[4], lo[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const float v0 = __uint_as_float(yw[i] << 16) + __uint_as_float(r[v4 * 8 + 2 * i]);
-              const float v1 = __uint_as_float(yw[i] & 0xffff0000u) + __uint_as_float(r[v4 * 8 + 2 * i + 1]);
-              const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
-              hi[i] = *(const uint32_t*)&h2;
-              const __nv_bfloat162 l2 = __floats2bfloat162_rn(v0 - __uint_as_float(hi[i] << 16), v1 - __uint_as_float(hi[i] & 0xffff0000u));
-              lo[i] = *(const uint32_t*)&l2;
-            }
-            *(uint4*)(P.grid_hi + o + q * 32 + v4 * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            *(uint4*)(P.grid_lo + o + q * 32 + v4 * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          for (int i = 0; i < 4; ++i) {
+            const float v0 = __uint_as_float(yw[i] << 16) + __uint_as_float(r[v4 * 8 + 2 * i]);
+            const float v1 = __uint_as_float(yw[i] & 0xffff0000u) + __uint_as_float(r[v4 * 8 + 2 * i + 1]);
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+            hi[i] = *(const uint32_t*)&h2;
+            const __nv_bfloat162 l2 = __floats2bfloat162_rn(v0 - __uint_as_float(hi[i] << 16), v1 - __uint_as_float(hi[i] & 0xffff0000u));
+            lo[i] = *(const uint32_t*)&l2;
+          }
+          const int so = lane * X_STG_PITCH + ((v4 ^ ((lane >> 1) & 3)) << 4);
+          *(uint4*)(st_hi + so) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *(uint4*)(st_lo + so) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int rr = 8 * i + (lane >> 2), piece = lane & 3;      // row of the warp, 16-byte piece of its 64 bytes
+          if (fpos[i] >= 0) {
+            const size_t o = obase + (size_t)fpos[i] * XD + q * 32 + piece * 8;
+            const int so = rr * X_STG_PITCH + ((piece ^ ((rr >> 1) & 3)) << 4);
+            *(uint4*)(P.grid_hi + o) = *(const uint4*)(st_hi + so);
+            *(uint4*)(P.grid_lo + o) = *(const uint4*)(st_lo + so);
           }
         }
+        __syncwarp();
       }
       tc_fence_before();
       mbar_arrive(&sh.d_empty);
@@ -361,12 +398,19 @@ cudaError_t ffk_exchange_tc(ff_plan* p, int h0, int g, void* grid_hi, void* grid
   // two CTAs per SM: double-buffer the token tile only if both still fit in shared memory
   P.ybufs = (2 * X_TILE_BYTES + 4 * P.nkeys * 128 + sizeof(XShared) + 2048) * 2 <= 227 * 1024 ? 2 : 1;
   const size_t smem = P.ybufs * X_TILE_BYTES + 4 * P.nkeys * 128 + sizeof(XShared) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(exchange_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(exchange_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(exchange_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(exchange_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const long long tiles = (long long)g * ((dm.Nmid + XT - 1) / XT + (dm.Nhigh + XT - 1) / XT);
   const int grid = tiles < 2 * p->sm_count ? (int)tiles : 2 * p->sm_count;
-  exchange_tc_kernel<<<grid, X_THREADS, smem, st>>>(*(const CUtensorMap*)p->tmap_x[0], *(const CUtensorMap*)p->tmap_x[1],
-                                                   *(const CUtensorMap*)p->tmap_x[2], *(const CUtensorMap*)p->tmap_x[3], P);
+  const CUtensorMap& m0 = *(const CUtensorMap*)p->tmap_x[0];
+  const CUtensorMap& m1 = *(const CUtensorMap*)p->tmap_x[1];
+  const CUtensorMap& m2 = *(const CUtensorMap*)p->tmap_x[2];
+  const CUtensorMap& m3 = *(const CUtensorMap*)p->tmap_x[3];
+  if (P.nkeys <= 32) exchange_tc_kernel<1><<<grid, X_THREADS, smem, st>>>(m0, m1, m2, m3, P);
+  else if (P.nkeys <= 64) exchange_tc_kernel<2><<<grid, X_THREADS, smem, st>>>(m0, m1, m2, m3, P);
+  else exchange_tc_kernel<3><<<grid, X_THREADS, smem, st>>>(m0, m1, m2, m3, P);
   p->launches += 1;
   return cudaGetLastError();
 }
