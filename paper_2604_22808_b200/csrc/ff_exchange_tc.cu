@@ -74,8 +74,10 @@ __device__ __forceinline__ XItem x_decode(const FFDims& dm, int h0, int it, int 
 }
 
 // NK32 = 32-key chunks of the score row that are in use (3m <= 32 NK32).
+// (With three chunks the score row does not fit the registers two resident CTAs leave a thread, so
+// that variant runs one CTA per SM.)
 template <int NK32>
-__global__ void __launch_bounds__(X_THREADS, 2)
+__global__ void __launch_bounds__(X_THREADS, NK32 == 3 ? 1 : 2)
 exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_constant__ CUtensorMap map_v_mid,
                    const __grid_constant__ CUtensorMap map_y_high, const __grid_constant__ CUtensorMap map_v_high,
                    const XParams P) {
@@ -395,15 +397,17 @@ cudaError_t ffk_exchange_tc(ff_plan* p, int h0, int g, void* grid_hi, void* grid
   P.pos_mid = p->pos_table; P.pos_high = p->pos_table + dm.Nmid;
   P.grid_hi = (__nv_bfloat16*)grid_hi; P.grid_lo = (__nv_bfloat16*)grid_lo;
   P.h0 = h0; P.g = g; P.nkeys = (3 * dm.m + 15) / 16 * 16; P.status = p->buf.status;
-  // two CTAs per SM: double-buffer the token tile only if both still fit in shared memory
-  P.ybufs = (2 * X_TILE_BYTES + 4 * P.nkeys * 128 + sizeof(XShared) + 2048) * 2 <= 227 * 1024 ? 2 : 1;
+  // CTAs per SM: two, or one for the widest score rows; the token tile is double-buffered if the
+  // resident CTAs still fit in shared memory
+  const int per_sm = P.nkeys > 64 ? 1 : 2;
+  P.ybufs = (2 * X_TILE_BYTES + 4 * P.nkeys * 128 + sizeof(XShared) + 2048) * per_sm <= 227 * 1024 ? 2 : 1;
   const size_t smem = P.ybufs * X_TILE_BYTES + 4 * P.nkeys * 128 + sizeof(XShared) + 1024;
   cudaError_t e = cudaFuncSetAttribute(exchange_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(exchange_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(exchange_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const long long tiles = (long long)g * ((dm.Nmid + XT - 1) / XT + (dm.Nhigh + XT - 1) / XT);
-  const int grid = tiles < 2 * p->sm_count ? (int)tiles : 2 * p->sm_count;
+  const int grid = tiles < per_sm * p->sm_count ? (int)tiles : per_sm * p->sm_count;
   const CUtensorMap& m0 = *(const CUtensorMap*)p->tmap_x[0];
   const CUtensorMap& m1 = *(const CUtensorMap*)p->tmap_x[1];
   const CUtensorMap& m2 = *(const CUtensorMap*)p->tmap_x[2];
