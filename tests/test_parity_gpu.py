@@ -124,6 +124,22 @@ def test_replicas_stage_by_stage(cfg, routed):
     plan.destroy()
 
 
+# Tile geometries of the tensor-core transform that the replicas above do not reach: 4 and 8 lines
+# per 128-position tile on the t axis, a 128-long w axis (one line per tile), a 16-long w axis
+# (store boxes of two lines), unequal h and w.  All three bands and the pass-through paths per head.
+GEOMETRIES = [
+    C._make("geom_32x32x16", 1, (32, 32, 16), 3, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 21, (500,)),
+    C._make("geom_16x16x128", 1, (16, 16, 128), 3, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 22, (500,)),
+    C._make("geom_64x16x32", 1, (64, 16, 32), 3, 128, "bf16", (1, 8), 8, 64, 8, 256, 16, 23, (500,)),
+]
+
+
+@pytest.mark.parametrize("cfg", GEOMETRIES, ids=lambda c: c.name)
+def test_transform_tile_geometries(cfg):
+    _run(cfg, alloc=[7, 2, 4])
+    _run(cfg, alloc=[1, 4, 2], impl=2)       # and the generic transform on the same inputs
+
+
 def test_replica_simt_attention_matches_too():
     _run(C.R64K, alloc=[2, 4, 1, 7, 4, 2], impl=1)
 
