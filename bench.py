@@ -31,6 +31,7 @@ METRIC = "freqformer_attn_layer_tokens_per_s"
 # dram__bytes_read.sum + dram__bytes_write.sum of the transform kernels per token and head, from the ncu
 # capture summarised in profiles/dct_tc_kernel_64k_6heads.md (forward: three passes over Q, K and V;
 # inverse: three passes over one tensor).
+FP32_FMA_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 74.5: plain fp32 FMA rate of the GPU (unit counts x max clock)
 NCU_DRAM_BYTES_PER_TOKEN_HEAD = {"transform": 7516.0, "inverse": 3138.0}
 
 
@@ -315,11 +316,17 @@ def run_cuda(args, cfg):
         top = max(stage_ms, key=stage_ms.get)
         n_launch = max(1, stage_launches.get(top) or 1)
         heads_total = cfg.batch * cfg.heads
-        if top == "attention":
+        tensor_core_path = cfg.dtype == "bf16" and cfg.head_dim == 128       # otherwise the generic fp32 kernels run
+        if top == "attention" and tensor_core_path:
             achieved = work["attn_flops"] / (stage_ms[top] * 1e-3) / 1e12
             roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                     "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
                     "kernel": "attention_tc_kernel"}
+        elif top == "attention":
+            # generic attention kernel: fp32 FMAs; peak = 148 SMs x 128 lanes x 2 FLOP x 1.965 GHz
+            achieved = work["attn_flops"] / (stage_ms[top] * 1e-3) / 1e12
+            roof = {"bound": "alu", "achieved": achieved, "peak": FP32_FMA_TFLOPS, "unit": "TFLOP/s",
+                    "frac": achieved / FP32_FMA_TFLOPS, "traffic": None, "kernel": "attention_simt_kernel"}
         else:
             nbytes = work["bytes_transform"] if top == "transform" else work["bytes_inverse"]
             achieved = nbytes / (stage_ms[top] * 1e-3) / 1e9
@@ -327,8 +334,9 @@ def run_cuda(args, cfg):
             # (profiles/dct_tc_kernel_64k_6heads.md); traffic is proportional to tokens x heads.
             per_token_head = NCU_DRAM_BYTES_PER_TOKEN_HEAD[top]
             roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": per_token_head * cfg.N * heads_total / n_launch,
-                    "kernel": "dct_tc_kernel (%s stage)" % top,
+                    "frac": achieved / peaks["hbm_gbs"],
+                    "traffic": per_token_head * cfg.N * heads_total / n_launch if tensor_core_path else None,
+                    "kernel": ("dct_tc_kernel (%s stage)" if tensor_core_path else "dct_pass_kernel (%s stage)") % top,
                     "algorithmic_bytes_per_launch": nbytes / n_launch}
         roof.update({"stage": top, "launches_per_step": stage_launches.get(top), "ms_per_step": stage_ms[top],
                      "ms_per_launch": stage_ms[top] / n_launch, "peak_source": peaks["source"]})

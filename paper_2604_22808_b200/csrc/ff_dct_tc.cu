@@ -61,8 +61,6 @@ struct DctTcParams {
   int group_start;         // index of the first one (tensor * BH + bh for the forward, bh for the inverse)
   int in_split;            // input is a hi/lo pair of grids (map0 = hi, map1 = lo)
   int nstage;              // ring depth
-  __nv_bfloat16* dst;      // hi grid [group][T][H][W][128], or the out tensor (MODE_LAST)
-  __nv_bfloat16* dst_lo;   // lo grid
   float* side;             // MODE_FIRST: [group][T][H][L_w][128] fp32
   __nv_bfloat16* spec_mid; __nv_bfloat16* spec_high;
   double* energy;          // [B][3][128]
@@ -632,16 +630,15 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
       if (e != cudaSuccess) return e;
     } else {
       P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 2 + 0) * TILE_BYTES;
-      P.dst = sc.a_hi; P.dst_lo = sc.a_lo; P.side = side;
+      P.side = side;
       e = launch_pass(p, mq, mk, mv, o0h, o0l, P, st);
       if (e != cudaSuccess) return e;
       P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 1 + 0) * TILE_BYTES;
-      P.dst = sc.b_hi; P.dst_lo = sc.b_lo;
       e = launch_pass(p, m1h, m1l, m1l, o1h, o1l, P, st);
       if (e != cudaSuccess) return e;
     }
     P.in_split = 1;
-    P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 0 + 0) * TILE_BYTES; P.dst = nullptr;
+    P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 0 + 0) * TILE_BYTES;
     e = launch_pass(p, m2h, m2l, m2l, m2h, m2l, P, st);    // (no tensor stores in this mode)
     if (e != cudaSuccess) return e;
     dim3 lgrid((unsigned)dm.L[2], (unsigned)g);
@@ -671,16 +668,13 @@ cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaS
   DctTcParams P{};
   P.dm = dm; P.status = p->buf.status; P.group = g; P.group_start = h0;
   P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 3 + 0) * TILE_BYTES;
-  P.dst = sc.b_hi; P.dst_lo = sc.b_lo;
   cudaError_t e = launch_pass(p, m_in, m_inl, m_inl, obh, obl, P, st);
   if (e != cudaSuccess) return e;
   if ((p->attn_impl & 4) && ffk_dct_wh_usable(dm, g, p->sm_count))
     return ffk_dct_wh_launch(p, 0, sc.b_hi, sc.b_lo, nullptr, h0, g, sc.ring, out, nullptr, nullptr, st);
   P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 4 + 0) * TILE_BYTES;
-  P.dst = sc.a_hi; P.dst_lo = sc.a_lo;
   e = launch_pass(p, mbh, mbl, mbl, oah, oal, P, st);
   if (e != cudaSuccess) return e;
   P.mode = MODE_LAST; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 5 + 0) * TILE_BYTES;
-  P.dst = (__nv_bfloat16*)out; P.dst_lo = nullptr;
   return launch_pass(p, mah, mal, mal, mout, mout, P, st);
 }

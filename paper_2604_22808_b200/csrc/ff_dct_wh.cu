@@ -50,10 +50,6 @@ struct WhParams {
   int ring, lag;               // ring slots, and how many slabs the second pass trails the first
   int* cnt_a;                  // [slabs] first-pass epilogue warps done
   int* cnt_b;                  // [slabs] second-pass epilogue warps done
-  __nv_bfloat16* ring_hi;      // [ring][H][W][128]
-  __nv_bfloat16* ring_lo;
-  __nv_bfloat16* out_hi;       // forward: hi grid [group][T][H][W][128]; inverse: the out tensor
-  __nv_bfloat16* out_lo;       // forward: lo grid; inverse: unused
   float* side;                 // forward: [group][T][H][L_w][128] fp32
   int* status;
 };
@@ -463,11 +459,11 @@ cudaError_t ffk_dct_wh_launch(ff_plan* p, int forward, const void* src0, const v
   const int S = g * dm.T;
   if (P.lag > S) P.lag = S;
   const size_t slab = (size_t)n * n * CH * 2;
-  P.ring_hi = (__nv_bfloat16*)ring;
-  P.ring_lo = (__nv_bfloat16*)((char*)ring + (size_t)P.ring * slab);
+  void* ring_hi = ring;                                  // [ring][H][W][128]
+  void* ring_lo = (char*)ring + (size_t)P.ring * slab;
   P.cnt_a = (int*)((char*)ring + 2 * (size_t)P.ring * slab);
   P.cnt_b = P.cnt_a + S;
-  P.out_hi = (__nv_bfloat16*)out_hi; P.out_lo = (__nv_bfloat16*)out_lo; P.side = side; P.status = p->buf.status;
+  P.side = side; P.status = p->buf.status;
   // one image serves both passes: I kron C (forward) or I kron C^T (inverse) of the w axis
   P.image = p->dct_images + (size_t)(2 * ((forward ? 0 : 3) + 2)) * TILE_BYTES;
   cudaError_t e = cudaMemsetAsync(P.cnt_a, 0, (size_t)2 * S * sizeof(int), st);
@@ -477,15 +473,15 @@ cudaError_t ffk_dct_wh_launch(ff_plan* p, int forward, const void* src0, const v
   bool ok;
   if (forward)
     ok = encode_wh_map(&m0, src0, n, dm.T, dm.BH, true) && encode_wh_map(&m1, src1, n, dm.T, dm.BH, true) &&
-         encode_wh_map(&m2, src2, n, dm.T, dm.BH, true) && encode_wh_map(&m3, P.ring_hi, n, P.ring, 1, false) &&
-         encode_wh_map(&m4, P.ring_lo, n, P.ring, 1, false) &&
-         encode_wh_store_map(&s_rh, P.ring_hi, n, P.ring, 1, true) && encode_wh_store_map(&s_rl, P.ring_lo, n, P.ring, 1, true) &&
+         encode_wh_map(&m2, src2, n, dm.T, dm.BH, true) && encode_wh_map(&m3, ring_hi, n, P.ring, 1, false) &&
+         encode_wh_map(&m4, ring_lo, n, P.ring, 1, false) &&
+         encode_wh_store_map(&s_rh, ring_hi, n, P.ring, 1, true) && encode_wh_store_map(&s_rl, ring_lo, n, P.ring, 1, true) &&
          encode_wh_store_map(&s_oh, out_hi, n, dm.T, g, false) && encode_wh_store_map(&s_ol, out_lo, n, dm.T, g, false);
   else
     ok = encode_wh_map(&m0, src0, n, dm.T, g, false) && encode_wh_map(&m1, src1, n, dm.T, g, false) &&
-         encode_wh_map(&m2, src1, n, dm.T, g, false) && encode_wh_map(&m3, P.ring_hi, n, P.ring, 1, true) &&
-         encode_wh_map(&m4, P.ring_lo, n, P.ring, 1, true) &&
-         encode_wh_store_map(&s_rh, P.ring_hi, n, P.ring, 1, false) && encode_wh_store_map(&s_rl, P.ring_lo, n, P.ring, 1, false) &&
+         encode_wh_map(&m2, src1, n, dm.T, g, false) && encode_wh_map(&m3, ring_hi, n, P.ring, 1, true) &&
+         encode_wh_map(&m4, ring_lo, n, P.ring, 1, true) &&
+         encode_wh_store_map(&s_rh, ring_hi, n, P.ring, 1, false) && encode_wh_store_map(&s_rl, ring_lo, n, P.ring, 1, false) &&
          encode_wh_store_map(&s_oh, out_hi, n, dm.T, dm.BH, true) && encode_wh_store_map(&s_ol, out_hi, n, dm.T, dm.BH, true);
   if (!ok) return cudaErrorInvalidValue;
   const size_t smem = NSTAGE * STAGE_BYTES + 2 * TILE_BYTES + sizeof(WhShared) + 1024;

@@ -140,6 +140,13 @@ def test_transform_tile_geometries(cfg):
     _run(cfg, alloc=[1, 4, 2], impl=2)       # and the generic transform on the same inputs
 
 
+def test_paper_reference_parameterisation_replica():
+    """d_k = 64, N_low_bar = N / 32, w = 64, constant-degree mid pattern (generic kernels)."""
+    cfg = C.R_PAPER_REF
+    _run(cfg, alloc=[1, 2, 4, 7])
+    _run(cfg)                                   # routed
+
+
 def test_replica_simt_attention_matches_too():
     _run(C.R64K, alloc=[2, 4, 1, 7, 4, 2], impl=1)
 
