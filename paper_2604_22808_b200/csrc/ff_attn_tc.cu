@@ -1,6 +1,6 @@
 // Mid- and high-band attention on the 5th-generation tensor cores ("Hierarchical frequency-domain
 // attention": strided block-sparse attention on the mid band, sliding-window attention on the high
-// band), bf16 operands, fp32 accumulation, head_dim 128.
+// band), bf16 operands, fp32 accumulation, head_dim 128 or 64 (template parameter HD).
 //
 // One persistent launch runs both branches from a worklist of (head, band, pair of query tiles)
 // items that is rebuilt from the head-to-band allocation before every launch.  A CTA owns every
@@ -30,12 +30,12 @@ using namespace sm100;
 namespace {
 
 constexpr int TILE = 128;            // query rows per stream = key rows per tile
-constexpr int HD = 128;              // head_dim
-constexpr int TILE_BYTES = TILE * HD * 2;
+constexpr int HD_MAX = 128;          // largest head_dim; the shared-memory slots are sized for it
+constexpr int TILE_BYTES = TILE * HD_MAX * 2;
 constexpr int HALF_BYTES = TILE_BYTES / 2;
 constexpr int MAX_UNITS = 1024;
 constexpr int NSPLIT = 2;                // softmax threads per query row
-constexpr int SCOLS = TILE / NSPLIT;     // key (and output) columns per softmax thread
+constexpr int SCOLS = TILE / NSPLIT;     // key columns per softmax thread
 constexpr int TC_THREADS = 64 + 2 * 128 * NSPLIT;   // TMA warp, MMA warp, 2 streams x 4 NSPLIT softmax warps
 constexpr float LAZY_LOG2 = 8.0f;    // rescale O only when the running max grows by more than this (log2 units)
 
@@ -49,8 +49,31 @@ struct TcParams {
   int rb_mid;         // rows per TMA box of the mid map = min(b, 128)
 };
 
-// Worklist: one unit per (head, mid residue class) and per (head, high band) that the allocation
-// executes; mid units first (their items are the long ones).  An item is a pair of query tiles.
+// The residue classes of the mid band come in two sizes: the first `rem` = nb mod s classes hold
+// one block more than the others.  Items of a (head, mid band) unit are numbered class by class.
+struct MidShape {
+  int rem;              // classes with the larger block count
+  int nclass;           // residue classes that exist: min(nb, s)
+  int nt_big, nt_small; // query (= key) tiles of a class of either size
+  int pairs_big, pairs_small;
+  int items;            // items of one head's mid band
+};
+
+__host__ __device__ __forceinline__ MidShape mid_shape(const FFDims& dm) {
+  MidShape m;
+  const long long q = dm.s > 0 ? dm.nb / dm.s : 0;
+  m.rem = dm.s > 0 ? (int)(dm.nb % dm.s) : 0;
+  m.nclass = (int)(dm.nb < dm.s ? dm.nb : dm.s);
+  m.nt_big = (int)(((q + 1) * dm.b + TILE - 1) / TILE);
+  m.nt_small = (int)((q * dm.b + TILE - 1) / TILE);
+  m.pairs_big = (m.nt_big + 1) / 2;
+  m.pairs_small = (m.nt_small + 1) / 2;
+  m.items = m.rem * m.pairs_big + (m.nclass - m.rem) * m.pairs_small;
+  return m;
+}
+
+// Worklist: one unit per (head, mid band) and per (head, high band) that the allocation executes;
+// mid units first (their items are the long ones).  An item is a pair of query tiles.
 __global__ void build_worklist_kernel(TcParams P) {
   if (threadIdx.x != 0 || blockIdx.x != 0) return;
   const FFDims& dm = P.dm;
@@ -58,15 +81,11 @@ __global__ void build_worklist_kernel(TcParams P) {
   int* desc = offsets + MAX_UNITS + 1;
   int* tiles = desc + MAX_UNITS;
   int nu = 0, total = 0;
-  const int nclass = (int)(dm.nb < dm.s ? dm.nb : dm.s);
-  for (int bh = 0; bh < dm.BH; ++bh) {
+  const MidShape ms = mid_shape(dm);
+  for (int bh = 0; bh < dm.BH && nu < MAX_UNITS; ++bh) {
     if (!(P.alloc[bh] & FF_BAND_MID)) continue;
-    for (int c = 0; c < nclass && nu < MAX_UNITS; ++c) {
-      const long long nblk = (dm.nb - c + dm.s - 1) / dm.s;
-      const int nt = (int)((nblk * dm.b + TILE - 1) / TILE);
-      offsets[nu] = total; desc[nu] = (bh << 12) | (1 << 10) | c; tiles[nu] = nt;
-      total += (nt + 1) / 2; ++nu;
-    }
+    offsets[nu] = total; desc[nu] = (bh << 12) | (1 << 10); tiles[nu] = 0;
+    total += ms.items; ++nu;
   }
   for (int bh = 0; bh < dm.BH && nu < MAX_UNITS; ++bh) {
     if (!(P.alloc[bh] & FF_BAND_HIGH)) continue;
@@ -102,7 +121,7 @@ struct Shared {
   unsigned long long xsum[2][2][NSPLIT][128];
 };
 
-__device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, int it) {
+__device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, const MidShape& ms, int it) {
   int lo = 0, hi = sh.n_units - 1;
   while (lo < hi) {                       // last unit whose offset <= it
     const int mid = (lo + hi + 1) >> 1;
@@ -110,14 +129,23 @@ __device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, 
   }
   Item x;
   const int dsc = sh.desc[lo];
-  x.bh = dsc >> 12; x.band = (dsc >> 10) & 3; x.c = dsc & 1023;
-  x.tile_a = 2 * (it - sh.offsets[lo]);
-  x.has_b = x.tile_a + 1 < sh.ntile[lo];
+  x.bh = dsc >> 12; x.band = (dsc >> 10) & 3; x.c = 0;
+  const int local = it - sh.offsets[lo];
   if (x.band == 1) {
+    int pr, nt;
+    if (local < ms.rem * ms.pairs_big) { x.c = local / ms.pairs_big; pr = local % ms.pairs_big; nt = ms.nt_big; }
+    else {
+      const int l2 = local - ms.rem * ms.pairs_big;
+      x.c = ms.rem + l2 / ms.pairs_small; pr = l2 % ms.pairs_small; nt = ms.nt_small;
+    }
+    x.tile_a = 2 * pr;
+    x.has_b = x.tile_a + 1 < nt;
     x.n = dm.Nmid;
-    x.nk = sh.ntile[lo];                  // every query tile of a class sees all its key tiles
+    x.nk = nt;                            // every query tile of a class sees all its key tiles
     x.ks = 0;
   } else {
+    x.tile_a = 2 * local;
+    x.has_b = x.tile_a + 1 < sh.ntile[lo];
     x.n = dm.Nhigh;
     const long long q0 = (long long)x.tile_a * TILE;
     x.ks = q0 - dm.R > 0 ? q0 - dm.R : 0;
@@ -148,18 +176,19 @@ __device__ __forceinline__ long long mid_rank(const FFDims& dm, int c, long long
 
 // Issues the TMA loads of one 128-row tile (two 64-column halves) into `dst`; the caller has
 // already announced the bytes on `bar`.  `first` = class-local position (mid) or band rank (high).
+// `halves` = head_dim / 64.
 __device__ __forceinline__ void load_tile(uint8_t* dst, const CUtensorMap* map, uint64_t* bar, const FFDims& dm,
-                                          const Item& x, int slice, long long first, int rb) {
+                                          const Item& x, int slice, long long first, int rb, int halves) {
   if (x.band == 2) {
     tma_load_3d(dst, map, bar, 0, (int)first, slice);
-    tma_load_3d(dst + HALF_BYTES, map, bar, 64, (int)first, slice);
+    if (halves > 1) tma_load_3d(dst + HALF_BYTES, map, bar, 64, (int)first, slice);
   } else {
     for (int i = 0; i < TILE / rb; ++i) {
       const long long row = mid_rank(dm, x.c, first + (long long)i * rb);
       // a block past the end of the band starts beyond the tensor: the copy fills zeros
       const int y = row < dm.Nmid ? (int)row : (int)dm.Nmid;
       tma_load_3d(dst + i * rb * 128, map, bar, 0, y, slice);
-      tma_load_3d(dst + HALF_BYTES + i * rb * 128, map, bar, 64, y, slice);
+      if (halves > 1) tma_load_3d(dst + HALF_BYTES + i * rb * 128, map, bar, 64, y, slice);
     }
   }
 }
@@ -201,7 +230,7 @@ __device__ __forceinline__ float ex2(float x) {
 // which hold Q~, K~ and V~ of head bh in slices bh, BH + bh and 2 BH + bh.  QKV_MAPS = true (the entry
 // point that allocates nothing): map_a, map_b, map_c are the caller's separate Q, K, V tensors of one
 // band, head bh in slice bh.
-template <bool QKV_MAPS>
+template <int HD, bool QKV_MAPS>
 __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, const CUtensorMap& map_b,
                                                   const CUtensorMap& map_c, const TcParams& P) {
   extern __shared__ uint8_t smem_raw[];
@@ -212,6 +241,9 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
   Shared& sh = *(Shared*)(smem + 6 * TILE_BYTES);
   const FFDims& dm = P.dm;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int HALVES = HD / 64;                  // 64-channel halves of a row
+  constexpr int TB = TILE * HD * 2;                // bytes of one tile
+  constexpr int OCOLS = HD / NSPLIT;               // output columns per softmax thread
 
   if (threadIdx.x == 0) {
     mbar_init(&sh.q_full, 1); mbar_init(&sh.q_empty, 1);
@@ -244,6 +276,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
   tc_fence_after();
   const uint32_t tm = sh.tmem_base;
   const int total = sh.total;
+  const MidShape ms = mid_shape(dm);
   volatile int* abort_flag = &sh.abort_flag;
 
   if (warp == 0) {
@@ -253,7 +286,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
       int iter = 0; unsigned g = 0;
       bool ok = true;
       for (int it = blockIdx.x; it < total && ok; it += gridDim.x, ++iter) {
-        const Item x = decode_item(sh, dm, it);
+        const Item x = decode_item(sh, dm, ms, it);
         const CUtensorMap* map = x.band == 1 ? &map_a : &map_b;
         const CUtensorMap* mapq = QKV_MAPS ? &map_a : map;
         const CUtensorMap* mapk = QKV_MAPS ? &map_b : map;
@@ -262,20 +295,20 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         const int rb = x.band == 1 ? P.rb_mid : TILE;
         if (iter >= 1) ok = mbar_wait(&sh.q_empty, (iter - 1) & 1, abort_flag);
         if (!ok) break;
-        mbar_arrive_expect_tx(&sh.q_full, x.has_b ? 2 * TILE_BYTES : TILE_BYTES);
-        load_tile(sQ, mapq, &sh.q_full, dm, x, x.bh, (long long)x.tile_a * TILE, rb);
-        if (x.has_b) load_tile(sQ + TILE_BYTES, mapq, &sh.q_full, dm, x, x.bh, (long long)(x.tile_a + 1) * TILE, rb);
+        mbar_arrive_expect_tx(&sh.q_full, x.has_b ? 2 * TB : TB);
+        load_tile(sQ, mapq, &sh.q_full, dm, x, x.bh, (long long)x.tile_a * TILE, rb, HALVES);
+        if (x.has_b) load_tile(sQ + TILE_BYTES, mapq, &sh.q_full, dm, x, x.bh, (long long)(x.tile_a + 1) * TILE, rb, HALVES);
         for (int j = 0; j < x.nk && ok; ++j, ++g) {
           const int st = g & 1;
           const long long first = x.band == 1 ? (long long)j * TILE : x.ks + (long long)j * TILE;
           if (g >= 2) ok = mbar_wait(&sh.k_empty[st], ((g >> 1) - 1) & 1, abort_flag);
           if (!ok) break;
-          mbar_arrive_expect_tx(&sh.k_full[st], TILE_BYTES);
-          load_tile(sK + st * TILE_BYTES, mapk, &sh.k_full[st], dm, x, slice_k, first, rb);
+          mbar_arrive_expect_tx(&sh.k_full[st], TB);
+          load_tile(sK + st * TILE_BYTES, mapk, &sh.k_full[st], dm, x, slice_k, first, rb, HALVES);
           if (g >= 2) ok = mbar_wait(&sh.v_empty[st], ((g >> 1) - 1) & 1, abort_flag);
           if (!ok) break;
-          mbar_arrive_expect_tx(&sh.v_full[st], TILE_BYTES);
-          load_tile(sV + st * TILE_BYTES, mapv, &sh.v_full[st], dm, x, slice_v, first, rb);
+          mbar_arrive_expect_tx(&sh.v_full[st], TB);
+          load_tile(sV + st * TILE_BYTES, mapv, &sh.v_full[st], dm, x, slice_v, first, rb, HALVES);
         }
       }
     }
@@ -293,7 +326,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         const int st = gt & 1;
         const uint32_t qbase = smem_u32(sQ + sx * TILE_BYTES), kbase = smem_u32(sK + st * TILE_BYTES);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
+        for (int k = 0; k < HD / 16; ++k) {
           const uint32_t off = (k >> 2) * HALF_BYTES + (k & 3) * 32;
           umma_ss(tm + sx * 128, smem_desc_sw128(qbase + off, 16, 1024), smem_desc_sw128(kbase + off, 16, 1024),
                   idesc_qk, k > 0 ? 1u : 0u);
@@ -322,7 +355,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         return true;
       };
       for (int it = blockIdx.x; it < total && ok; it += gridDim.x, ++iter) {
-        const Item x = decode_item(sh, dm, it);
+        const Item x = decode_item(sh, dm, ms, it);
         ok = mbar_wait(&sh.q_full, iter & 1, abort_flag);
         if (!ok) break;
         const unsigned g0 = g;
@@ -373,17 +406,18 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
     const int sx = (warp - 2) / (4 * NSPLIT);
     const int part = ((warp - 2) >> 2) % NSPLIT;
     const int row = quarter * 32 + lane;
-    const int col0 = part * SCOLS;
+    const int col0 = part * SCOLS;                      // first key column of this thread
+    const int ocol0 = part * OCOLS;                     // first output column of this thread
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const uint32_t s_addr = tm + lane_addr + sx * 128;
-    const uint32_t o_addr = tm + lane_addr + 256 + sx * 128 + col0;      // this thread's output columns
+    const uint32_t o_addr = tm + lane_addr + 256 + sx * 128 + ocol0;     // this thread's output columns
     const float sl2 = rsqrtf((float)HD) * 1.4426950408889634f;
     unsigned cs = 0;                  // key tiles this stream has processed (phases of s_full / p_full)
     unsigned co = 0;                  // phases of o_full consumed
     unsigned ci = 0;                  // items this stream has processed
     bool ok = true;
     for (int it = blockIdx.x; it < total && ok; it += gridDim.x) {
-      const Item x = decode_item(sh, dm, it);
+      const Item x = decode_item(sh, dm, ms, it);
       if (sx == 1 && !x.has_b) continue;
       const int tile = x.tile_a + sx;
       // band rank of this thread's query row
@@ -455,7 +489,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
-          for (int c = 0; c < SCOLS / 32; ++c) {
+          for (int c = 0; c < OCOLS / 32; ++c) {
             uint32_t r[32];
             tmem_ld32(o_addr + c * 32, r);
             tmem_wait_ld();
@@ -514,9 +548,9 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
       tc_fence_after();
       const float inv = 1.f / l;
       const bool store = p < x.n;
-      __nv_bfloat16* y = (x.band == 1 ? P.y_mid : P.y_high) + ((size_t)x.bh * x.n + (store ? p : 0)) * HD + col0;
+      __nv_bfloat16* y = (x.band == 1 ? P.y_mid : P.y_high) + ((size_t)x.bh * x.n + (store ? p : 0)) * HD + ocol0;
 #pragma unroll
-      for (int c = 0; c < SCOLS / 32; ++c) {
+      for (int c = 0; c < OCOLS / 32; ++c) {
         uint32_t r[32];
         tmem_ld32(o_addr + c * 32, r);
         tmem_wait_ld();
@@ -556,17 +590,18 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
   }
 }
 
+template <int HD>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_mid, const __grid_constant__ CUtensorMap map_high,
                     const TcParams P) {
-  attention_tc_body<false>(map_mid, map_high, map_high, P);
+  attention_tc_body<HD, false>(map_mid, map_high, map_high, P);
 }
 
 // Same kernel on the caller's separate Q, K, V tensors of one band (see ff_high_attention_noalloc).
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attention_tc_qkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                         const __grid_constant__ CUtensorMap map_v, const TcParams P) {
-  attention_tc_body<true>(map_q, map_k, map_v, P);
+  attention_tc_body<HD_MAX, true>(map_q, map_k, map_v, P);
 }
 
 // Scratch of ff_high_attention_noalloc: the worklist, one band mask per head and a status word.
@@ -580,15 +615,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-bool encode_band_map(CUtensorMap* map, void* base, long long rows, int slices, int box_rows) {
+bool encode_band_map(CUtensorMap* map, void* base, long long rows, int slices, int box_rows, int hd = HD_MAX) {
   static EncodeTiledFn enc = nullptr;
   if (!enc) {
     cudaDriverEntryPointQueryResult qr;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", (void**)&enc, cudaEnableDefault, &qr) != cudaSuccess || !enc)
       return false;
   }
-  cuuint64_t dims[3] = {(cuuint64_t)HD, (cuuint64_t)rows, (cuuint64_t)slices};
-  cuuint64_t strides[2] = {(cuuint64_t)HD * 2, (cuuint64_t)rows * HD * 2};
+  cuuint64_t dims[3] = {(cuuint64_t)hd, (cuuint64_t)rows, (cuuint64_t)slices};
+  cuuint64_t strides[2] = {(cuuint64_t)hd * 2, (cuuint64_t)rows * hd * 2};
   cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
   cuuint32_t es[3] = {1, 1, 1};
   return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -599,13 +634,13 @@ bool encode_band_map(CUtensorMap* map, void* base, long long rows, int slices, i
 
 size_t ffk_tc_work_bytes() { return (size_t)(2 + 3 * MAX_UNITS + 1) * sizeof(int); }
 
-// The tensor-core kernel covers bf16, head_dim 128 and block sizes that tile 128 rows evenly.
+// The tensor-core kernel covers bf16, head_dim 128 or 64 and block sizes that tile 128 rows evenly.
 bool ffk_tc_supported(const FFDims& dm) {
-  if (dm.fp32 || dm.d != HD) return false;
+  if (dm.fp32 || (dm.d != 128 && dm.d != 64)) return false;
   const bool b_ok = (dm.b <= TILE) ? (dm.b >= 8 && TILE % dm.b == 0) : (dm.b % TILE == 0);
   if (!b_ok) return false;
-  const long long nclass = dm.nb < dm.s ? dm.nb : dm.s;
-  if ((long long)dm.BH * (nclass + 1) > MAX_UNITS || dm.BH >= (1 << 19)) return false;
+  if ((long long)dm.BH * 2 > MAX_UNITS || dm.BH >= (1 << 19)) return false;
+  if ((long long)dm.BH * (mid_shape(dm).items + (dm.Nhigh + 2 * TILE - 1) / (2 * TILE)) >= (1LL << 31)) return false;
   if (dm.Nmid >= (1LL << 31) - 256 || dm.Nhigh >= (1LL << 31) - 256) return false;
   return true;
 }
@@ -614,8 +649,8 @@ bool ffk_tc_prepare(ff_plan* p) {
   static_assert(sizeof(CUtensorMap) <= sizeof(p->tmap_mid), "tensor map storage too small");
   const FFDims& dm = p->dm;
   const int rb = dm.b < TILE ? dm.b : TILE;
-  return encode_band_map((CUtensorMap*)p->tmap_mid, p->buf.spec_mid, dm.Nmid, 3 * dm.BH, rb) &&
-         encode_band_map((CUtensorMap*)p->tmap_high, p->buf.spec_high, dm.Nhigh, 3 * dm.BH, TILE);
+  return encode_band_map((CUtensorMap*)p->tmap_mid, p->buf.spec_mid, dm.Nmid, 3 * dm.BH, rb, dm.d) &&
+         encode_band_map((CUtensorMap*)p->tmap_high, p->buf.spec_high, dm.Nhigh, 3 * dm.BH, TILE, dm.d);
 }
 
 cudaError_t ffk_attention_tc(ff_plan* p, cudaStream_t st) {
@@ -628,10 +663,13 @@ cudaError_t ffk_attention_tc(ff_plan* p, cudaStream_t st) {
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const size_t smem = 6 * TILE_BYTES + sizeof(Shared) + 1024;
-  e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  e = cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  attention_tc_kernel<<<p->sm_count, TC_THREADS, smem, st>>>(*(const CUtensorMap*)p->tmap_mid,
-                                                             *(const CUtensorMap*)p->tmap_high, P);
+  const CUtensorMap& mm = *(const CUtensorMap*)p->tmap_mid;
+  const CUtensorMap& mh = *(const CUtensorMap*)p->tmap_high;
+  if (dm.d == 128) attention_tc_kernel<128><<<p->sm_count, TC_THREADS, smem, st>>>(mm, mh, P);
+  else attention_tc_kernel<64><<<p->sm_count, TC_THREADS, smem, st>>>(mm, mh, P);
   p->launches += 2;
   return cudaGetLastError();
 }
@@ -689,7 +727,7 @@ extern "C" ff_status_t ff_high_attention_noalloc(const void* q, const void* k, c
   }
   cudaStream_t st = (cudaStream_t)cuda_stream;
   TcParams P{};
-  P.dm.B = 1; P.dm.heads = heads; P.dm.BH = heads; P.dm.d = HD; P.dm.R = radius;
+  P.dm.B = 1; P.dm.heads = heads; P.dm.BH = heads; P.dm.d = HD_MAX; P.dm.R = radius;
   P.dm.Nhigh = n; P.dm.Nmid = 0; P.dm.nb = 0; P.dm.s = 1; P.dm.b = TILE; P.dm.r = 1;
   P.work = (int*)scratch;
   uint8_t* masks = scratch + NOALLOC_WORK_BYTES;
