@@ -100,13 +100,13 @@ BY_NAME.update({c.name: c for c in REPLICAS})
 # = the box of about 0.794 of every axis), r = 4 so that N_low_bar = N / 32, window w = 64 (R = 32),
 # m = 8, and a mid pattern of constant degree k_mid = 256: blocks of 32 ranks with stride
 # s = N_mid / 256 rounded, so that a residue class holds 8 blocks.  head_dim 64 is outside the
-# tensor-core kernels (head_dim 128); this workload runs on the generic kernels.
+# tensor-core exchange kernel (head_dim 128 only), which the generic kernel replaces here.
 PAPER_REF_64K = FFConfig(name="paper_ref_64k", batch=1, T=16, H=64, W=64, heads=16, head_dim=64, dtype="bf16",
                          low_cut=(8, 32, 32), mid_cut=(13, 51, 51), r=4, b=32, s=100, R=32, m=8, seed=5,
                          timesteps=(500.0,))
-# ... and its replica on a grid the oracle covers in full: 2048 tokens, N_low_bar = N / 32 = 64,
-# four blocks per residue class.
-R_PAPER_REF = FFConfig(name="paper_ref_replica", batch=1, T=8, H=16, W=16, heads=4, head_dim=64, dtype="bf16",
-                       low_cut=(4, 8, 8), mid_cut=(6, 13, 13), r=4, b=32, s=6, R=32, m=8, seed=15,
+# ... and its replica on a grid the oracle covers in full (axis lengths the tensor-core transform
+# covers): 4096 tokens, N_low_bar = N / 32 = 128, nine blocks per residue class.
+R_PAPER_REF = FFConfig(name="paper_ref_replica", batch=1, T=16, H=16, W=16, heads=4, head_dim=64, dtype="bf16",
+                       low_cut=(8, 8, 8), mid_cut=(13, 13, 13), r=4, b=32, s=6, R=32, m=8, seed=15,
                        timesteps=(500.0,))
 BY_NAME.update({c.name: c for c in (PAPER_REF_64K, R_PAPER_REF)})

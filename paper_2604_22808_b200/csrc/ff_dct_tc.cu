@@ -1,5 +1,5 @@
 // Separable transform on the tensor cores ("Separable spectral decomposition", "Reconstruction"),
-// bf16 storage, head_dim 128.  Every axis pass is a batched contraction over "lines" of n grid
+// bf16 storage, head_dim 128 or 64 (template parameter CH).  Every axis pass is a batched contraction over "lines" of n grid
 // positions along the axis (all other coordinates fixed): out[a][c] = sum_b Mat[a][b] in[b][c].
 // A CTA works on tiles of 128 grid positions = 128/n adjacent lines, fetched by one TMA box per
 // 64-channel half (a contiguous run of memory for the w axis; 128/n neighbouring w positions per
@@ -41,9 +41,9 @@ using namespace sm100;
 
 namespace {
 
-constexpr int CH = 128;
+constexpr int CH_MAX = 128;                          // largest head_dim; shared-memory tiles are sized for it
 constexpr int TILE_ROWS = 128;
-constexpr int TILE_BYTES = TILE_ROWS * CH * 2;     // 32 KB: 128 rows of bf16
+constexpr int TILE_BYTES = TILE_ROWS * CH_MAX * 2; // 32 KB: 128 rows of bf16
 constexpr int HALF_BYTES = TILE_BYTES / 2;
 constexpr int MAX_STAGE = 4;
 constexpr int NACC = 4;
@@ -113,6 +113,7 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
 // Three source maps (Q, K, V) in MODE_FIRST; otherwise map0 (= hi) and, for split input, map1 (= lo).
 // map_oh / map_ol: destination hi / lo grids with the box of one epilogue warp (32 positions x 32
 // channels), all modes but SPLIT; MODE_LAST has no lo grid.
+template <int CH>
 __global__ void __launch_bounds__(DCT_TC_THREADS, 1)
 dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
               const __grid_constant__ CUtensorMap map2, const __grid_constant__ CUtensorMap map_oh,
@@ -174,12 +175,12 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
           map = tensor == 0 ? &map0 : (tensor == 1 ? &map1 : &map2);
           slice = th % dm.BH;
         }
-        mbar_arrive_expect_tx(&sh.full[slot], STAGE_BYTES);
+        mbar_arrive_expect_tx(&sh.full[slot], (P.in_split ? 2 : 1) * TILE_ROWS * CH * 2);
         tma_load_5d(dst, map, &sh.full[slot], 0, w, h, t, slice);
-        tma_load_5d(dst + HALF_BYTES, map, &sh.full[slot], 64, w, h, t, slice);
+        if (CH == 128) tma_load_5d(dst + HALF_BYTES, map, &sh.full[slot], 64, w, h, t, slice);
         if (P.in_split) {
           tma_load_5d(dst + TILE_BYTES, &map1, &sh.full[slot], 0, w, h, t, slice);
-          tma_load_5d(dst + TILE_BYTES + HALF_BYTES, &map1, &sh.full[slot], 64, w, h, t, slice);
+          if (CH == 128) tma_load_5d(dst + TILE_BYTES + HALF_BYTES, &map1, &sh.full[slot], 64, w, h, t, slice);
         }
       }
     }
@@ -217,7 +218,8 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     const int l = seq ? j >> ln : j & (kf - 1);           // line of the tile
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const int ew = warp - 2;                              // epilogue warp 0..7: warps 0-3 take channels 0..63, 4-7 channels 64..127
-    const int q_lo = (ew >> 2) * 2;
+    constexpr int NQ = CH / 64;                           // 32-channel chunks per thread
+    const int q_lo = (ew >> 2) * NQ;
     // Grid offset of the warp's first row (tile row 32 quarter) from the tile origin: the warp's 32
     // rows are the box [32 channels] x [these offsets .. + the extents the store map was built with]
     const int j0 = quarter * 32;
@@ -226,14 +228,14 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     const int Lhw = dm.L[1] * dm.L[2], Mhw = dm.M[1] * dm.M[2];
     // (SPLIT) lane k of a warp accumulates the energies of channels 32 q + 2 (k % 16) + {0, 1} over the
     // warp's rows of parity k / 16: ea = mid + high rows, em = mid rows
-    float ea[2][2] = {}, em[2][2] = {};                   // [chunk of the thread][channel of the pair]
+    float ea[NQ][2] = {}, em[NQ][2] = {};                 // [chunk of the thread][channel of the pair]
     int e_sample = -1;
     unsigned it = 0;
     bool ok = true;
     auto flush_energy = [&]() {
       if (e_sample >= 0 && P.energy) {
 #pragma unroll
-        for (int qi = 0; qi < 2; ++qi)
+        for (int qi = 0; qi < NQ; ++qi)
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
             const int c = (q_lo + qi) * 32 + 2 * (lane & 15) + e;
@@ -288,14 +290,14 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
       const int out_slice = P.mode == MODE_LAST ? th : gi;
       const unsigned nonlow_rows = __ballot_sync(0xffffffffu, band > 0), mid_rows = __ballot_sync(0xffffffffu, band == 1);
       // both 32-channel chunks of the row at once; the accumulator buffer is free as soon as they are read
-      uint32_t rr2[2][32];
-      tmem_ld32(tm + lane_addr + ab * 128 + q_lo * 32, rr2[0]);
-      tmem_ld32(tm + lane_addr + ab * 128 + q_lo * 32 + 32, rr2[1]);
+      uint32_t rr2[NQ][32];
+#pragma unroll
+      for (int qi = 0; qi < NQ; ++qi) tmem_ld32(tm + lane_addr + ab * 128 + (q_lo + qi) * 32, rr2[qi]);
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(&sh.acc_empty[ab]);
 #pragma unroll
-      for (int qi = 0; qi < 2; ++qi) {
+      for (int qi = 0; qi < NQ; ++qi) {
         const int q = q_lo + qi;
         uint32_t (&r)[32] = rr2[qi];
         if (row_f32) {
@@ -398,13 +400,14 @@ constexpr int LOW_TG = 4;
 // LOW_CT = k_t chunk: the smallest of 2, 4, 8 that covers L_t keeps the accumulators (and with them
 // the registers per thread) small, so that more CTAs are resident and more loads in flight.
 template <int LOW_CT>
-__global__ void __launch_bounds__(CH * LOW_TG) low_band_kernel(const float* side, const float* CT, const float* CHm,
+__global__ void __launch_bounds__(CH_MAX * LOW_TG) low_band_kernel(const float* side, const float* CT, const float* CHm,
                                                                float* spec_low, double* energy, FFDims dm, int group_start) {
   const int kw = blockIdx.x;
   const int gi = blockIdx.y, th = group_start + gi;
+  const int CH = dm.d;                                   // threads = d x LOW_TG
   const int c = threadIdx.x % CH, tg = threadIdx.x / CH;
   __shared__ float ch_rows[LOW_CH][128];          // C_H rows of the current k_h chunk
-  __shared__ float red[LOW_CT * LOW_CH][CH];
+  __shared__ float red[LOW_CT * LOW_CH][CH_MAX];
   float e = 0.f;
   for (int kh0 = 0; kh0 < dm.L[1]; kh0 += LOW_CH) {
     __syncthreads();
@@ -476,8 +479,9 @@ bool encode_grid_map(CUtensorMap* map, const void* base, const FFDims& dm, int s
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", (void**)&enc, cudaEnableDefault, &qr) != cudaSuccess || !enc)
       return false;
   }
-  cuuint64_t dims[5] = {(cuuint64_t)CH, (cuuint64_t)dm.W, (cuuint64_t)dm.H, (cuuint64_t)dm.T, (cuuint64_t)slices};
-  cuuint64_t strides[4] = {(cuuint64_t)CH * 2, (cuuint64_t)dm.W * CH * 2, (cuuint64_t)dm.H * dm.W * CH * 2,
+  const cuuint64_t CH = (cuuint64_t)dm.d;
+  cuuint64_t dims[5] = {CH, (cuuint64_t)dm.W, (cuuint64_t)dm.H, (cuuint64_t)dm.T, (cuuint64_t)slices};
+  cuuint64_t strides[4] = {CH * 2, (cuuint64_t)dm.W * CH * 2, (cuuint64_t)dm.H * dm.W * CH * 2,
                            (cuuint64_t)dm.N * CH * 2};
   const int n = axis == 2 ? dm.W : (axis == 1 ? dm.H : dm.T);
   const int kf = TILE_ROWS / n;
@@ -499,8 +503,9 @@ bool encode_store_map(CUtensorMap* map, const void* base, const FFDims& dm, int 
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", (void**)&enc, cudaEnableDefault, &qr) != cudaSuccess || !enc)
       return false;
   }
-  cuuint64_t dims[5] = {(cuuint64_t)CH, (cuuint64_t)dm.W, (cuuint64_t)dm.H, (cuuint64_t)dm.T, (cuuint64_t)slices};
-  cuuint64_t strides[4] = {(cuuint64_t)CH * 2, (cuuint64_t)dm.W * CH * 2, (cuuint64_t)dm.H * dm.W * CH * 2,
+  const cuuint64_t CH = (cuuint64_t)dm.d;
+  cuuint64_t dims[5] = {CH, (cuuint64_t)dm.W, (cuuint64_t)dm.H, (cuuint64_t)dm.T, (cuuint64_t)slices};
+  cuuint64_t strides[4] = {CH * 2, (cuuint64_t)dm.W * CH * 2, (cuuint64_t)dm.H * dm.W * CH * 2,
                            (cuuint64_t)dm.N * CH * 2};
   const int n = axis == 2 ? dm.W : (axis == 1 ? dm.H : dm.T);
   const int kf = TILE_ROWS / n;
@@ -527,11 +532,13 @@ cudaError_t launch_pass(ff_plan* p, const CUtensorMap& m0, const CUtensorMap& m1
   if (nstage > MAX_STAGE) nstage = MAX_STAGE;
   P.nstage = nstage;
   const size_t smem = nstage * stage + fixed;
-  cudaError_t e = cudaFuncSetAttribute(dct_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(dct_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(dct_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int stages = (int)(P.group * (P.dm.N / TILE_ROWS));
   const int grid = stages < p->sm_count ? stages : p->sm_count;
-  dct_tc_kernel<<<grid, DCT_TC_THREADS, smem, st>>>(m0, m1, m2, moh, mol, P);
+  if (P.dm.d == 128) dct_tc_kernel<128><<<grid, DCT_TC_THREADS, smem, st>>>(m0, m1, m2, moh, mol, P);
+  else dct_tc_kernel<64><<<grid, DCT_TC_THREADS, smem, st>>>(m0, m1, m2, moh, mol, P);
   p->launches += 1;
   return cudaGetLastError();
 }
@@ -542,7 +549,7 @@ bool axis_ok(int n) { return n == 16 || n == 32 || n == 64 || n == 128; }
 
 // bf16, head_dim 128, power-of-two axis lengths 16..128, low box small enough for the fp32 side path.
 bool ffk_dct_tc_supported(const FFDims& dm) {
-  if (dm.fp32 || dm.d != CH || !axis_ok(dm.T) || !axis_ok(dm.H) || !axis_ok(dm.W)) return false;
+  if (dm.fp32 || (dm.d != 128 && dm.d != 64) || !axis_ok(dm.T) || !axis_ok(dm.H) || !axis_ok(dm.W)) return false;
   // a tile groups 128/n lines: consecutive h for the w pass, consecutive w for the h and t passes
   return dm.H % (TILE_ROWS / dm.W) == 0 && dm.W % (TILE_ROWS / dm.H) == 0 && dm.W % (TILE_ROWS / dm.T) == 0;
 }
@@ -578,8 +585,8 @@ bool ffk_dct_tc_build_image(ff_plan* p, int axis, int inverse, const float* mat,
 
 // Scratch: two hi/lo pairs of bf16 grids and the fp32 side buffer for `group` tensor-heads.
 size_t ffk_dct_tc_scratch_bytes(const FFDims& dm, int group) {
-  const size_t grid = (size_t)group * dm.N * CH * 2;
-  const size_t side = (size_t)group * dm.T * dm.H * dm.L[2] * CH * 4;
+  const size_t grid = (size_t)group * dm.N * dm.d * 2;
+  const size_t side = (size_t)group * dm.T * dm.H * dm.L[2] * dm.d * 4;
   const size_t ring = ffk_dct_wh_supported(dm) ? ffk_dct_wh_scratch_bytes(dm, group) : 0;
   return 4 * ((grid + 255) / 256 * 256) + (side + 255) / 256 * 256 + (ring + 255) / 256 * 256;
 }
@@ -587,13 +594,13 @@ size_t ffk_dct_tc_scratch_bytes(const FFDims& dm, int group) {
 namespace {
 struct Scratch { __nv_bfloat16 *a_hi, *a_lo, *b_hi, *b_lo; float* side; void* ring; };
 Scratch carve(ff_plan* p) {
-  const size_t grid_bytes = ((size_t)p->dct_group * p->dm.N * CH * 2 + 255) / 256 * 256;
+  const size_t grid_bytes = ((size_t)p->dct_group * p->dm.N * p->dm.d * 2 + 255) / 256 * 256;
   char* base = (char*)p->buf.scratchA;
   Scratch s;
   s.a_hi = (__nv_bfloat16*)base; s.a_lo = (__nv_bfloat16*)(base + grid_bytes);
   s.b_hi = (__nv_bfloat16*)(base + 2 * grid_bytes); s.b_lo = (__nv_bfloat16*)(base + 3 * grid_bytes);
   s.side = (float*)(base + 4 * grid_bytes);
-  const size_t side_bytes = ((size_t)p->dct_group * p->dm.T * p->dm.H * p->dm.L[2] * CH * 4 + 255) / 256 * 256;
+  const size_t side_bytes = ((size_t)p->dct_group * p->dm.T * p->dm.H * p->dm.L[2] * p->dm.d * 4 + 255) / 256 * 256;
   s.ring = base + 4 * grid_bytes + side_bytes;
   return s;
 }
@@ -642,9 +649,9 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
     e = launch_pass(p, m2h, m2l, m2l, m2h, m2l, P, st);    // (no tensor stores in this mode)
     if (e != cudaSuccess) return e;
     dim3 lgrid((unsigned)dm.L[2], (unsigned)g);
-    if (dm.L[0] <= 2) low_band_kernel<2><<<lgrid, CH * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
-    else if (dm.L[0] <= 4) low_band_kernel<4><<<lgrid, CH * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
-    else low_band_kernel<8><<<lgrid, CH * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
+    if (dm.L[0] <= 2) low_band_kernel<2><<<lgrid, dm.d * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
+    else if (dm.L[0] <= 4) low_band_kernel<4><<<lgrid, dm.d * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
+    else low_band_kernel<8><<<lgrid, dm.d * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
     p->launches += 1;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;

@@ -641,14 +641,23 @@ cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// Generic exchange + recombination into the hi/lo bf16 grids of the tensor-core inverse; DPL = d / 32.
+template <int DPL>
+static cudaError_t exchange_to_grids(ff_plan* p, dim3 grid, size_t smem, int h0, __nv_bfloat16* ghi, __nv_bfloat16* glo,
+                                     int low_only, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(exchange_recombine_kernel<__nv_bfloat16, DPL, __nv_bfloat16>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  exchange_recombine_kernel<__nv_bfloat16, DPL, __nv_bfloat16><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, p->dm, h0, ghi, glo, low_only);
+  return cudaGetLastError();
+}
+
 // Tensor-core inverse: exchange + recombination into a bf16 grid, then the three axis passes.
 static cudaError_t exchange_inverse_tc(ff_plan* p, void* out, cudaStream_t st) {
   const FFDims& dm = p->dm;
   const int G = p->dct_group;
   const size_t smem = (size_t)3 * dm.m * dm.d * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(exchange_recombine_kernel<__nv_bfloat16, 4, __nv_bfloat16>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
+  cudaError_t e = cudaSuccess;
   for (int h0 = 0; h0 < dm.BH; h0 += G) {
     const int g = (dm.BH - h0 < G) ? dm.BH - h0 : G;
     dim3 grid((unsigned)((dm.N + EXC_WARPS - 1) / EXC_WARPS), (unsigned)g);
@@ -658,12 +667,10 @@ static cudaError_t exchange_inverse_tc(ff_plan* p, void* out, cudaStream_t st) {
     if (p->xtc_ok) {
       // mid and high bands on the tensor cores, the (small, fp32) low band with the generic kernel
       dim3 lgrid((unsigned)((dm.Nlow + EXC_WARPS - 1) / EXC_WARPS), (unsigned)g);
-      exchange_recombine_kernel<__nv_bfloat16, 4, __nv_bfloat16><<<lgrid, EXC_WARPS * 32, smem, st>>>(p->buf, dm, h0, ghi, glo, 1);
-      e = cudaGetLastError();
+      e = dm.d == 128 ? exchange_to_grids<4>(p, lgrid, smem, h0, ghi, glo, 1, st) : exchange_to_grids<2>(p, lgrid, smem, h0, ghi, glo, 1, st);
       if (e == cudaSuccess) e = ffk_exchange_tc(p, h0, g, ghi, glo, st);
     } else {
-      exchange_recombine_kernel<__nv_bfloat16, 4, __nv_bfloat16><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, dm, h0, ghi, glo, 0);
-      e = cudaGetLastError();
+      e = dm.d == 128 ? exchange_to_grids<4>(p, grid, smem, h0, ghi, glo, 0, st) : exchange_to_grids<2>(p, grid, smem, h0, ghi, glo, 0, st);
     }
     if (e != cudaSuccess) return e;
     p->launches += 1;

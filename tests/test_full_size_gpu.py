@@ -91,3 +91,8 @@ def test_1m_full():
 
 def test_128k_sweep_full():
     _run_full(C.G128K, [0, 1, 2, 3, 4], per_band=1)
+
+
+def test_paper_reference_64k_full():
+    """The paper's reference parameterisation (d_k 64, N/32 low band, w 64, degree-256 mid pattern)."""
+    _run_full(C.PAPER_REF_64K, [0], per_band=1)

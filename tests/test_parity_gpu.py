@@ -141,10 +141,12 @@ def test_transform_tile_geometries(cfg):
 
 
 def test_paper_reference_parameterisation_replica():
-    """d_k = 64, N_low_bar = N / 32, w = 64, constant-degree mid pattern (generic kernels)."""
+    """d_k = 64, N_low_bar = N / 32, w = 64, constant-degree mid pattern: the head_dim 64 variants of
+    the tensor-core transform and attention kernels, and the generic kernels on the same inputs."""
     cfg = C.R_PAPER_REF
     _run(cfg, alloc=[1, 2, 4, 7])
     _run(cfg)                                   # routed
+    _run(cfg, alloc=[7, 4, 2, 1], impl=3)       # generic attention and transform
 
 
 def test_replica_simt_attention_matches_too():
