@@ -1,5 +1,6 @@
 // Cross-band residual exchange + recombination on the tensor cores ("Cross-band residual
-// exchange", "Reconstruction"), bf16 storage, head_dim 128, for the mid and high bands:
+// exchange", "Reconstruction"), bf16 storage, head_dim 128 or 64 (template parameter XD), for the
+// mid and high bands:
 //     Y^[p] = Y[p] + softmax(Y[p] Z^T / sqrt(d)) Z,   Z = the 2m summary tokens of the other two bands
 // written to the coefficient grid at the position of band rank p (a table built at plan creation).
 //
@@ -26,8 +27,8 @@ using namespace sm100;
 namespace {
 
 constexpr int XT = 128;                 // tokens per tile
-constexpr int XD = 128;                 // head_dim
-constexpr int X_TILE_BYTES = XT * XD * 2;
+constexpr int XD_MAX = 128;             // largest head_dim; the shared-memory tiles are sized for it
+constexpr int X_TILE_BYTES = XT * XD_MAX * 2;
 constexpr int X_HALF = X_TILE_BYTES / 2;
 constexpr int X_THREADS = 320;           // TMA warp, MMA warp, 4 softmax warps, 4 store warps
 
@@ -76,7 +77,7 @@ __device__ __forceinline__ XItem x_decode(const FFDims& dm, int h0, int it, int 
 // NK32 = 32-key chunks of the score row that are in use (3m <= 32 NK32).
 // (With three chunks the score row does not fit the registers two resident CTAs leave a thread, so
 // that variant runs one CTA per SM.)
-template <int NK32>
+template <int NK32, int XD>
 __global__ void __launch_bounds__(X_THREADS, NK32 == 3 ? 1 : 2)
 exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_constant__ CUtensorMap map_v_mid,
                    const __grid_constant__ CUtensorMap map_y_high, const __grid_constant__ CUtensorMap map_v_high,
@@ -124,9 +125,9 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         const int slot = n % YB;
         if (n >= YB) ok = mbar_wait(&sh.y_empty[slot], ((n / YB) - 1) & 1, abort_flag);
         if (!ok) break;
-        mbar_arrive_expect_tx(&sh.y_full[slot], X_TILE_BYTES);
+        mbar_arrive_expect_tx(&sh.y_full[slot], XT * XD * 2);
         tma_load_3d(sY + slot * X_TILE_BYTES, map, &sh.y_full[slot], 0, x.tile * XT, slice);
-        tma_load_3d(sY + slot * X_TILE_BYTES + X_HALF, map, &sh.y_full[slot], 64, x.tile * XT, slice);
+        if (XD == 128) tma_load_3d(sY + slot * X_TILE_BYTES + X_HALF, map, &sh.y_full[slot], 64, x.tile * XT, slice);
       }
     }
   } else if (warp == 1) {
@@ -149,7 +150,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         tc_fence_after();
         const uint32_t ybase = smem_u32(sY + slot * X_TILE_BYTES);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {                     // S = Y (Zhi + Zlo)^T, K = head_dim
+        for (int k = 0; k < XD / 16; ++k) {               // S = Y (Zhi + Zlo)^T, K = head_dim
           const uint64_t a = smem_desc_sw128(ybase + (k >> 2) * X_HALF + (k & 3) * 32, 16, 1024);
           const uint32_t zo = (k >> 2) * zhalf + (k & 3) * 32;
           umma_ss(tmem, a, smem_desc_sw128(zhi + zo, 16, 1024), idesc1, k > 0 ? 1u : 0u);
@@ -191,7 +192,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         }
         const float* S = P.summary + (size_t)x.bh * 3 * m * XD;
         for (int idx = tid; idx < nk * XD; idx += 128) {
-          const int j = idx >> 7, c = idx & 127;
+          const int j = idx / XD, c = idx % XD;
           const float v = j < 3 * m ? S[j * XD + c] : 0.f;
           const __nv_bfloat16 hi = __float2bfloat16_rn(v);
           const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
@@ -279,7 +280,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       uint8_t* st_hi = sh.stage[quarter][0];
       uint8_t* st_lo = sh.stage[quarter][1];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+      for (int q = 0; q < XD / 32; ++q) {
         uint32_t r[32];
         tmem_ld32(tmem + lane_addr + 128 + q * 32, r);
         tmem_wait_ld();
@@ -340,15 +341,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-bool encode_rows_map(CUtensorMap* map, void* base, long long rows, int slices) {
+bool encode_rows_map(CUtensorMap* map, void* base, long long rows, int slices, int d) {
   static EncodeTiledFn enc = nullptr;
   if (!enc) {
     cudaDriverEntryPointQueryResult qr;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", (void**)&enc, cudaEnableDefault, &qr) != cudaSuccess || !enc)
       return false;
   }
-  cuuint64_t dims[3] = {(cuuint64_t)XD, (cuuint64_t)rows, (cuuint64_t)slices};
-  cuuint64_t strides[2] = {(cuuint64_t)XD * 2, (cuuint64_t)rows * XD * 2};
+  cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)slices};
+  cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)rows * d * 2};
   cuuint32_t box[3] = {64, XT, 1};
   cuuint32_t es[3] = {1, 1, 1};
   return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -358,7 +359,7 @@ bool encode_rows_map(CUtensorMap* map, void* base, long long rows, int slices) {
 }  // namespace
 
 bool ffk_exchange_tc_supported(const FFDims& dm) {
-  return !dm.fp32 && dm.d == XD && dm.m >= 1 && dm.m <= 32 && dm.N < (1LL << 31);
+  return !dm.fp32 && (dm.d == 128 || dm.d == 64) && dm.m >= 1 && dm.m <= 32 && dm.N < (1LL << 31);
 }
 
 // Rank -> flat coefficient index tables of the mid and high bands (plan-owned device memory).
@@ -383,10 +384,10 @@ bool ffk_exchange_tc_build_tables(ff_plan* p) {
 
 bool ffk_exchange_tc_prepare(ff_plan* p) {
   const FFDims& dm = p->dm;
-  return encode_rows_map((CUtensorMap*)p->tmap_x[0], p->buf.y_mid, dm.Nmid, dm.BH) &&
-         encode_rows_map((CUtensorMap*)p->tmap_x[1], p->buf.spec_mid, dm.Nmid, 3 * dm.BH) &&
-         encode_rows_map((CUtensorMap*)p->tmap_x[2], p->buf.y_high, dm.Nhigh, dm.BH) &&
-         encode_rows_map((CUtensorMap*)p->tmap_x[3], p->buf.spec_high, dm.Nhigh, 3 * dm.BH);
+  return encode_rows_map((CUtensorMap*)p->tmap_x[0], p->buf.y_mid, dm.Nmid, dm.BH, dm.d) &&
+         encode_rows_map((CUtensorMap*)p->tmap_x[1], p->buf.spec_mid, dm.Nmid, 3 * dm.BH, dm.d) &&
+         encode_rows_map((CUtensorMap*)p->tmap_x[2], p->buf.y_high, dm.Nhigh, dm.BH, dm.d) &&
+         encode_rows_map((CUtensorMap*)p->tmap_x[3], p->buf.spec_high, dm.Nhigh, 3 * dm.BH, dm.d);
 }
 
 // Exchange + recombination of the mid and high bands of heads [h0, h0+g) into the hi/lo grids.
@@ -402,19 +403,25 @@ cudaError_t ffk_exchange_tc(ff_plan* p, int h0, int g, void* grid_hi, void* grid
   const int per_sm = P.nkeys > 64 ? 1 : 2;
   P.ybufs = (2 * X_TILE_BYTES + 4 * P.nkeys * 128 + sizeof(XShared) + 2048) * per_sm <= 227 * 1024 ? 2 : 1;
   const size_t smem = P.ybufs * X_TILE_BYTES + 4 * P.nkeys * 128 + sizeof(XShared) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(exchange_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(exchange_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(exchange_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
   const long long tiles = (long long)g * ((dm.Nmid + XT - 1) / XT + (dm.Nhigh + XT - 1) / XT);
   const int grid = tiles < per_sm * p->sm_count ? (int)tiles : per_sm * p->sm_count;
   const CUtensorMap& m0 = *(const CUtensorMap*)p->tmap_x[0];
   const CUtensorMap& m1 = *(const CUtensorMap*)p->tmap_x[1];
   const CUtensorMap& m2 = *(const CUtensorMap*)p->tmap_x[2];
   const CUtensorMap& m3 = *(const CUtensorMap*)p->tmap_x[3];
-  if (P.nkeys <= 32) exchange_tc_kernel<1><<<grid, X_THREADS, smem, st>>>(m0, m1, m2, m3, P);
-  else if (P.nkeys <= 64) exchange_tc_kernel<2><<<grid, X_THREADS, smem, st>>>(m0, m1, m2, m3, P);
-  else exchange_tc_kernel<3><<<grid, X_THREADS, smem, st>>>(m0, m1, m2, m3, P);
+  cudaError_t e = cudaSuccess;
+#define FF_XCH(NK, D)                                                                                              \
+  do {                                                                                                             \
+    e = cudaFuncSetAttribute(exchange_tc_kernel<NK, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);   \
+    if (e == cudaSuccess) exchange_tc_kernel<NK, D><<<grid, X_THREADS, smem, st>>>(m0, m1, m2, m3, P);             \
+  } while (0)
+  if (dm.d == 128) {
+    if (P.nkeys <= 32) FF_XCH(1, 128); else if (P.nkeys <= 64) FF_XCH(2, 128); else FF_XCH(3, 128);
+  } else {
+    if (P.nkeys <= 32) FF_XCH(1, 64); else if (P.nkeys <= 64) FF_XCH(2, 64); else FF_XCH(3, 64);
+  }
+#undef FF_XCH
+  if (e != cudaSuccess) return e;
   p->launches += 1;
   return cudaGetLastError();
 }
