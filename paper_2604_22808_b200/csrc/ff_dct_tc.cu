@@ -28,7 +28,9 @@
 //               from which the low band is computed at full precision
 //        MIDDLE hi/lo intermediate -> hi/lo intermediate
 //        SPLIT  intermediate -> band-major mid/high coefficient buffers (rank evaluated in
-//               registers) with the router's band energies accumulated from the stored (bf16) coefficients
+//               registers) with the router's band energies accumulated from the stored (bf16) coefficients;
+//               for a low box wider than W/4 also the low band, in fp32 from the accumulators (the
+//               fp32 side rows and the low-band kernel are then skipped)
 //        LAST   intermediate -> the caller's out tensor
 #include <cuda.h>
 
@@ -63,6 +65,8 @@ struct DctTcParams {
   int nstage;              // ring depth
   float* side;             // MODE_FIRST: [group][T][H][L_w][128] fp32
   __nv_bfloat16* spec_mid; __nv_bfloat16* spec_high;
+  float* spec_low;         // MODE_SPLIT with low_from_acc: [3 BH][N_low][d] fp32
+  int low_from_acc;        // the low band comes from the band-split pass's accumulators, not from the fp32 side rows
   double* energy;          // [B][3][128]
   int* status;
 };
@@ -113,7 +117,8 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
 // Three source maps (Q, K, V) in MODE_FIRST; otherwise map0 (= hi) and, for split input, map1 (= lo).
 // map_oh / map_ol: destination hi / lo grids with the box of one epilogue warp (32 positions x 32
 // channels), all modes but SPLIT; MODE_LAST has no lo grid.
-template <int CH>
+// LOWACC: the low band comes from this kernel's band-split pass (see DctTcParams::low_from_acc).
+template <int CH, bool LOWACC>
 __global__ void __launch_bounds__(DCT_TC_THREADS, 1)
 dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
               const __grid_constant__ CUtensorMap map2, const __grid_constant__ CUtensorMap map_oh,
@@ -228,7 +233,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     const int Lhw = dm.L[1] * dm.L[2], Mhw = dm.M[1] * dm.M[2];
     // (SPLIT) lane k of a warp accumulates the energies of channels 32 q + 2 (k % 16) + {0, 1} over the
     // warp's rows of parity k / 16: ea = mid + high rows, em = mid rows
-    float ea[NQ][2] = {}, em[NQ][2] = {};                 // [chunk of the thread][channel of the pair]
+    float ea[NQ][2] = {}, em[NQ][2] = {}, el[NQ][2] = {};  // [chunk of the thread][channel of the pair]; el = low rows
     int e_sample = -1;
     unsigned it = 0;
     bool ok = true;
@@ -241,7 +246,8 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
             const int c = (q_lo + qi) * 32 + 2 * (lane & 15) + e;
             atomicAdd(P.energy + ((size_t)e_sample * 3 + 1) * CH + c, (double)em[qi][e]);
             atomicAdd(P.energy + ((size_t)e_sample * 3 + 2) * CH + c, (double)(ea[qi][e] - em[qi][e]));
-            ea[qi][e] = em[qi][e] = 0.f;
+            if (LOWACC) atomicAdd(P.energy + ((size_t)e_sample * 3 + 0) * CH + c, (double)el[qi][e]);
+            ea[qi][e] = em[qi][e] = el[qi][e] = 0.f;
           }
       }
     };
@@ -267,7 +273,9 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
         const int offM = (h < dm.M[1] ? h : dm.M[1]) * dm.M[2] + (h < dm.M[1] ? (ww < dm.M[2] ? ww : dm.M[2]) : 0);
         const long long cm = kt < dm.M[0] ? (long long)kt * Mhw + offM : (long long)dm.M[0] * Mhw;
         if (kt < dm.L[0] && hw_low) {
-          band = 0;                                                                  // low band: fp32 path
+          band = 0;                                                                  // low band: fp32
+          if (LOWACC)
+            row_f32 = P.spec_low + (((size_t)tensor * dm.BH + bh) * dm.Nlow + ((long long)kt * dm.L[1] + h) * dm.L[2] + ww) * CH;
         } else if (kt < dm.M[0] && hw_mid) {
           const int offL = (h < dm.L[1] ? h : dm.L[1]) * dm.L[2] + (h < dm.L[1] ? (ww < dm.L[2] ? ww : dm.L[2]) : 0);
           const long long cl = kt < dm.L[0] ? (long long)kt * Lhw + offL : dm.Nlow;
@@ -277,7 +285,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
           band = 2;
           row_hi = P.spec_high + (((size_t)tensor * dm.BH + bh) * dm.Nhigh + ((((long long)kt * dm.H + h) * dm.W + ww) - cm)) * CH;
         }
-      } else if (P.mode == MODE_FIRST && a < dm.L[2]) {
+      } else if (P.mode == MODE_FIRST && a < dm.L[2] && !LOWACC) {
         row_f32 = P.side + ((((size_t)gi * dm.T + t) * dm.H + h + l) * dm.L[2] + a) * CH;
       }
       // (SPLIT) lane L stores for rows 8 i + L/4 of its warp: fetch those rows' destinations
@@ -360,6 +368,16 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
                 if ((md >> (2 * i)) & 1) { m0 += s0; m1 += s1; }
               }
               ea[qi][0] += a0; ea[qi][1] += a1; em[qi][0] += m0; em[qi][1] += m1;
+              if (LOWACC && nonlow_rows != 0xffffffffu) {       // the warp holds low-band rows (rare)
+                float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                  const uint32_t wd = *(const uint32_t*)(st_hi + (2 * i + par) * STG_PITCH + (((cp >> 2) ^ (i & 3)) << 4) + (cp & 3) * 4);
+                  const float v0 = __uint_as_float(wd << 16), v1 = __uint_as_float(wd & 0xffff0000u);
+                  if (!((nl >> (2 * i)) & 1)) { l0 = fmaf(v0, v0, l0); l1 = fmaf(v1, v1, l1); }
+                }
+                el[qi][0] += l0; el[qi][1] += l1;
+              }
             }
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -399,15 +417,14 @@ constexpr int LOW_TG = 4;
 
 // LOW_CT = k_t chunk: the smallest of 2, 4, 8 that covers L_t keeps the accumulators (and with them
 // the registers per thread) small, so that more CTAs are resident and more loads in flight.
-template <int LOW_CT>
-__global__ void __launch_bounds__(CH_MAX * LOW_TG) low_band_kernel(const float* side, const float* CT, const float* CHm,
+template <int LOW_CT, int CH>
+__global__ void __launch_bounds__(CH * LOW_TG) low_band_kernel(const float* side, const float* CT, const float* CHm,
                                                                float* spec_low, double* energy, FFDims dm, int group_start) {
   const int kw = blockIdx.x;
   const int gi = blockIdx.y, th = group_start + gi;
-  const int CH = dm.d;                                   // threads = d x LOW_TG
-  const int c = threadIdx.x % CH, tg = threadIdx.x / CH;
+  const int c = threadIdx.x % CH, tg = threadIdx.x / CH;     // threads = d x LOW_TG
   __shared__ float ch_rows[LOW_CH][128];          // C_H rows of the current k_h chunk
-  __shared__ float red[LOW_CT * LOW_CH][CH_MAX];
+  __shared__ float red[LOW_CT * LOW_CH][CH];
   float e = 0.f;
   for (int kh0 = 0; kh0 < dm.L[1]; kh0 += LOW_CH) {
     __syncthreads();
@@ -532,13 +549,18 @@ cudaError_t launch_pass(ff_plan* p, const CUtensorMap& m0, const CUtensorMap& m1
   if (nstage > MAX_STAGE) nstage = MAX_STAGE;
   P.nstage = nstage;
   const size_t smem = nstage * stage + fixed;
-  cudaError_t e = cudaFuncSetAttribute(dct_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(dct_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
+  cudaError_t e = cudaSuccess;
   const int stages = (int)(P.group * (P.dm.N / TILE_ROWS));
   const int grid = stages < p->sm_count ? stages : p->sm_count;
-  if (P.dm.d == 128) dct_tc_kernel<128><<<grid, DCT_TC_THREADS, smem, st>>>(m0, m1, m2, moh, mol, P);
-  else dct_tc_kernel<64><<<grid, DCT_TC_THREADS, smem, st>>>(m0, m1, m2, moh, mol, P);
+#define FF_DCT(D, LA)                                                                                              \
+  do {                                                                                                             \
+    e = cudaFuncSetAttribute(dct_tc_kernel<D, LA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
+    if (e == cudaSuccess) dct_tc_kernel<D, LA><<<grid, DCT_TC_THREADS, smem, st>>>(m0, m1, m2, moh, mol, P);       \
+  } while (0)
+  if (P.dm.d == 128) { if (P.low_from_acc) FF_DCT(128, true); else FF_DCT(128, false); }
+  else { if (P.low_from_acc) FF_DCT(64, true); else FF_DCT(64, false); }
+#undef FF_DCT
+  if (e != cudaSuccess) return e;
   p->launches += 1;
   return cudaGetLastError();
 }
@@ -627,6 +649,10 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
   P.dm = dm; P.status = p->buf.status;
   P.spec_mid = (__nv_bfloat16*)p->buf.spec_mid; P.spec_high = (__nv_bfloat16*)p->buf.spec_high;
   P.energy = want_energy ? p->buf.energy : nullptr;
+  // A low box wider than a quarter of the w axis would make the fp32 side rows a large extra copy of the
+  // data: take the low band from the tensor-core accumulators of the last pass instead.
+  P.low_from_acc = dm.L[2] * 4 > dm.W;
+  P.spec_low = p->buf.spec_low;
   for (int g0 = 0; g0 < total; g0 += G) {
     const int g = total - g0 < G ? total - g0 : G;
     P.group = g; P.group_start = g0;
@@ -649,9 +675,11 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
     e = launch_pass(p, m2h, m2l, m2l, m2h, m2l, P, st);    // (no tensor stores in this mode)
     if (e != cudaSuccess) return e;
     dim3 lgrid((unsigned)dm.L[2], (unsigned)g);
-    if (dm.L[0] <= 2) low_band_kernel<2><<<lgrid, dm.d * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
-    else if (dm.L[0] <= 4) low_band_kernel<4><<<lgrid, dm.d * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
-    else low_band_kernel<8><<<lgrid, dm.d * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0);
+    if (P.low_from_acc) continue;                  // the band-split pass has written the low band already
+#define FF_LOW(CT, D) low_band_kernel<CT, D><<<lgrid, D * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0)
+    if (dm.d == 128) { if (dm.L[0] <= 2) FF_LOW(2, 128); else if (dm.L[0] <= 4) FF_LOW(4, 128); else FF_LOW(8, 128); }
+    else { if (dm.L[0] <= 2) FF_LOW(2, 64); else if (dm.L[0] <= 4) FF_LOW(4, 64); else FF_LOW(8, 64); }
+#undef FF_LOW
     p->launches += 1;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
