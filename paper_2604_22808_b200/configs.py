@@ -105,8 +105,9 @@ PAPER_REF_64K = FFConfig(name="paper_ref_64k", batch=1, T=16, H=64, W=64, heads=
                          low_cut=(8, 32, 32), mid_cut=(13, 51, 51), r=4, b=32, s=100, R=32, m=8, seed=5,
                          timesteps=(500.0,))
 # ... and its replica on a grid the oracle covers in full (axis lengths the tensor-core transform
-# covers): 4096 tokens, N_low_bar = N / 32 = 128, nine blocks per residue class.
-R_PAPER_REF = FFConfig(name="paper_ref_replica", batch=1, T=16, H=16, W=16, heads=4, head_dim=64, dtype="bf16",
-                       low_cut=(8, 8, 8), mid_cut=(13, 13, 13), r=4, b=32, s=6, R=32, m=8, seed=15,
+# covers): 16384 tokens, N_low_bar = N / 32 = 512 (four tiles of the dense low branch), eight or
+# nine blocks per residue class.
+R_PAPER_REF = FFConfig(name="paper_ref_replica", batch=1, T=16, H=32, W=32, heads=4, head_dim=64, dtype="bf16",
+                       low_cut=(8, 16, 16), mid_cut=(13, 26, 26), r=4, b=32, s=26, R=32, m=8, seed=15,
                        timesteps=(500.0,))
 BY_NAME.update({c.name: c for c in (PAPER_REF_64K, R_PAPER_REF)})

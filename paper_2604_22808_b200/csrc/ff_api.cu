@@ -105,7 +105,7 @@ void ff_compute_layout(const FFDims& dm, bool with_staging, FFLayout* lay) {
   if (Gt > 3 * BH) Gt = 3 * BH;
   lay->tc_group = (int)Gt;
   const size_t tc_scratch = ffk_dct_tc_supported(dm) ? ffk_dct_tc_scratch_bytes(dm, (int)Gt) : 0;
-  const size_t sizes[20] = {
+  const size_t sizes[21] = {
       3 * BH * (size_t)dm.Nlow * d * 4,   // 0 spec_low
       3 * BH * (size_t)dm.Nmid * d * e,   // 1 spec_mid
       3 * BH * (size_t)dm.Nhigh * d * e,  // 2 spec_high
@@ -126,9 +126,10 @@ void ff_compute_layout(const FFDims& dm, bool with_staging, FFLayout* lay) {
       with_staging ? BH * (size_t)dm.N * d * e : 0,
       with_staging ? BH * (size_t)dm.N * d * e : 0,
       ffk_tc_work_bytes(),                // 19 worklist
+      dm.fp32 ? 0 : 3 * BH * (size_t)dm.Nbar * d * 2,   // 20 pooled low band as bf16
   };
   size_t off = 0;
-  for (int i = 0; i < 20; ++i) { lay->off[i] = off; off += align_up(sizes[i], 256); }
+  for (int i = 0; i < 21; ++i) { lay->off[i] = off; off += align_up(sizes[i], 256); }
   lay->total = off;
 }
 
@@ -258,6 +259,7 @@ extern "C" ff_status_t ff_plan_set_workspace(ff_plan_t* p, void* ptr, size_t byt
   b.stage_q = p->ws_has_staging ? base + o[15] : nullptr; b.stage_k = p->ws_has_staging ? base + o[16] : nullptr;
   b.stage_v = p->ws_has_staging ? base + o[17] : nullptr; b.stage_out = p->ws_has_staging ? base + o[18] : nullptr;
   b.work = (int*)(base + o[19]);
+  b.pooled_bf = p->dm.fp32 ? nullptr : (__nv_bfloat16*)(base + o[20]);
   FF_CUDA(p, cudaMemset(b.status, 0, 256));
   p->tc_ok = ffk_tc_supported(p->dm) && ffk_tc_prepare(p);
   p->xtc_ok = p->pos_table && ffk_exchange_tc_supported(p->dm) && ffk_exchange_tc_prepare(p);
@@ -388,7 +390,7 @@ extern "C" ff_status_t ff_forward(ff_plan_t* p, const void* Q, const void* K, co
   if (alloc_dev) FF_CUDA(p, cudaMemcpyAsync(p->buf.alloc, alloc_dev, p->dm.BH, cudaMemcpyDeviceToDevice, st));
   FF_CUDA(p, ffk_pool_low(p, st));
   if (p->tc_ok && !(p->attn_impl & 1)) {
-    FF_CUDA(p, ffk_attention_simt(p, FF_BAND_LOW, st));
+    if (!p->low_tc_ok) FF_CUDA(p, ffk_attention_simt(p, FF_BAND_LOW, st));
     FF_CUDA(p, ffk_attention_tc(p, st));
   } else {
     FF_CUDA(p, ffk_attention_simt(p, FF_BAND_LOW | FF_BAND_MID | FF_BAND_HIGH, st));

@@ -1,6 +1,7 @@
-// Mid- and high-band attention on the 5th-generation tensor cores ("Hierarchical frequency-domain
-// attention": strided block-sparse attention on the mid band, sliding-window attention on the high
-// band), bf16 operands, fp32 accumulation, head_dim 128 or 64 (template parameter HD).
+// Band attention on the 5th-generation tensor cores ("Hierarchical frequency-domain attention":
+// strided block-sparse attention on the mid band, sliding-window attention on the high band, and
+// dense attention on the pooled low band when that is at least a tile long), bf16 operands, fp32
+// accumulation, head_dim 128 or 64 (template parameter HD).
 //
 // One persistent launch runs both branches from a worklist of (head, band, pair of query tiles)
 // items that is rebuilt from the head-to-band allocation before every launch.  A CTA owns every
@@ -45,6 +46,8 @@ struct TcParams {
   int* work;          // [0] = number of units, [1] = total items, then offsets[MAX_UNITS+1], desc[MAX_UNITS], tiles[MAX_UNITS]
   __nv_bfloat16* y_mid;
   __nv_bfloat16* y_high;
+  float* y_low;       // [BH][Nbar][d] fp32, written when low_on
+  int low_on;         // heads whose mask has the low band run it here (band code 0: dense over Nbar pooled tokens)
   int* status;
   int rb_mid;         // rows per TMA box of the mid map = min(b, 128)
 };
@@ -82,6 +85,14 @@ __global__ void build_worklist_kernel(TcParams P) {
   int* tiles = desc + MAX_UNITS;
   int nu = 0, total = 0;
   const MidShape ms = mid_shape(dm);
+  if (P.low_on) {
+    const int nt = (int)((dm.Nbar + TILE - 1) / TILE);
+    for (int bh = 0; bh < dm.BH && nu < MAX_UNITS; ++bh) {
+      if (!(P.alloc[bh] & FF_BAND_LOW)) continue;
+      offsets[nu] = total; desc[nu] = (bh << 12); tiles[nu] = nt;
+      total += (nt + 1) / 2; ++nu;
+    }
+  }
   for (int bh = 0; bh < dm.BH && nu < MAX_UNITS; ++bh) {
     if (!(P.alloc[bh] & FF_BAND_MID)) continue;
     offsets[nu] = total; desc[nu] = (bh << 12) | (1 << 10); tiles[nu] = 0;
@@ -113,6 +124,7 @@ struct Shared {
   uint32_t tmem_base;
   int abort_flag;
   int n_units, total;
+  MidShape ms;        // kept here rather than in every thread's registers
   int offsets[MAX_UNITS + 1];
   int desc[MAX_UNITS];
   int ntile[MAX_UNITS];
@@ -121,7 +133,9 @@ struct Shared {
   unsigned long long xsum[2][2][NSPLIT][128];
 };
 
-__device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, const MidShape& ms, int it) {
+template <bool HAS_LOW>
+__device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, int it) {
+  const MidShape& ms = sh.ms;
   int lo = 0, hi = sh.n_units - 1;
   while (lo < hi) {                       // last unit whose offset <= it
     const int mid = (lo + hi + 1) >> 1;
@@ -143,6 +157,12 @@ __device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, 
     x.n = dm.Nmid;
     x.nk = nt;                            // every query tile of a class sees all its key tiles
     x.ks = 0;
+  } else if (HAS_LOW && x.band == 0) {
+    x.tile_a = 2 * local;
+    x.has_b = x.tile_a + 1 < sh.ntile[lo];
+    x.n = dm.Nbar;
+    x.nk = sh.ntile[lo];                  // dense: every query tile sees every key tile
+    x.ks = 0;
   } else {
     x.tile_a = 2 * local;
     x.has_b = x.tile_a + 1 < sh.ntile[lo];
@@ -160,7 +180,7 @@ __device__ __forceinline__ Item decode_item(const Shared& sh, const FFDims& dm, 
 // band: when the tile meets the window of the stream's 128 query rows.
 __device__ __forceinline__ bool stream_active(const Item& x, const FFDims& dm, int sx, int j) {
   if (sx == 1 && !x.has_b) return false;
-  if (x.band == 1) return true;
+  if (x.band != 2) return true;
   const long long t0 = x.ks + (long long)j * TILE;
   const long long q0 = (long long)(x.tile_a + sx) * TILE;
   return t0 <= q0 + TILE - 1 + dm.R && t0 + TILE - 1 >= q0 - dm.R && t0 < x.n;
@@ -179,7 +199,7 @@ __device__ __forceinline__ long long mid_rank(const FFDims& dm, int c, long long
 // `halves` = head_dim / 64.
 __device__ __forceinline__ void load_tile(uint8_t* dst, const CUtensorMap* map, uint64_t* bar, const FFDims& dm,
                                           const Item& x, int slice, long long first, int rb, int halves) {
-  if (x.band == 2) {
+  if (x.band != 1) {
     tma_load_3d(dst, map, bar, 0, (int)first, slice);
     if (halves > 1) tma_load_3d(dst + HALF_BYTES, map, bar, 64, (int)first, slice);
   } else {
@@ -230,7 +250,8 @@ __device__ __forceinline__ float ex2(float x) {
 // which hold Q~, K~ and V~ of head bh in slices bh, BH + bh and 2 BH + bh.  QKV_MAPS = true (the entry
 // point that allocates nothing): map_a, map_b, map_c are the caller's separate Q, K, V tensors of one
 // band, head bh in slice bh.
-template <int HD, bool QKV_MAPS>
+// HAS_LOW: the worklist may hold low-band items (band code 0).
+template <int HD, bool QKV_MAPS, bool HAS_LOW>
 __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, const CUtensorMap& map_b,
                                                   const CUtensorMap& map_c, const TcParams& P) {
   extern __shared__ uint8_t smem_raw[];
@@ -256,6 +277,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
     sh.abort_flag = 0;
     sh.n_units = P.work[0];
     sh.total = P.work[1];
+    sh.ms = mid_shape(dm);
     fence_mbar_init();
   }
   __syncthreads();
@@ -276,18 +298,17 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
   tc_fence_after();
   const uint32_t tm = sh.tmem_base;
   const int total = sh.total;
-  const MidShape ms = mid_shape(dm);
   volatile int* abort_flag = &sh.abort_flag;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      tma_prefetch_desc(&map_a); tma_prefetch_desc(&map_b);
+      tma_prefetch_desc(&map_a); tma_prefetch_desc(&map_b); tma_prefetch_desc(&map_c);
       int iter = 0; unsigned g = 0;
       bool ok = true;
       for (int it = blockIdx.x; it < total && ok; it += gridDim.x, ++iter) {
-        const Item x = decode_item(sh, dm, ms, it);
-        const CUtensorMap* map = x.band == 1 ? &map_a : &map_b;
+        const Item x = decode_item<HAS_LOW>(sh, dm, it);
+        const CUtensorMap* map = x.band == 1 ? &map_a : (!HAS_LOW || x.band == 2 || QKV_MAPS ? &map_b : &map_c);
         const CUtensorMap* mapq = QKV_MAPS ? &map_a : map;
         const CUtensorMap* mapk = QKV_MAPS ? &map_b : map;
         const CUtensorMap* mapv = QKV_MAPS ? &map_c : map;
@@ -300,7 +321,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         if (x.has_b) load_tile(sQ + TILE_BYTES, mapq, &sh.q_full, dm, x, x.bh, (long long)(x.tile_a + 1) * TILE, rb, HALVES);
         for (int j = 0; j < x.nk && ok; ++j, ++g) {
           const int st = g & 1;
-          const long long first = x.band == 1 ? (long long)j * TILE : x.ks + (long long)j * TILE;
+          const long long first = x.band == 2 ? x.ks + (long long)j * TILE : (long long)j * TILE;
           if (g >= 2) ok = mbar_wait(&sh.k_empty[st], ((g >> 1) - 1) & 1, abort_flag);
           if (!ok) break;
           mbar_arrive_expect_tx(&sh.k_full[st], TB);
@@ -355,7 +376,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         return true;
       };
       for (int it = blockIdx.x; it < total && ok; it += gridDim.x, ++iter) {
-        const Item x = decode_item(sh, dm, ms, it);
+        const Item x = decode_item<HAS_LOW>(sh, dm, it);
         ok = mbar_wait(&sh.q_full, iter & 1, abort_flag);
         if (!ok) break;
         const unsigned g0 = g;
@@ -417,7 +438,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
     unsigned ci = 0;                  // items this stream has processed
     bool ok = true;
     for (int it = blockIdx.x; it < total && ok; it += gridDim.x) {
-      const Item x = decode_item(sh, dm, ms, it);
+      const Item x = decode_item<HAS_LOW>(sh, dm, it);
       if (sx == 1 && !x.has_b) continue;
       const int tile = x.tile_a + sx;
       // band rank of this thread's query row
@@ -440,6 +461,10 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
             for (int cc = TILE - 1; cc >= 0; --cc)
               if (mid_rank(dm, x.c, u0 + cc) < dm.Nmid) { chi = cc; break; }
           }
+        } else if (HAS_LOW && x.band == 0) {
+          const long long left = x.n - (long long)j * TILE;     // pooled tokens from this tile on
+          full = left >= TILE;
+          if (!full) chi = (int)left - 1;
         } else {
           const long long t0 = x.ks + (long long)j * TILE;
           const long long q0 = (long long)tile * TILE;
@@ -549,12 +574,18 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
       const float inv = 1.f / l;
       const bool store = p < x.n;
       __nv_bfloat16* y = (x.band == 1 ? P.y_mid : P.y_high) + ((size_t)x.bh * x.n + (store ? p : 0)) * HD + ocol0;
+      float* yl = HAS_LOW && x.band == 0 ? P.y_low + ((size_t)x.bh * x.n + (store ? p : 0)) * HD + ocol0 : nullptr;   // low band: fp32
 #pragma unroll
       for (int c = 0; c < OCOLS / 32; ++c) {
         uint32_t r[32];
         tmem_ld32(o_addr + c * 32, r);
         tmem_wait_ld();
-        if (store) {
+        if (store && yl) {
+#pragma unroll
+          for (int v4 = 0; v4 < 8; ++v4)
+            *(float4*)(yl + c * 32 + v4 * 4) = make_float4(__uint_as_float(r[v4 * 4]) * inv, __uint_as_float(r[v4 * 4 + 1]) * inv,
+                                                           __uint_as_float(r[v4 * 4 + 2]) * inv, __uint_as_float(r[v4 * 4 + 3]) * inv);
+        } else if (store) {
 #pragma unroll
           for (int v4 = 0; v4 < 4; ++v4) {
             uint32_t w[4];
@@ -590,18 +621,19 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
   }
 }
 
-template <int HD>
+template <int HD, bool HAS_LOW>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_mid, const __grid_constant__ CUtensorMap map_high,
+                    const __grid_constant__ CUtensorMap map_low,
                     const TcParams P) {
-  attention_tc_body<HD, false>(map_mid, map_high, map_high, P);
+  attention_tc_body<HD, false, HAS_LOW>(map_mid, map_high, map_low, P);
 }
 
 // Same kernel on the caller's separate Q, K, V tensors of one band (see ff_high_attention_noalloc).
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attention_tc_qkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                         const __grid_constant__ CUtensorMap map_v, const TcParams P) {
-  attention_tc_body<HD_MAX, true>(map_q, map_k, map_v, P);
+  attention_tc_body<HD_MAX, true, false>(map_q, map_k, map_v, P);
 }
 
 // Scratch of ff_high_attention_noalloc: the worklist, one band mask per head and a status word.
@@ -649,8 +681,14 @@ bool ffk_tc_prepare(ff_plan* p) {
   static_assert(sizeof(CUtensorMap) <= sizeof(p->tmap_mid), "tensor map storage too small");
   const FFDims& dm = p->dm;
   const int rb = dm.b < TILE ? dm.b : TILE;
-  return encode_band_map((CUtensorMap*)p->tmap_mid, p->buf.spec_mid, dm.Nmid, 3 * dm.BH, rb, dm.d) &&
-         encode_band_map((CUtensorMap*)p->tmap_high, p->buf.spec_high, dm.Nhigh, 3 * dm.BH, TILE, dm.d);
+  if (!encode_band_map((CUtensorMap*)p->tmap_mid, p->buf.spec_mid, dm.Nmid, 3 * dm.BH, rb, dm.d) ||
+      !encode_band_map((CUtensorMap*)p->tmap_high, p->buf.spec_high, dm.Nhigh, 3 * dm.BH, TILE, dm.d))
+    return false;
+  // The low branch joins this launch when the pooled band is at least one tile long (shorter ones
+  // stay on the generic fp32 kernel, which is exact and costs microseconds there).
+  p->low_tc_ok = p->buf.pooled_bf && dm.Nbar >= TILE && dm.Nbar < (1LL << 31) - 256 && (long long)dm.BH * 3 <= MAX_UNITS &&
+                 encode_band_map((CUtensorMap*)p->tmap_low, p->buf.pooled_bf, dm.Nbar, 3 * dm.BH, TILE, dm.d);
+  return true;
 }
 
 cudaError_t ffk_attention_tc(ff_plan* p, cudaStream_t st) {
@@ -658,18 +696,24 @@ cudaError_t ffk_attention_tc(ff_plan* p, cudaStream_t st) {
   TcParams P;
   P.dm = dm; P.alloc = p->buf.alloc; P.work = p->buf.work;
   P.y_mid = (__nv_bfloat16*)p->buf.y_mid; P.y_high = (__nv_bfloat16*)p->buf.y_high;
+  P.y_low = p->buf.y_low; P.low_on = p->low_tc_ok ? 1 : 0;
   P.status = p->buf.status; P.rb_mid = dm.b < TILE ? dm.b : TILE;
   build_worklist_kernel<<<1, 32, 0, st>>>(P);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const size_t smem = 6 * TILE_BYTES + sizeof(Shared) + 1024;
-  e = cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
   const CUtensorMap& mm = *(const CUtensorMap*)p->tmap_mid;
   const CUtensorMap& mh = *(const CUtensorMap*)p->tmap_high;
-  if (dm.d == 128) attention_tc_kernel<128><<<p->sm_count, TC_THREADS, smem, st>>>(mm, mh, P);
-  else attention_tc_kernel<64><<<p->sm_count, TC_THREADS, smem, st>>>(mm, mh, P);
+  const CUtensorMap& ml = p->low_tc_ok ? *(const CUtensorMap*)p->tmap_low : mh;
+#define FF_ATT(D, LOW)                                                                                             \
+  do {                                                                                                             \
+    e = cudaFuncSetAttribute(attention_tc_kernel<D, LOW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+    if (e == cudaSuccess) attention_tc_kernel<D, LOW><<<p->sm_count, TC_THREADS, smem, st>>>(mm, mh, ml, P);       \
+  } while (0)
+  if (dm.d == 128) { if (p->low_tc_ok) FF_ATT(128, true); else FF_ATT(128, false); }
+  else { if (p->low_tc_ok) FF_ATT(64, true); else FF_ATT(64, false); }
+#undef FF_ATT
+  if (e != cudaSuccess) return e;
   p->launches += 2;
   return cudaGetLastError();
 }

@@ -52,6 +52,7 @@ struct FFBuffers {
   void* spec_mid;    // st [3][BH][Nmid][d]
   void* spec_high;   // st [3][BH][Nhigh][d]
   float* pooled;     // [3][BH][Nbar][d]
+  __nv_bfloat16* pooled_bf;  // the same values as bf16, operands of the tensor-core low branch (NULL if unused)
   float* y_low;      // [BH][Nbar][d]
   void* y_mid;       // st [BH][Nmid][d]
   void* y_high;      // st [BH][Nhigh][d]
@@ -103,6 +104,8 @@ struct ff_plan {
   uint8_t* dct_images;                         // 6 x (hi, lo) matrix images of the tensor-core transform (plan-owned)
   alignas(64) unsigned char tmap_mid[128];     // CUtensorMap over the mid-band / high-band coefficient buffers
   alignas(64) unsigned char tmap_high[128];
+  alignas(64) unsigned char tmap_low[128];     // ... over the pooled low band (bf16 copy), when low_tc_ok
+  bool low_tc_ok;                              // the low branch runs in the tensor-core attention launch
   long long launches;
   bool profiling;
   cudaEvent_t ev[FF_STAGE_COUNT + 1];

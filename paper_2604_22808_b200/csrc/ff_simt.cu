@@ -241,7 +241,7 @@ __global__ void router_kernel(const double* energy, const float* timestep, const
 }
 
 // Low-band compression: mean over groups of r consecutive low ranks, for Q~, K~ and V~.
-__global__ void pool_low_kernel(const float* spec_low, float* pooled, FFDims dm) {
+__global__ void pool_low_kernel(const float* spec_low, float* pooled, __nv_bfloat16* pooled_bf, FFDims dm) {
   const long long g = blockIdx.x;
   const int th = blockIdx.y;
   const int c = threadIdx.x;
@@ -250,7 +250,9 @@ __global__ void pool_low_kernel(const float* spec_low, float* pooled, FFDims dm)
   const long long p1 = (p0 + dm.r < dm.Nlow) ? p0 + dm.r : dm.Nlow;
   float acc = 0.f;
   for (long long p = p0; p < p1; ++p) acc += spec_low[((size_t)th * dm.Nlow + p) * dm.d + c];
-  pooled[((size_t)th * dm.Nbar + g) * dm.d + c] = acc / (float)(p1 - p0);
+  const float v = acc / (float)(p1 - p0);
+  pooled[((size_t)th * dm.Nbar + g) * dm.d + c] = v;
+  if (pooled_bf) pooled_bf[((size_t)th * dm.Nbar + g) * dm.d + c] = __float2bfloat16_rn(v);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -592,7 +594,7 @@ cudaError_t ffk_router(ff_plan* p, uint8_t* alloc_out, cudaStream_t st) {
 cudaError_t ffk_pool_low(ff_plan* p, cudaStream_t st) {
   const FFDims& dm = p->dm;
   dim3 grid((unsigned)dm.Nbar, (unsigned)(3 * dm.BH));
-  pool_low_kernel<<<grid, dm.d, 0, st>>>(p->buf.spec_low, p->buf.pooled, dm);
+  pool_low_kernel<<<grid, dm.d, 0, st>>>(p->buf.spec_low, p->buf.pooled, p->low_tc_ok ? p->buf.pooled_bf : nullptr, dm);
   p->launches += 1;
   return cudaGetLastError();
 }
