@@ -110,4 +110,9 @@ PAPER_REF_64K = FFConfig(name="paper_ref_64k", batch=1, T=16, H=64, W=64, heads=
 R_PAPER_REF = FFConfig(name="paper_ref_replica", batch=1, T=16, H=32, W=32, heads=4, head_dim=64, dtype="bf16",
                        low_cut=(8, 16, 16), mid_cut=(13, 26, 26), r=4, b=32, s=26, R=32, m=8, seed=15,
                        timesteps=(500.0,))
-BY_NAME.update({c.name: c for c in (PAPER_REF_64K, R_PAPER_REF)})
+# The same parameterisation at the paper's longest sequence: N = 1,048,576, N_low_bar = 32,768 (the
+# dense low branch is no longer negligible), 1561 residue classes of 7 or 8 blocks.
+PAPER_REF_1M = FFConfig(name="paper_ref_1m", batch=1, T=64, H=128, W=128, heads=16, head_dim=64, dtype="bf16",
+                        low_cut=(32, 64, 64), mid_cut=(51, 102, 102), r=4, b=32, s=1561, R=32, m=8, seed=6,
+                        timesteps=(500.0,))
+BY_NAME.update({c.name: c for c in (PAPER_REF_64K, PAPER_REF_1M, R_PAPER_REF)})

@@ -96,3 +96,8 @@ def test_128k_sweep_full():
 def test_paper_reference_64k_full():
     """The paper's reference parameterisation (d_k 64, N/32 low band, w 64, degree-256 mid pattern)."""
     _run_full(C.PAPER_REF_64K, [0], per_band=1)
+
+
+def test_paper_reference_1m_full():
+    """... at 1M tokens: N_low_bar = 32768 (dense low branch on the tensor cores), 1561 residue classes."""
+    _run_full(C.PAPER_REF_1M, [0], per_band=1)
