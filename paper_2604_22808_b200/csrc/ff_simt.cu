@@ -242,10 +242,11 @@ __global__ void router_kernel(const double* energy, const float* timestep, const
 
 // Low-band compression: mean over groups of r consecutive low ranks, for Q~, K~ and V~.
 __global__ void pool_low_kernel(const float* spec_low, float* pooled, __nv_bfloat16* pooled_bf, FFDims dm) {
-  const long long g = blockIdx.x;
+  // block = (d channels) x (POOL_ROWS pooled tokens)
+  const long long g = (long long)blockIdx.x * blockDim.y + threadIdx.y;
   const int th = blockIdx.y;
   const int c = threadIdx.x;
-  if (c >= dm.d) return;
+  if (c >= dm.d || g >= dm.Nbar) return;
   const long long p0 = g * dm.r;
   const long long p1 = (p0 + dm.r < dm.Nlow) ? p0 + dm.r : dm.Nlow;
   float acc = 0.f;
@@ -593,8 +594,9 @@ cudaError_t ffk_router(ff_plan* p, uint8_t* alloc_out, cudaStream_t st) {
 
 cudaError_t ffk_pool_low(ff_plan* p, cudaStream_t st) {
   const FFDims& dm = p->dm;
-  dim3 grid((unsigned)dm.Nbar, (unsigned)(3 * dm.BH));
-  pool_low_kernel<<<grid, dm.d, 0, st>>>(p->buf.spec_low, p->buf.pooled, p->low_tc_ok ? p->buf.pooled_bf : nullptr, dm);
+  const int rows = dm.d <= 128 ? 512 / dm.d : 1;            // pooled tokens per CTA
+  dim3 grid((unsigned)((dm.Nbar + rows - 1) / rows), (unsigned)(3 * dm.BH)), block((unsigned)dm.d, (unsigned)rows);
+  pool_low_kernel<<<grid, block, 0, st>>>(p->buf.spec_low, p->buf.pooled, p->low_tc_ok ? p->buf.pooled_bf : nullptr, dm);
   p->launches += 1;
   return cudaGetLastError();
 }
