@@ -47,7 +47,7 @@ constexpr int CH_MAX = 128;                          // largest head_dim; shared
 constexpr int TILE_ROWS = 128;
 constexpr int TILE_BYTES = TILE_ROWS * CH_MAX * 2; // 32 KB: 128 rows of bf16
 constexpr int HALF_BYTES = TILE_BYTES / 2;
-constexpr int MAX_STAGE = 4;
+constexpr int MAX_STAGE = 8;
 constexpr int NACC = 4;
 constexpr int DCT_TC_THREADS = 320;        // TMA warp, MMA warp, 8 epilogue warps
 
@@ -133,7 +133,8 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
   const bool seq = P.axis == 2;                           // lines follow one another (w axis) or interleave
   const int NSTAGE = P.nstage;
   const bool tma_out = P.mode != MODE_SPLIT;
-  const int STAGE_BYTES = P.in_split ? 2 * TILE_BYTES : TILE_BYTES;
+  constexpr int TB = TILE_ROWS * CH * 2;                  // bytes of one data tile (16 KB for 64 channels)
+  const int STAGE_BYTES = P.in_split ? 2 * TB : TB;       // hi tile, then lo tile
   uint8_t* sData = smem;                                  // NSTAGE x STAGE_BYTES
   uint8_t* sHi = smem + NSTAGE * STAGE_BYTES;             // matrix hi: [K half][128 rows][128 B], swizzled
   uint8_t* sLo = sHi + TILE_BYTES;                        // matrix lo
@@ -180,12 +181,12 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
           map = tensor == 0 ? &map0 : (tensor == 1 ? &map1 : &map2);
           slice = th % dm.BH;
         }
-        mbar_arrive_expect_tx(&sh.full[slot], (P.in_split ? 2 : 1) * TILE_ROWS * CH * 2);
+        mbar_arrive_expect_tx(&sh.full[slot], STAGE_BYTES);
         tma_load_5d(dst, map, &sh.full[slot], 0, w, h, t, slice);
         if (CH == 128) tma_load_5d(dst + HALF_BYTES, map, &sh.full[slot], 64, w, h, t, slice);
         if (P.in_split) {
-          tma_load_5d(dst + TILE_BYTES, &map1, &sh.full[slot], 0, w, h, t, slice);
-          if (CH == 128) tma_load_5d(dst + TILE_BYTES + HALF_BYTES, &map1, &sh.full[slot], 64, w, h, t, slice);
+          tma_load_5d(dst + TB, &map1, &sh.full[slot], 0, w, h, t, slice);
+          if (CH == 128) tma_load_5d(dst + TB + HALF_BYTES, &map1, &sh.full[slot], 64, w, h, t, slice);
         }
       }
     }
@@ -210,7 +211,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
           const uint64_t xhi = smem_desc_sw128(dbase + ks * 2048, HALF_BYTES, 1024);
           umma_ss(d_tm, ahi, xhi, idesc, ks > 0 ? 1u : 0u);
           umma_ss(d_tm, smem_desc_sw128(lo_base + aoff, 16, 1024), xhi, idesc, 1u);
-          if (P.in_split) umma_ss(d_tm, ahi, smem_desc_sw128(dbase + TILE_BYTES + ks * 2048, HALF_BYTES, 1024), idesc, 1u);
+          if (P.in_split) umma_ss(d_tm, ahi, smem_desc_sw128(dbase + TB + ks * 2048, HALF_BYTES, 1024), idesc, 1u);
         }
         umma_commit(&sh.empty[slot]);
         umma_commit(&sh.acc_full[ab]);
@@ -543,7 +544,7 @@ bool encode_store_map(CUtensorMap* map, const void* base, const FFDims& dm, int 
 cudaError_t launch_pass(ff_plan* p, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& m2,
                         const CUtensorMap& moh, const CUtensorMap& mol, DctTcParams& P, cudaStream_t st) {
   const size_t img = TILE_BYTES;
-  const size_t stage = P.in_split ? 2 * TILE_BYTES : TILE_BYTES;
+  const size_t stage = (size_t)(P.in_split ? 2 : 1) * TILE_ROWS * P.dm.d * 2;
   const size_t fixed = 2 * img + sizeof(DctShared) + 1024;
   int nstage = (int)((232448 - 256 - fixed) / stage);   // 227 KB of shared memory per CTA
   if (nstage > MAX_STAGE) nstage = MAX_STAGE;
