@@ -289,6 +289,7 @@ def run_cuda(args, cfg):
     barrier()
     clocks = sampler.stop()
     ms_step = reduce_max_(ev[0].elapsed_time(ev[-1]) / args.steps)
+    per_step = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps))     # this rank's steps
     launches = plan.last_launches()
     if plan.device_status() != 0:
         raise RuntimeError(B.library().ff_last_error(plan.handle).decode())
@@ -361,6 +362,7 @@ def run_cuda(args, cfg):
             "gpu_launches": launches * args.steps,
             "clocks": clocks,
             "stages_ms": stage_ms,
+            "ms_per_step_median": per_step[len(per_step) // 2], "ms_per_step_best": per_step[0],
             "useful_attention_tflops": work["attn_flops"] / (ms_step * 1e-3) / 1e12,
             "attention_stage_tflops": work["attn_flops"] / (max(stage_ms["attention"], 1e-9) * 1e-3) / 1e12,
             "transform_stage_gbs": work["bytes_transform"] / (max(stage_ms["transform"], 1e-9) * 1e-3) / 1e9,
