@@ -140,6 +140,24 @@ def test_transform_tile_geometries(cfg):
     _run(cfg, alloc=[1, 4, 2], impl=2)       # and the generic transform on the same inputs
 
 
+# Operator-parameter grid of the paper's ablations (compression ratio r, mid degree through block
+# size and stride, window, number of summary tokens) on one 16K-token grid, all through the
+# tensor-core kernels: degenerate windows (R = 0: Y = V~; R >= N_high: dense), a stride of 1 (dense
+# mid band), blocks of 128 and of 16 ranks, no exchange (m = 0), the widest summary set (m = 32).
+ABLATIONS = [
+    dict(r=2, b=32, s=4, R=64, m=4),
+    dict(r=4, b=128, s=2, R=0, m=8),
+    dict(r=8, b=16, s=16, R=100000, m=32),
+    dict(r=1, b=64, s=1, R=300, m=0),
+]
+
+
+@pytest.mark.parametrize("par", ABLATIONS, ids=lambda d: "r{r}_b{b}_s{s}_R{R}_m{m}".format(**d))
+def test_operator_parameter_grid(par):
+    cfg = C.R64K.scaled("ablation", heads=3, seed=31, **par)
+    _run(cfg, alloc=[7, 2, 5])
+
+
 def test_paper_reference_parameterisation_replica():
     """d_k = 64, N_low_bar = N / 32, w = 64, constant-degree mid pattern: the head_dim 64 variants of
     the tensor-core transform and attention kernels, and the generic kernels on the same inputs."""
