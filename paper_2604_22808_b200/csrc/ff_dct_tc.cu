@@ -272,19 +272,21 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
         const int kt = a, ww = w + l;
         const bool hw_low = h < dm.L[1] && ww < dm.L[2], hw_mid = h < dm.M[1] && ww < dm.M[2];
         const int offM = (h < dm.M[1] ? h : dm.M[1]) * dm.M[2] + (h < dm.M[1] ? (ww < dm.M[2] ? ww : dm.M[2]) : 0);
-        const long long cm = kt < dm.M[0] ? (long long)kt * Mhw + offM : (long long)dm.M[0] * Mhw;
+        // (axis lengths are at most 128, so every count fits 32 bits)
+        const int cm = kt < dm.M[0] ? kt * Mhw + offM : dm.M[0] * Mhw;
+        const size_t th_slice = (size_t)tensor * dm.BH + bh;
         if (kt < dm.L[0] && hw_low) {
           band = 0;                                                                  // low band: fp32
           if (LOWACC)
-            row_f32 = P.spec_low + (((size_t)tensor * dm.BH + bh) * dm.Nlow + ((long long)kt * dm.L[1] + h) * dm.L[2] + ww) * CH;
+            row_f32 = P.spec_low + (th_slice * dm.Nlow + (unsigned)((kt * dm.L[1] + h) * dm.L[2] + ww)) * CH;
         } else if (kt < dm.M[0] && hw_mid) {
           const int offL = (h < dm.L[1] ? h : dm.L[1]) * dm.L[2] + (h < dm.L[1] ? (ww < dm.L[2] ? ww : dm.L[2]) : 0);
-          const long long cl = kt < dm.L[0] ? (long long)kt * Lhw + offL : dm.Nlow;
+          const int cl = kt < dm.L[0] ? kt * Lhw + offL : (int)dm.Nlow;
           band = 1;
-          row_hi = P.spec_mid + (((size_t)tensor * dm.BH + bh) * dm.Nmid + (cm - cl)) * CH;
+          row_hi = P.spec_mid + (th_slice * dm.Nmid + (unsigned)(cm - cl)) * CH;
         } else {
           band = 2;
-          row_hi = P.spec_high + (((size_t)tensor * dm.BH + bh) * dm.Nhigh + ((((long long)kt * dm.H + h) * dm.W + ww) - cm)) * CH;
+          row_hi = P.spec_high + (th_slice * dm.Nhigh + (unsigned)(((kt * dm.H + h) * dm.W + ww) - cm)) * CH;
         }
       } else if (P.mode == MODE_FIRST && a < dm.L[2] && !LOWACC) {
         row_f32 = P.side + ((((size_t)gi * dm.T + t) * dm.H + h + l) * dm.L[2] + a) * CH;
