@@ -54,6 +54,7 @@ struct XShared {
   int abort_flag;
   // per softmax warp: 32 rows x 64 bytes of hi and of lo (16-byte chunks XOR-swizzled with row / 2)
   alignas(16) uint8_t stage[4][2][32 * X_STG_PITCH];
+  float inv[2][XT];          // (three-chunk variant) 1 / row sum of the tile, by tile parity
 };
 
 struct XItem { int bh, band, tile; };
@@ -75,10 +76,12 @@ __device__ __forceinline__ XItem x_decode(const FFDims& dm, int h0, int it, int 
 }
 
 // NK32 = 32-key chunks of the score row that are in use (3m <= 32 NK32).
-// (With three chunks the score row does not fit the registers two resident CTAs leave a thread, so
-// that variant runs one CTA per SM.)
+// With three chunks the score row does not fit the registers two resident CTAs leave a thread: that
+// variant sweeps the scores twice (maximum, then exponentials chunk by chunk), writes P unnormalised
+// and lets the store warps scale the update by 1 / row sum.  Its P_lo chunks sit in columns 96, 112
+// and 80, where no unread score can be overwritten.
 template <int NK32, int XD>
-__global__ void __launch_bounds__(X_THREADS, NK32 == 3 ? 1 : 2)
+__global__ void __launch_bounds__(X_THREADS, 2)
 exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_constant__ CUtensorMap map_v_mid,
                    const __grid_constant__ CUtensorMap map_y_high, const __grid_constant__ CUtensorMap map_v_high,
                    const XParams P) {
@@ -165,7 +168,8 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
           const uint64_t bh_ = smem_desc_sw128(zhi + k * 2048, zhalf, 1024);
           umma_ts(tmem + 128, tmem + k * 8, bh_, idesc2, k > 0 ? 1u : 0u);
           umma_ts(tmem + 128, tmem + k * 8, smem_desc_sw128(zlo + k * 2048, zhalf, 1024), idesc2, 1u);
-          umma_ts(tmem + 128, tmem + 48 + k * 8, bh_, idesc2, 1u);
+          const uint32_t plo = NK32 == 3 ? (k < 2 ? 96u : (k < 4 ? 112u : 80u)) + (k & 1) * 8 : 48u + k * 8;
+          umma_ts(tmem + 128, tmem + plo, bh_, idesc2, 1u);
         }
         umma_commit(&sh.d_full);
       }
@@ -209,44 +213,85 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       if (!ok) break;
       tc_fence_after();
       const int own0 = x.band * m, own1 = own0 + m;       // this band's own summaries are not attended
-      // all scores of the row into registers (they are overwritten by P below)
-      uint32_t sc[NK32 * 32];
+      if (NK32 == 3) {
+        // first sweep: the row maximum
+        float mx = -INFINITY;
 #pragma unroll
-      for (int c3 = 0; c3 < NK32; ++c3) {
-        uint32_t r[32];
-        tmem_ld32(tmem + lane_addr + c3 * 32, r);
+        for (int c3 = 0; c3 < NK32; ++c3) {
+          uint32_t r[32];
+          tmem_ld32(tmem + lane_addr + c3 * 32, r);
+          tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) sc[c3 * 32 + i] = r[i];
-      }
-      tmem_wait_ld();
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          for (int i = 0; i < 32; ++i) {
+            const int j = c3 * 32 + i;
+            if (j < 3 * m && (j < own0 || j >= own1)) mx = fmaxf(mx, __uint_as_float(r[i]));
+          }
+        }
+        const float mb = mx * sl2;
+        // second sweep: exponentials and their sum, P (unnormalised, bf16 hi + lo) chunk by chunk
+        float den0 = 0.f, den1 = 0.f;
 #pragma unroll
-      for (int j = 0; j < NK32 * 32; ++j)
-        if (j < 3 * m && (j < own0 || j >= own1)) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(sc[j]));
-      const float mb = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
-      float den4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int j = 0; j < NK32 * 32; ++j) {
-        float pv = 0.f;
-        if (j < 3 * m && (j < own0 || j >= own1)) pv = ex2f_approx(fmaf(__uint_as_float(sc[j]), sl2, -mb));
-        den4[j & 3] += pv;
-        sc[j] = __float_as_uint(pv);
-      }
-      const float inv = 1.f / ((den4[0] + den4[1]) + (den4[2] + den4[3]));
-#pragma unroll
-      for (int c3 = 0; c3 < NK32; ++c3) {
-        if (c3 * 32 < nk) {
+        for (int c3 = 0; c3 < NK32; ++c3) {
+          uint32_t r[32];
+          tmem_ld32(tmem + lane_addr + c3 * 32, r);
+          tmem_wait_ld();
           uint32_t ph[16], pl[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float p0 = __uint_as_float(sc[c3 * 32 + 2 * i]) * inv, p1 = __uint_as_float(sc[c3 * 32 + 2 * i + 1]) * inv;
+            const int j = c3 * 32 + 2 * i;
+            float p0 = 0.f, p1 = 0.f;
+            if (j < 3 * m && (j < own0 || j >= own1)) p0 = ex2f_approx(fmaf(__uint_as_float(r[2 * i]), sl2, -mb));
+            if (j + 1 < 3 * m && (j + 1 < own0 || j + 1 >= own1)) p1 = ex2f_approx(fmaf(__uint_as_float(r[2 * i + 1]), sl2, -mb));
+            den0 += p0; den1 += p1;
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
             ph[i] = *(const uint32_t*)&h2;
             const __nv_bfloat162 l2 = __floats2bfloat162_rn(p0 - __uint_as_float(ph[i] << 16), p1 - __uint_as_float(ph[i] & 0xffff0000u));
             pl[i] = *(const uint32_t*)&l2;
           }
-          tmem_st16(tmem + lane_addr + c3 * 16, ph);
-          tmem_st16(tmem + lane_addr + 48 + c3 * 16, pl);
+          tmem_st16(tmem + lane_addr + c3 * 16, ph);                              // over scores already read
+          tmem_st16(tmem + lane_addr + (c3 == 0 ? 96 : (c3 == 1 ? 112 : 80)), pl);
+        }
+        sh.inv[n & 1][row] = 1.f / (den0 + den1);
+      } else {
+      // all scores of the row into registers (they are overwritten by P below)
+        uint32_t sc[NK32 * 32];
+#pragma unroll
+        for (int c3 = 0; c3 < NK32; ++c3) {
+          uint32_t r[32];
+          tmem_ld32(tmem + lane_addr + c3 * 32, r);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) sc[c3 * 32 + i] = r[i];
+        }
+        tmem_wait_ld();
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int j = 0; j < NK32 * 32; ++j)
+          if (j < 3 * m && (j < own0 || j >= own1)) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(sc[j]));
+        const float mb = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
+        float den4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int j = 0; j < NK32 * 32; ++j) {
+          float pv = 0.f;
+          if (j < 3 * m && (j < own0 || j >= own1)) pv = ex2f_approx(fmaf(__uint_as_float(sc[j]), sl2, -mb));
+          den4[j & 3] += pv;
+          sc[j] = __float_as_uint(pv);
+        }
+        const float inv = 1.f / ((den4[0] + den4[1]) + (den4[2] + den4[3]));
+#pragma unroll
+        for (int c3 = 0; c3 < NK32; ++c3) {
+          if (c3 * 32 < nk) {
+            uint32_t ph[16], pl[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float p0 = __uint_as_float(sc[c3 * 32 + 2 * i]) * inv, p1 = __uint_as_float(sc[c3 * 32 + 2 * i + 1]) * inv;
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+              ph[i] = *(const uint32_t*)&h2;
+              const __nv_bfloat162 l2 = __floats2bfloat162_rn(p0 - __uint_as_float(ph[i] << 16), p1 - __uint_as_float(ph[i] & 0xffff0000u));
+              pl[i] = *(const uint32_t*)&l2;
+            }
+            tmem_st16(tmem + lane_addr + c3 * 16, ph);
+            tmem_st16(tmem + lane_addr + 48 + c3 * 16, pl);
+          }
         }
       }
       tmem_wait_st();
@@ -277,6 +322,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       for (int i = 0; i < 4; ++i) fpos[i] = __shfl_sync(0xffffffffu, f, 8 * i + (lane >> 2));
       const size_t obase = (size_t)(x.bh - P.h0) * dm.N * XD;
       const uint8_t* yrow = sY + slot * X_TILE_BYTES + row * 128;
+      const float dscale = NK32 == 3 ? sh.inv[n & 1][row] : 1.f;    // (three-chunk variant: P was left unnormalised)
       uint8_t* st_hi = sh.stage[quarter][0];
       uint8_t* st_lo = sh.stage[quarter][1];
 #pragma unroll
@@ -293,8 +339,8 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
           uint32_t hi[4], lo[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const float v0 = __uint_as_float(yw[i] << 16) + __uint_as_float(r[v4 * 8 + 2 * i]);
-            const float v1 = __uint_as_float(yw[i] & 0xffff0000u) + __uint_as_float(r[v4 * 8 + 2 * i + 1]);
+            const float v0 = fmaf(__uint_as_float(r[v4 * 8 + 2 * i]), dscale, __uint_as_float(yw[i] << 16));
+            const float v1 = fmaf(__uint_as_float(r[v4 * 8 + 2 * i + 1]), dscale, __uint_as_float(yw[i] & 0xffff0000u));
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
             hi[i] = *(const uint32_t*)&h2;
             const __nv_bfloat162 l2 = __floats2bfloat162_rn(v0 - __uint_as_float(hi[i] << 16), v1 - __uint_as_float(hi[i] & 0xffff0000u));
@@ -398,9 +444,8 @@ cudaError_t ffk_exchange_tc(ff_plan* p, int h0, int g, void* grid_hi, void* grid
   P.pos_mid = p->pos_table; P.pos_high = p->pos_table + dm.Nmid;
   P.grid_hi = (__nv_bfloat16*)grid_hi; P.grid_lo = (__nv_bfloat16*)grid_lo;
   P.h0 = h0; P.g = g; P.nkeys = (3 * dm.m + 15) / 16 * 16; P.status = p->buf.status;
-  // CTAs per SM: two, or one for the widest score rows; the token tile is double-buffered if the
-  // resident CTAs still fit in shared memory
-  const int per_sm = P.nkeys > 64 ? 1 : 2;
+  // Two CTAs per SM; the token tile is double-buffered if both still fit in shared memory
+  const int per_sm = 2;
   P.ybufs = (2 * X_TILE_BYTES + 4 * P.nkeys * 128 + sizeof(XShared) + 2048) * per_sm <= 227 * 1024 ? 2 : 1;
   const size_t smem = P.ybufs * X_TILE_BYTES + 4 * P.nkeys * 128 + sizeof(XShared) + 1024;
   const long long tiles = (long long)g * ((dm.Nmid + XT - 1) / XT + (dm.Nhigh + XT - 1) / XT);
