@@ -54,7 +54,7 @@ struct XShared {
   int abort_flag;
   // per softmax warp: 32 rows x 64 bytes of hi and of lo (16-byte chunks XOR-swizzled with row / 2)
   alignas(16) uint8_t stage[4][2][32 * X_STG_PITCH];
-  float inv[2][XT];          // (three-chunk variant) 1 / row sum of the tile, by tile parity
+  float inv[2][XT];          // (two-sweep variants) 1 / row sum of the tile, by tile parity
 };
 
 struct XItem { int bh, band, tile; };
@@ -76,10 +76,10 @@ __device__ __forceinline__ XItem x_decode(const FFDims& dm, int h0, int it, int 
 }
 
 // NK32 = 32-key chunks of the score row that are in use (3m <= 32 NK32).
-// With three chunks the score row does not fit the registers two resident CTAs leave a thread: that
-// variant sweeps the scores twice (maximum, then exponentials chunk by chunk), writes P unnormalised
-// and lets the store warps scale the update by 1 / row sum.  Its P_lo chunks sit in columns 96, 112
-// and 80, where no unread score can be overwritten.
+// With two or three chunks the score row does not fit the registers two resident CTAs leave a
+// thread: those variants sweep the scores twice (maximum, then exponentials chunk by chunk), write
+// P unnormalised and let the store warps scale the update by 1 / row sum.  Their P_lo chunks sit in
+// columns 96, 112 and 80, where no unread score can be overwritten.
 template <int NK32, int XD>
 __global__ void __launch_bounds__(X_THREADS, 2)
 exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_constant__ CUtensorMap map_v_mid,
@@ -168,7 +168,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
           const uint64_t bh_ = smem_desc_sw128(zhi + k * 2048, zhalf, 1024);
           umma_ts(tmem + 128, tmem + k * 8, bh_, idesc2, k > 0 ? 1u : 0u);
           umma_ts(tmem + 128, tmem + k * 8, smem_desc_sw128(zlo + k * 2048, zhalf, 1024), idesc2, 1u);
-          const uint32_t plo = NK32 == 3 ? (k < 2 ? 96u : (k < 4 ? 112u : 80u)) + (k & 1) * 8 : 48u + k * 8;
+          const uint32_t plo = NK32 >= 2 ? (k < 2 ? 96u : (k < 4 ? 112u : 80u)) + (k & 1) * 8 : 48u + k * 8;
           umma_ts(tmem + 128, tmem + plo, bh_, idesc2, 1u);
         }
         umma_commit(&sh.d_full);
@@ -213,7 +213,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       if (!ok) break;
       tc_fence_after();
       const int own0 = x.band * m, own1 = own0 + m;       // this band's own summaries are not attended
-      if (NK32 == 3) {
+      if (NK32 >= 2) {
         // first sweep: the row maximum
         float mx = -INFINITY;
 #pragma unroll
@@ -322,7 +322,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       for (int i = 0; i < 4; ++i) fpos[i] = __shfl_sync(0xffffffffu, f, 8 * i + (lane >> 2));
       const size_t obase = (size_t)(x.bh - P.h0) * dm.N * XD;
       const uint8_t* yrow = sY + slot * X_TILE_BYTES + row * 128;
-      const float dscale = NK32 == 3 ? sh.inv[n & 1][row] : 1.f;    // (three-chunk variant: P was left unnormalised)
+      const float dscale = NK32 >= 2 ? sh.inv[n & 1][row] : 1.f;    // (two-sweep variants: P was left unnormalised)
       uint8_t* st_hi = sh.stage[quarter][0];
       uint8_t* st_lo = sh.stage[quarter][1];
 #pragma unroll
