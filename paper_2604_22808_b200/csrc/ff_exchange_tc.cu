@@ -10,7 +10,8 @@
 // tile n + 1 while the store warps finish tile n.  Per tile:
 //   TMA     the 128 band tokens (operator output where the head's mask has the band, V~ otherwise)
 //   MMA 1   S[128 x 3m] = Y Z^T against all 3m summaries of the head (own band masked in the softmax)
-//   softmax one token per thread (row = TMEM lane); normalised P written back to TMEM as bf16 hi + lo
+//   softmax one token per thread (row = TMEM lane); P written back to TMEM as bf16 hi + lo (normalised
+//           for up to 32 keys, otherwise unnormalised with the row sum handed to the store warps)
 //   MMA 2   D[128 x 128] = P Z  (A = P from tensor memory, B = the same Z image read MN-major)
 //   store   Y + D as a bf16 hi/lo pair; a thread owns a token, the warp stages 32 channels of its 32
 //           tokens in shared memory and four lanes then write a token's 64 contiguous bytes
