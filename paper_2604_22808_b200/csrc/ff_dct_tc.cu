@@ -420,10 +420,14 @@ constexpr int LOW_TG = 4;
 
 // LOW_CT = k_t chunk: the smallest of 2, 4, 8 that covers L_t keeps the accumulators (and with them
 // the registers per thread) small, so that more CTAs are resident and more loads in flight.
+// With few (k_w, tensor-head) pairs in a launch (large grids, small groups) the t axis is also split
+// over gridDim.z CTAs, which then add their parts into the zeroed output; the energy is summed by
+// low_energy_kernel afterwards.
 template <int LOW_CT, int CH>
 __global__ void __launch_bounds__(CH * LOW_TG) low_band_kernel(const float* side, const float* CT, const float* CHm,
                                                                float* spec_low, double* energy, FFDims dm, int group_start) {
   const int kw = blockIdx.x;
+  const int t_per = dm.T / (int)gridDim.z, t_lo = (int)blockIdx.z * t_per;   // this CTA's t range
   const int gi = blockIdx.y, th = group_start + gi;
   const int c = threadIdx.x % CH, tg = threadIdx.x / CH;     // threads = d x LOW_TG
   __shared__ float ch_rows[LOW_CH][128];          // C_H rows of the current k_h chunk
@@ -443,7 +447,7 @@ __global__ void __launch_bounds__(CH * LOW_TG) low_band_kernel(const float* side
       for (int i = 0; i < LOW_CT; ++i)
 #pragma unroll
         for (int q = 0; q < LOW_CH; ++q) acc[i][q] = 0.f;
-      for (int t = tg; t < dm.T; t += LOW_TG) {
+      for (int t = t_lo + tg; t < t_lo + t_per; t += LOW_TG) {
         const float* col = side + ((((size_t)gi * dm.T + t) * dm.H) * dm.L[2] + kw) * CH + c;
         float s[LOW_CH];
 #pragma unroll
@@ -477,13 +481,22 @@ __global__ void __launch_bounds__(CH * LOW_TG) low_band_kernel(const float* side
         if (kt0 + i >= dm.L[0] || kh0 + q >= dm.L[1]) continue;
         const long long rank = ((long long)(kt0 + i) * dm.L[1] + kh0 + q) * dm.L[2] + kw;
         const float v = red[o][c];
-        spec_low[((size_t)th * dm.Nlow + rank) * CH + c] = v;
-        e = fmaf(v, v, e);
+        float* dst = spec_low + ((size_t)th * dm.Nlow + rank) * CH + c;
+        if (gridDim.z == 1) { *dst = v; e = fmaf(v, v, e); } else atomicAdd(dst, v);
       }
       __syncthreads();
     }
   }
-  if (energy) atomicAdd(energy + ((size_t)((th % dm.BH) / dm.heads) * 3) * CH + c, (double)e);
+  if (energy && gridDim.z == 1) atomicAdd(energy + ((size_t)((th % dm.BH) / dm.heads) * 3) * CH + c, (double)e);
+}
+
+// Low-band energy of tensor-heads [group_start, group_start + gridDim.x): thread = channel.
+__global__ void low_energy_kernel(const float* spec_low, double* energy, FFDims dm, int group_start) {
+  const int th = group_start + blockIdx.x, c = threadIdx.x;
+  const float* v = spec_low + (size_t)th * dm.Nlow * dm.d + c;
+  float e = 0.f;
+  for (long long r = 0; r < dm.Nlow; ++r) { const float x = v[(size_t)r * dm.d]; e = fmaf(x, x, e); }
+  atomicAdd(energy + ((size_t)((th % dm.BH) / dm.heads) * 3) * dm.d + c, (double)e);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -677,12 +690,19 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
     P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 0 + 0) * TILE_BYTES;
     e = launch_pass(p, m2h, m2l, m2l, m2h, m2l, P, st);    // (no tensor stores in this mode)
     if (e != cudaSuccess) return e;
-    dim3 lgrid((unsigned)dm.L[2], (unsigned)g);
     if (P.low_from_acc) continue;                  // the band-split pass has written the low band already
+    int tz = 1;                                    // split t when the launch would not fill the GPU
+    while (dm.L[2] * g * tz < p->sm_count && tz * 2 * LOW_TG <= dm.T) tz *= 2;
+    dim3 lgrid((unsigned)dm.L[2], (unsigned)g, (unsigned)tz);
+    if (tz > 1) {
+      e = cudaMemsetAsync(p->buf.spec_low + (size_t)g0 * dm.Nlow * dm.d, 0, (size_t)g * dm.Nlow * dm.d * sizeof(float), st);
+      if (e != cudaSuccess) return e;
+    }
 #define FF_LOW(CT, D) low_band_kernel<CT, D><<<lgrid, D * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0)
     if (dm.d == 128) { if (dm.L[0] <= 2) FF_LOW(2, 128); else if (dm.L[0] <= 4) FF_LOW(4, 128); else FF_LOW(8, 128); }
     else { if (dm.L[0] <= 2) FF_LOW(2, 64); else if (dm.L[0] <= 4) FF_LOW(4, 64); else FF_LOW(8, 64); }
 #undef FF_LOW
+    if (tz > 1 && P.energy) { low_energy_kernel<<<g, dm.d, 0, st>>>(p->buf.spec_low, P.energy, dm, g0); p->launches += 1; }
     p->launches += 1;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
