@@ -129,8 +129,24 @@ __device__ __forceinline__ bool wait_counter(const int* cnt, int target, volatil
     if (*abort_flag) return false;
     if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return false; }
   }
-  asm volatile("fence.proxy.async;" ::: "memory");
+  asm volatile("fence.proxy.async.global;" ::: "memory");
   return true;
+}
+
+// The same with the counter already sampled (a relaxed load issued one tile earlier, so that its
+// latency overlaps the previous tile's copies): if the sample suffices, an acquire fence orders the
+// reads that follow; otherwise poll.
+__device__ __forceinline__ bool wait_counter_sampled(const int* cnt, int sample, int target, volatile int* abort_flag) {
+  if (sample < target) return wait_counter(cnt, target, abort_flag);
+  asm volatile("fence.acquire.gpu;" ::: "memory");
+  asm volatile("fence.proxy.async.global;" ::: "memory");
+  return true;
+}
+
+__device__ __forceinline__ int load_relaxed(const int* p) {
+  int v;
+  asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
 }
 
 // m0..m2: first-pass input (forward: Q, K, V; inverse: hi grid, lo grid, unused).
@@ -178,15 +194,24 @@ dct_wh_kernel(const __grid_constant__ CUtensorMap m0, const __grid_constant__ CU
       const uint64_t pol_ring = policy_evict_last(), pol_stream = policy_evict_first();
       unsigned it = 0;
       bool ok = true;
+      // the counter a tile depends on: the slab's first pass is stored / the ring slot has been consumed
+      auto counter_of = [&](const WhTile& y) -> const int* {
+        return y.second ? P.cnt_a + y.slab : (y.slab >= P.ring ? P.cnt_b + y.slab - P.ring : nullptr);
+      };
+      const int* cnt_next = blockIdx.x < total ? counter_of(wh_decode(blockIdx.x, tps, S, D)) : nullptr;
+      int sample_next = cnt_next ? load_relaxed(cnt_next) : 0;
       for (int idx = blockIdx.x; idx < total && ok; idx += gridDim.x, ++it) {
         const WhTile x = wh_decode(idx, tps, S, D);
         const int gi = x.slab / dm.T, t = x.slab % dm.T, slot = x.slab % P.ring;
         const bool along_w = (x.second == 0) == (P.forward != 0);
         const bool split = x.second || !P.forward;
         const uint64_t pol = x.second ? pol_ring : pol_stream;
-        // dependencies: the slab's first pass is stored / the ring slot has been consumed
-        if (x.second) ok = wait_counter(P.cnt_a + x.slab, 8 * tps, abort_flag);
-        else if (x.slab >= P.ring) ok = wait_counter(P.cnt_b + x.slab - P.ring, 8 * tps, abort_flag);
+        const int* cnt = cnt_next;
+        const int sample = sample_next;
+        // sample the next tile's counter now; it is looked at one iteration later
+        cnt_next = idx + (int)gridDim.x < total ? counter_of(wh_decode(idx + gridDim.x, tps, S, D)) : nullptr;
+        sample_next = cnt_next ? load_relaxed(cnt_next) : 0;
+        if (cnt) ok = wait_counter_sampled(cnt, sample, 8 * tps, abort_flag);
         if (!ok) break;
         const int st = it % NSTAGE;
         if (it >= NSTAGE) ok = mbar_wait(&sh.empty[st], ((it / NSTAGE) - 1) & 1, abort_flag);
@@ -335,9 +360,8 @@ dct_wh_kernel(const __grid_constant__ CUtensorMap m0, const __grid_constant__ CU
       if (lane == 0) {
         if (pending) {
           bulk_wait2();
-          asm volatile("fence.proxy.async;" ::: "memory");
-          __threadfence();
-          atomicAdd(pending, 1);
+          asm volatile("fence.proxy.async.global;" ::: "memory");
+          asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(pending) : "memory");
         }
         pending = (x.second ? P.cnt_b : P.cnt_a) + x.slab;
       }
@@ -345,9 +369,8 @@ dct_wh_kernel(const __grid_constant__ CUtensorMap m0, const __grid_constant__ CU
     if (lane == 0) {
       bulk_wait0();
       if (pending) {
-        asm volatile("fence.proxy.async;" ::: "memory");
-        __threadfence();
-        atomicAdd(pending, 1);
+        asm volatile("fence.proxy.async.global;" ::: "memory");
+        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(pending) : "memory");
       }
     }
   }
