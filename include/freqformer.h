@@ -200,8 +200,11 @@ ff_status_t ff_get_tap(const ff_plan_t *plan, int32_t which, const void **dev_pt
 
 /* Kernel selection, a bit mask (0 = the defaults): 1 = generic SIMT attention instead of the
  * tensor-core kernel, 2 = generic SIMT transform instead of the tensor-core passes, 4 = w and h
- * passes fused in one launch with the intermediate kept in L2 (measured slower than separate passes
- * on B200; kept for experiments).  For tests and benchmarks. */
+ * passes fused in one launch with the intermediate kept in L2 (measured level with the separate
+ * passes on B200; kept for experiments).  For tests and benchmarks.
+ * The tensor-core kernels cover bf16 storage with head_dim 128 or 64, axis lengths 16, 32, 64 or 128
+ * and mid block sizes that tile 128 ranks; the pooled low band joins the tensor-core attention launch
+ * from 128 pooled tokens on.  Every other configuration runs on the generic fp32 kernels. */
 ff_status_t ff_plan_set_attention_impl(ff_plan_t *plan, int32_t impl);
 
 /* ---- for callers that cannot allocate device memory ---------------------------------------------
