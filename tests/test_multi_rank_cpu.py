@@ -58,3 +58,32 @@ def test_reference_arm_runs_on_rank_zero_only():
     import json
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
+
+
+def test_forced_allocation_option():
+    """`--alloc L,M,H`: heads [0,L) low, the next M mid, the rest high, repeated per sample."""
+    cfg = C.G128K                                   # batch 2, 24 heads
+    masks = bench.forced_allocation(cfg, "12,8,4")
+    assert len(masks) == cfg.batch * cfg.heads
+    assert masks[:24] == [1] * 12 + [2] * 8 + [4] * 4 and masks[24:] == masks[:24]
+    assert bench.forced_allocation(cfg, "") is None
+    for bad in ("12,8", "12,8,5", "-1,13,12"):
+        try:
+            bench.forced_allocation(cfg, bad)
+        except SystemExit:
+            continue
+        raise AssertionError(f"--alloc {bad} was accepted")
+
+
+def test_layer_work_counts_follow_the_cost_formulas():
+    """bench.py's interaction counts (its useful-FLOP figure) equal the oracle's counters."""
+    from oracle import freqformer_oracle as O
+    for cfg in (C.TINY, C.G64K, C.R1M, C.PAPER_REF_64K):
+        sizes = [len(x) for x in O.band_members(cfg.grid, cfg.low_cut, cfg.mid_cut)]
+        n_bar = -(-sizes[0] // cfg.r)
+        expect = (n_bar * n_bar, O.mid_interactions(sizes[1], cfg.b, cfg.s), O.high_interactions(sizes[2], cfg.R))
+        assert bench.interactions(cfg) == expect, (cfg.name, bench.interactions(cfg), expect)
+        alloc = [1, 2, 4, 7][: cfg.heads] * cfg.batch
+        work = bench.layer_work(cfg, alloc)
+        per_mask = {1: expect[0], 2: expect[1], 4: expect[2], 7: sum(expect)}
+        assert work["attn_flops"] == 4 * cfg.head_dim * sum(per_mask[m] for m in alloc)
