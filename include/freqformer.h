@@ -162,6 +162,17 @@ ff_status_t ff_workspace_bytes_host(const ff_config_t *cfg, size_t *bytes);
  * clears it. */
 ff_status_t ff_plan_device_status(ff_plan_t *plan, void *cuda_stream);
 
+/* Self-test of the failure path (no counterpart in the paper): launches one small CTA in which two
+ * warps wait on a barrier nobody arrives at, with a limit of `limit_cycles` SM clock cycles (1 ..
+ * 2e9, i.e. at most about a second).  The first waiter's limit runs out, it raises the CTA's abort
+ * flag, the second waiter leaves on the flag, and the CTA records FF_ERR_TIMEOUT in the plan's
+ * device status word exactly as the tensor-core kernels do.  Synchronises the stream.
+ *   waiters_released  host, out: how many of the two waits returned "abandoned" (2 when all is well)
+ * Afterwards ff_plan_device_status returns FF_ERR_TIMEOUT once (and clears the word); the plan and
+ * the CUDA context stay usable. */
+ff_status_t ff_plan_selftest_bounded_wait(ff_plan_t *plan, int64_t limit_cycles,
+                                          int32_t *waiters_released, void *cuda_stream);
+
 /* Number of kernel launches the last ff_forward / ff_route on this plan issued. */
 ff_status_t ff_plan_last_launches(const ff_plan_t *plan, int64_t *launches);
 

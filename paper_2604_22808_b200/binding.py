@@ -28,7 +28,8 @@ FF_BAND_LOW, FF_BAND_MID, FF_BAND_HIGH = 1, 2, 4
 EXPORTS = ("ff_config_validate", "ff_band_sizes", "ff_band_rank", "ff_workspace_bytes", "ff_workspace_bytes_host",
            "ff_plan_create", "ff_plan_workspace_bytes", "ff_plan_set_workspace", "ff_destroy", "ff_last_error",
            "ff_route", "ff_forward", "ff_forward_host", "ff_plan_device_status", "ff_plan_last_launches",
-           "ff_get_tap", "ff_plan_set_attention_impl", "ff_plan_set_profiling", "ff_plan_stage_times", "ff_high_attention_noalloc")
+           "ff_get_tap", "ff_plan_set_attention_impl", "ff_plan_set_profiling", "ff_plan_stage_times", "ff_high_attention_noalloc",
+           "ff_plan_selftest_bounded_wait")
 STAGES = ("transform", "router", "attention", "summary", "inverse")
 
 
@@ -77,6 +78,7 @@ def library() -> C.CDLL:
         lib.ff_plan_set_profiling.argtypes = [C.c_void_p, C.c_int32]
         lib.ff_plan_stage_times.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
         lib.ff_high_attention_noalloc.argtypes = [C.c_void_p] * 4 + [C.c_int32, C.c_int64, C.c_int32, C.c_int32, C.c_void_p]
+        lib.ff_plan_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int32), C.c_void_p]
         lib.ff_config_validate.argtypes = [C.POINTER(ff_config_t)]
         lib.ff_band_sizes.argtypes = [C.POINTER(ff_config_t), C.POINTER(C.c_int64)]
         lib.ff_band_rank.argtypes = [C.POINTER(ff_config_t), C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_int32),
@@ -221,6 +223,12 @@ class Plan:
 
     def device_status(self) -> int:
         return library().ff_plan_device_status(self.handle, self._stream())
+
+    def selftest_bounded_wait(self, limit_cycles: int) -> int:
+        """Runs the bounded-wait self-test; returns how many of its two waits were abandoned."""
+        n = C.c_int32(-1)
+        _check(library().ff_plan_selftest_bounded_wait(self.handle, int(limit_cycles), C.byref(n), self._stream()), self.handle)
+        return n.value
 
     def last_launches(self) -> int:
         n = C.c_int64()

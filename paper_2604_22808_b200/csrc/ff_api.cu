@@ -449,3 +449,42 @@ extern "C" ff_status_t ff_get_tap(const ff_plan_t* p, int32_t which, const void*
   }
   return FF_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// Self-test of the bounded device-side wait every tensor-core kernel is built on: one CTA waits,
+// with a limit of `limit_cycles`, on a barrier nobody ever arrives at; when the limit runs out the
+// first waiter raises the CTA's abort flag, the second waiter (another warp) sees the flag and
+// leaves too, and the CTA records FF_ERR_TIMEOUT in the plan's status word and returns.  Nothing
+// hangs: the longest possible wait is the limit (at most 2e9 cycles, about a second).
+// ------------------------------------------------------------------------------------------------
+#include "ff_sm100.cuh"
+
+namespace {
+__global__ void bounded_wait_selftest_kernel(int* status, long long limit_cycles, int* observed) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) { sm100::mbar_init(&bar, 1); abort_flag = 0; sm100::fence_mbar_init(); }
+  __syncthreads();
+  bool ok = true;
+  if (threadIdx.x == 0) ok = sm100::mbar_wait(&bar, 0, &abort_flag, limit_cycles);         // runs out
+  if (threadIdx.x == 32) ok = sm100::mbar_wait(&bar, 0, &abort_flag, 4 * limit_cycles);    // leaves on the flag
+  if (threadIdx.x == 0 || threadIdx.x == 32) atomicAdd(observed, ok ? 0 : 1);
+  __syncthreads();
+  if (threadIdx.x == 0 && abort_flag) atomicExch(status, FF_ERR_TIMEOUT | 0x500);
+}
+}  // namespace
+
+extern "C" ff_status_t ff_plan_selftest_bounded_wait(ff_plan_t* p, int64_t limit_cycles, int32_t* waiters_released,
+                                                     void* stream) {
+  if (!p || !waiters_released) return fail(p, FF_ERR_INVALID_ARG, "plan or waiters_released is NULL%s");
+  if (!p->ws) return fail(p, FF_ERR_WORKSPACE, "ff_plan_set_workspace has not been called%s");
+  if (limit_cycles < 1 || limit_cycles > 2000000000LL) return fail(p, FF_ERR_INVALID_ARG, "limit_cycles must be in [1, 2e9]%s");
+  cudaStream_t st = (cudaStream_t)stream;
+  int* observed = p->buf.status + 1;               // the status region is 256 bytes; word 0 is the status
+  FF_CUDA(p, cudaMemsetAsync(observed, 0, sizeof(int), st));
+  bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(p->buf.status, limit_cycles, observed);
+  FF_CUDA(p, cudaGetLastError());
+  FF_CUDA(p, cudaMemcpyAsync(waiters_released, observed, sizeof(int), cudaMemcpyDeviceToHost, st));
+  FF_CUDA(p, cudaStreamSynchronize(st));
+  return FF_OK;
+}

@@ -227,6 +227,34 @@ def test_error_paths_on_device():
     plan.destroy()
 
 
+def test_bounded_wait_expires_cleanly():
+    """A device-side wait that nothing satisfies runs out after its (short) limit, the CTA reports
+    FF_ERR_TIMEOUT through the status word, and the plan and the context stay usable."""
+    import torch
+    from paper_2604_22808_b200 import binding as B
+    cfg = C.TINY
+    Q, K, V = Hn.host_inputs(cfg)
+    weights = I.router_weights(cfg)
+    out0, plan = Hn.gpu_forward(cfg, Q, K, V, weights, None, timesteps=[cfg.timesteps[0]])
+    assert plan.device_status() == 0
+    assert plan.selftest_bounded_wait(2_000_000) == 2          # about a millisecond
+    assert plan.device_status() == 5                            # FF_ERR_TIMEOUT, reported once ...
+    assert "kernel 5" in B.library().ff_last_error(plan.handle).decode()
+    assert plan.device_status() == 0                            # ... and cleared
+    lib = B.library()
+    n = B.C.c_int32(0)
+    assert lib.ff_plan_selftest_bounded_wait(plan.handle, 0, B.C.byref(n), None) == 1        # limit out of range
+    assert lib.ff_plan_selftest_bounded_wait(plan.handle, 3_000_000_000, B.C.byref(n), None) == 1
+    # the same plan still computes the same result
+    dev = [torch.from_numpy(x).cuda() for x in (Q, K, V)]
+    out = torch.empty_like(dev[0])
+    plan.forward(dev[0], dev[1], dev[2], out, timesteps=[cfg.timesteps[0]])
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    assert np.abs(out.cpu().numpy() - out0).max() < 1e-5        # (summary sums are atomic: last bits may move)
+    plan.destroy()
+
+
 def test_host_buffer_entry_point():
     import torch
     from paper_2604_22808_b200 import binding as B
