@@ -68,6 +68,28 @@ def interactions(cfg):
     return n_bar * n_bar, i_mid, i_high
 
 
+def issued_pairs(cfg):
+    """(query, key) pairs the tensor-core attention kernel computes per head and band, whole
+    128 x 128 tiles including their masked parts: mid = every tile pair of a residue class, high =
+    the key tiles that meet a query tile's window, low = every tile pair of the pooled band."""
+    n_low, n_bar, n_mid, n_high = band_sizes(cfg)
+    T = 128
+    nb = -(-n_mid // cfg.b)
+    i_mid = 0
+    for c in range(min(cfg.s, nb)):
+        blocks = len(range(c, nb, cfg.s))
+        nt = -(-blocks * cfg.b // T)
+        i_mid += nt * nt * T * T
+    i_high = 0
+    for qt in range(-(-n_high // T)):
+        q0 = qt * T
+        lo, hi = max(0, q0 - cfg.R), min(n_high, q0 + T + cfg.R)
+        # key tiles start at the pair's first key (multiples of 128 from there); count tiles meeting [lo, hi)
+        i_high += (-(-(hi - lo) // T)) * T * T
+    nt_low = -(-n_bar // T)
+    return nt_low * nt_low * T * T, i_mid, i_high
+
+
 def layer_work(cfg, alloc):
     """Useful attention FLOPs (4 d per pair: QK^T and PV) and algorithmic HBM bytes of one forward."""
     d, e = cfg.head_dim, (4 if cfg.dtype == "fp32" else 2)
@@ -224,6 +246,11 @@ def forced_allocation(cfg, text):
     return ([1] * n[0] + [2] * n[1] + [4] * n[2]) * cfg.batch
 
 
+def tensor_core_path_any(cfg) -> bool:
+    """Does this workload run on the tensor-core kernels (bf16, head_dim 128 or 64)?"""
+    return cfg.dtype == "bf16" and cfg.head_dim in (64, 128)
+
+
 def aggregate_tokens_per_s(cfg, world: int, ms_step_max: float) -> float:
     """Whole-job throughput: the tokens all ranks processed over the slowest rank's step time."""
     return cfg.batch * cfg.N * world / (ms_step_max * 1e-3)
@@ -317,7 +344,7 @@ def run_cuda(args, cfg):
         top = max(stage_ms, key=stage_ms.get)
         n_launch = max(1, stage_launches.get(top) or 1)
         heads_total = cfg.batch * cfg.heads
-        tensor_core_path = cfg.dtype == "bf16" and cfg.head_dim == 128       # otherwise the generic fp32 kernels run
+        tensor_core_path = tensor_core_path_any(cfg)                         # otherwise the generic fp32 kernels run
         if top == "attention" and tensor_core_path:
             achieved = work["attn_flops"] / (stage_ms[top] * 1e-3) / 1e12
             roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
@@ -364,6 +391,10 @@ def run_cuda(args, cfg):
             "stages_ms": stage_ms,
             "ms_per_step_median": per_step[len(per_step) // 2], "ms_per_step_best": per_step[0],
             "useful_attention_tflops": work["attn_flops"] / (ms_step * 1e-3) / 1e12,
+            # whole tiles the tensor-core kernel computes (masked parts included); the pooled low band only from 128 tokens on
+            "attention_stage_issued_tflops": (4 * cfg.head_dim * sum(
+                sum(p for l, p in enumerate(issued_pairs(cfg)) if (mk >> l & 1) and (l > 0 or band_sizes(cfg)[1] >= 128))
+                for mk in alloc) / (max(stage_ms["attention"], 1e-9) * 1e-3) / 1e12) if tensor_core_path_any(cfg) else None,
             "attention_stage_tflops": work["attn_flops"] / (max(stage_ms["attention"], 1e-9) * 1e-3) / 1e12,
             "transform_stage_gbs": work["bytes_transform"] / (max(stage_ms["transform"], 1e-9) * 1e-3) / 1e9,
             "inverse_stage_gbs": work["bytes_inverse"] / (max(stage_ms["inverse"], 1e-9) * 1e-3) / 1e9,
