@@ -195,15 +195,19 @@ __global__ void router_kernel(const double* energy, const float* timestep, const
   const int half = dm.dt / 2;
   const double t = (double)timestep[sample];
   for (int i = threadIdx.x; i < half; i += blockDim.x) {
-    const double om = pow(10000.0, -(double)i / (double)half);
-    x[3 * d + i] = (float)sin(t * om);
-    x[3 * d + half + i] = (float)cos(t * om);
+    const double om = exp2(-(double)i / (double)half * 13.287712379549449);     // 10000^(-i/half); log2(10000)
+    double sn, cs;
+    sincos(t * om, &sn, &cs);
+    x[3 * d + i] = (float)sn;
+    x[3 * d + half + i] = (float)cs;
   }
   __syncthreads();
-  for (int j = threadIdx.x; j < hid; j += blockDim.x) {
-    float acc = b1[j];
-    for (int i = 0; i < nin; ++i) acc = fmaf(W1[(size_t)j * nin + i], x[i], acc);
-    h[j] = fmaxf(acc, 0.f);
+  // hidden layer: one warp per unit, lanes stride over the inputs (coalesced rows of W1)
+  for (int j = threadIdx.x >> 5; j < hid; j += blockDim.x >> 5) {
+    float acc = 0.f;
+    for (int i = threadIdx.x & 31; i < nin; i += 32) acc = fmaf(W1[(size_t)j * nin + i], x[i], acc);
+    acc = warp_sum(acc);
+    if ((threadIdx.x & 31) == 0) h[j] = fmaxf(acc + b1[j], 0.f);
   }
   __syncthreads();
   if (threadIdx.x < 3) {
@@ -586,7 +590,7 @@ cudaError_t ffk_band_energy(ff_plan* p, cudaStream_t st) {
 cudaError_t ffk_router(ff_plan* p, uint8_t* alloc_out, cudaStream_t st) {
   const FFDims& dm = p->dm;
   const size_t smem = (size_t)(3 * dm.d + dm.dt + dm.hid) * sizeof(float);
-  router_kernel<<<dm.B, 128, smem, st>>>(p->buf.energy, p->buf.timestep, p->W1, p->b1, p->W2, p->b2, alloc_out,
+  router_kernel<<<dm.B, 256, smem, st>>>(p->buf.energy, p->buf.timestep, p->W1, p->b1, p->W2, p->b2, alloc_out,
                                          p->buf.pi, dm);
   p->launches += 1;
   return cudaGetLastError();
