@@ -227,6 +227,26 @@ def test_error_paths_on_device():
     plan.destroy()
 
 
+@pytest.mark.parametrize("batch,heads", [(1, 1), (3, 5)])
+def test_head_and_batch_counts(batch, heads):
+    """Head and batch counts that do not divide the kernels' launch groups, routed per sample."""
+    cfg = C.R64K.scaled(f"r64k_b{batch}_h{heads}", batch=batch, heads=heads, seed=41,
+                        timesteps=tuple([800.0, 500.0, 100.0][:batch]))
+    Q, K, V = Hn.host_inputs(cfg)
+    weights = I.router_weights(cfg)
+    U = I.summary_projection(cfg)
+    ts = list(cfg.timesteps)
+    res = Hn.oracle_forward(cfg, Q, K, V, weights, U, ts, alloc=None, want_taps=False)
+    out, plan = Hn.gpu_forward(cfg, Q, K, V, weights, None, timesteps=ts)
+    from paper_2604_22808_b200 import binding as B
+    gpu_alloc = plan.tap(B.TAP_ALLOC).cpu().numpy().reshape(cfg.batch, cfg.heads)
+    for bi in range(cfg.batch):
+        if Hn.allocation_is_stable(res[bi]["pi"], cfg.heads):
+            assert np.array_equal(gpu_alloc[bi], res[bi]["alloc"])
+            Hn.assert_close(out[bi], res[bi]["out"], cfg.dtype, f"out sample {bi}")
+    plan.destroy()
+
+
 def test_run_to_run_determinism():
     """Two forwards of one plan on the same inputs: the mid- and high-band coefficients and operator
     outputs are bit-identical (fixed work assignment, no atomics on those paths); the fp32 low band
