@@ -434,3 +434,26 @@ def test_router_allocation_path_runs_and_is_consistent():
     sizes = np.array(res["sizes"])[:, None]
     tok = sum((x.astype(np.float64) ** 2).sum(axis=(0, 1, 2, 3)) for x in (Q, K, V))
     assert np.allclose((E * sizes * 3 * cfg.heads).sum(0), tok, rtol=1e-10)
+
+
+def test_paper_reference_workloads_match_the_reference_cost():
+    """The paper-reference workloads reproduce the "Reference complexity instantiation": N_low_bar =
+    N / 32 exactly, a mid degree of 256 (a residue class = 8 blocks of 32 ranks) and w = 65 keys; with
+    the integer boxes the band fractions are 0.125 / 0.391 / 0.484, so the exact interaction count
+    lands within a few per cent of 0.0009765625 N^2 + 128 N."""
+    from paper_2604_22808_b200 import configs as C
+    for cfg in (C.PAPER_REF_64K, C.PAPER_REF_1M):
+        sizes = [len(x) for x in O.band_members(cfg.grid, cfg.low_cut, cfg.mid_cut)] if cfg.N <= 70000 else None
+        n_low = cfg.low_cut[0] * cfg.low_cut[1] * cfg.low_cut[2]
+        n_mid = cfg.mid_cut[0] * cfg.mid_cut[1] * cfg.mid_cut[2] - n_low
+        n_high = cfg.N - n_low - n_mid
+        if sizes is not None:
+            assert sizes == [n_low, n_mid, n_high]
+        assert n_low * 8 == cfg.N and -(-n_low // cfg.r) * 32 == cfg.N
+        i_mid = O.mid_interactions(n_mid, cfg.b, cfg.s)
+        assert abs(i_mid / n_mid - 256) < 4                       # average mid degree
+        assert 2 * cfg.R + 1 == 65
+        exact = (cfg.N // 32) ** 2 + i_mid + O.high_interactions(n_high, cfg.R)
+        reference = O.paper_attention_cost_reference(cfg.N, 1.0)  # = 0.0009765625 N^2 + 128 N
+        assert abs(reference - (0.0009765625 * cfg.N ** 2 + 128 * cfg.N)) < 1e-6 * reference
+        assert abs(exact - reference) < 0.05 * reference
