@@ -399,6 +399,9 @@ def run_cuda(args, cfg):
             "transform_stage_gbs": work["bytes_transform"] / (max(stage_ms["transform"], 1e-9) * 1e-3) / 1e9,
             "inverse_stage_gbs": work["bytes_inverse"] / (max(stage_ms["inverse"], 1e-9) * 1e-3) / 1e9,
             "paper_context": "simulated estimates only: 9.3-27.3x attention-FLOP and 8.8-20.9x score-traffic reduction vs dense",
+            # the same ratio for this workload and allocation, from the interaction counts (exchange included)
+            "interaction_reduction_vs_dense": (len(alloc) * cfg.N * cfg.N) / max(1, work["attn_flops"] // (4 * cfg.head_dim)
+                                                                              + len(alloc) * 2 * cfg.m * cfg.N),
         }
         print(json.dumps(line))
     plan.destroy()
