@@ -150,9 +150,12 @@ ff_status_t ff_forward(ff_plan_t *plan, const void *Q, const void *K, const void
                        void *cuda_stream);
 
 /* Same computation with HOST buffers: copies Q, K, V host->device into staging space inside the
- * workspace, runs ff_forward, copies out device->host, all on `cuda_stream`, then synchronises.
+ * workspace, runs ff_forward, copies out device->host, then synchronises.  On the tensor-core path
+ * the copies run on a second stream owned by the plan, ordered after the work already queued on
+ * `cuda_stream`: the forward transform starts on the first group of tensor-heads while the later
+ * ones are still arriving, and finished groups of output heads leave while the rest is computed.
  * The workspace must have been sized with ff_workspace_bytes_host.  alloc_host may be NULL
- * (route internally); pinned host memory makes the copies asynchronous. */
+ * (route internally); pinned host memory makes the copies asynchronous (and the overlap real). */
 ff_status_t ff_forward_host(ff_plan_t *plan, const void *Q_host, const void *K_host,
                             const void *V_host, const uint8_t *alloc_host, const float *timestep,
                             void *out_host, void *cuda_stream);

@@ -163,6 +163,10 @@ extern "C" ff_status_t ff_destroy(ff_plan_t* p) {
   if (!p) return FF_OK;
   for (int a = 0; a < 3; ++a) { cudaFree(p->basis[a]); cudaFree(p->basis_t[a]); }
   if (p->ev[0]) for (int i = 0; i <= FF_STAGE_COUNT; ++i) cudaEventDestroy(p->ev[i]);
+  if (p->copy_stream) {
+    for (int i = 0; i <= 2 * FF_COPY_EVENTS; ++i) cudaEventDestroy(p->ev_copy[i]);
+    cudaStreamDestroy(p->copy_stream);
+  }
   cudaFree(p->dct_images); cudaFree(p->pos_table);
   cudaFree(p->W1); cudaFree(p->b1); cudaFree(p->W2); cudaFree(p->b2); cudaFree(p->U);
   delete p;
@@ -410,19 +414,60 @@ extern "C" ff_status_t ff_forward_host(ff_plan_t* p, const void* Qh, const void*
   if (!p->ws) return fail(p, FF_ERR_WORKSPACE, "ff_plan_set_workspace has not been called%s");
   if (!p->ws_has_staging) return fail(p, FF_ERR_WORKSPACE, "workspace lacks staging space: size it with ff_workspace_bytes_host%s");
   cudaStream_t st = (cudaStream_t)stream;
-  const size_t bytes = (size_t)p->dm.BH * p->dm.N * p->dm.d * (p->dm.fp32 ? 4 : 2);
-  FF_CUDA(p, cudaMemcpyAsync(p->buf.stage_q, Qh, bytes, cudaMemcpyHostToDevice, st));
-  FF_CUDA(p, cudaMemcpyAsync(p->buf.stage_k, Kh, bytes, cudaMemcpyHostToDevice, st));
-  FF_CUDA(p, cudaMemcpyAsync(p->buf.stage_v, Vh, bytes, cudaMemcpyHostToDevice, st));
+  const FFDims& dm = p->dm;
+  const size_t head_bytes = (size_t)dm.N * dm.d * (dm.fp32 ? 4 : 2);
+  const size_t bytes = (size_t)dm.BH * head_bytes;
+  // On the tensor-core path the copies are pipelined with the transforms: the forward transform works
+  // through Q, K, V in groups of tensor-heads and waits only for its own group's copy; the inverse
+  // hands every finished group of heads to the copy stream.
+  const int G = p->dct_group;
+  const int total = 3 * dm.BH;
+  const bool piped = p->dct_tc_ok && !(p->attn_impl & 2) && G > 0 && (total + G - 1) / G <= FF_COPY_EVENTS &&
+                     (dm.BH + G - 1) / G <= FF_COPY_EVENTS;
+  if (piped && !p->copy_stream) {
+    FF_CUDA(p, cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking));
+    for (int i = 0; i <= 2 * FF_COPY_EVENTS; ++i) FF_CUDA(p, cudaEventCreateWithFlags(&p->ev_copy[i], cudaEventDisableTiming));
+  }
   // The caller's masks travel through the tail of the (not yet used) output staging area.
   uint8_t* alloc_dev = nullptr;
   if (alloc_host) {
     alloc_dev = (uint8_t*)p->buf.stage_out;
-    FF_CUDA(p, cudaMemcpyAsync(alloc_dev, alloc_host, p->dm.BH, cudaMemcpyHostToDevice, st));
+    FF_CUDA(p, cudaMemcpyAsync(alloc_dev, alloc_host, dm.BH, cudaMemcpyHostToDevice, st));
+  }
+  if (piped) {
+    // the copy stream starts after everything already queued on the caller's stream
+    FF_CUDA(p, cudaEventRecord(p->ev_copy[2 * FF_COPY_EVENTS], st));
+    FF_CUDA(p, cudaStreamWaitEvent(p->copy_stream, p->ev_copy[2 * FF_COPY_EVENTS], 0));
+    const void* src[3] = {Qh, Kh, Vh};
+    void* dst[3] = {p->buf.stage_q, p->buf.stage_k, p->buf.stage_v};
+    for (int g0 = 0, gi = 0; g0 < total; g0 += G, ++gi) {
+      const int g1 = g0 + G < total ? g0 + G : total;
+      for (int th = g0; th < g1;) {                 // a group may straddle two tensors
+        const int tensor = th / dm.BH, h = th % dm.BH;
+        const int n = (g1 - th) < (dm.BH - h) ? (g1 - th) : (dm.BH - h);
+        FF_CUDA(p, cudaMemcpyAsync((char*)dst[tensor] + (size_t)h * head_bytes, (const char*)src[tensor] + (size_t)h * head_bytes,
+                                   (size_t)n * head_bytes, cudaMemcpyHostToDevice, p->copy_stream));
+        th += n;
+      }
+      FF_CUDA(p, cudaEventRecord(p->ev_copy[gi], p->copy_stream));
+    }
+    p->pipe_in = p->pipe_out = true;
+    p->pipe_out_host = out_host;
+    p->pipe_head_bytes = head_bytes;
+  } else {
+    FF_CUDA(p, cudaMemcpyAsync(p->buf.stage_q, Qh, bytes, cudaMemcpyHostToDevice, st));
+    FF_CUDA(p, cudaMemcpyAsync(p->buf.stage_k, Kh, bytes, cudaMemcpyHostToDevice, st));
+    FF_CUDA(p, cudaMemcpyAsync(p->buf.stage_v, Vh, bytes, cudaMemcpyHostToDevice, st));
   }
   ff_status_t s = ff_forward(p, p->buf.stage_q, p->buf.stage_k, p->buf.stage_v, alloc_dev, timestep, p->buf.stage_out, st);
-  if (s != FF_OK) return s;
-  FF_CUDA(p, cudaMemcpyAsync(out_host, p->buf.stage_out, bytes, cudaMemcpyDeviceToHost, st));
+  const bool was_piped = p->pipe_out;
+  p->pipe_in = p->pipe_out = false;
+  if (s != FF_OK) { if (was_piped) cudaStreamSynchronize(p->copy_stream); return s; }
+  if (was_piped) {
+    FF_CUDA(p, cudaStreamSynchronize(p->copy_stream));
+  } else {
+    FF_CUDA(p, cudaMemcpyAsync(out_host, p->buf.stage_out, bytes, cudaMemcpyDeviceToHost, st));
+  }
   FF_CUDA(p, cudaStreamSynchronize(st));
   return FF_OK;
 }

@@ -673,6 +673,10 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
     const int g = total - g0 < G ? total - g0 : G;
     P.group = g; P.group_start = g0;
     cudaError_t e;
+    if (p->pipe_in) {                              // host-buffer entry point: this group's copy must have landed
+      e = cudaStreamWaitEvent(st, p->ev_copy[g0 / G], 0);
+      if (e != cudaSuccess) return e;
+    }
     if ((p->attn_impl & 4) && ffk_dct_wh_usable(dm, g, p->sm_count)) {
       // w and h passes in one launch, the intermediate staying in L2
       e = ffk_dct_wh_launch(p, 1, Q, K, V, g0, g, sc.ring, sc.b_hi, sc.b_lo, side, st);

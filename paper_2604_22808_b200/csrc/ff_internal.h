@@ -78,6 +78,8 @@ struct FFLayout {
   int tc_group;      // tensor-heads per tensor-core transform launch
 };
 
+constexpr int FF_COPY_EVENTS = 64;
+
 struct ff_plan {
   ff_config_t cfg;
   FFDims dm;
@@ -107,6 +109,13 @@ struct ff_plan {
   alignas(64) unsigned char tmap_low[128];     // ... over the pooled low band (bf16 copy), when low_tc_ok
   bool low_tc_ok;                              // the low branch runs in the tensor-core attention launch
   long long launches;
+  // ff_forward_host on the tensor-core path: copies run on a second stream, one event per launch
+  // group of the forward transform (host -> device) and of the inverse transform (device -> host)
+  cudaStream_t copy_stream;
+  cudaEvent_t ev_copy[2 * FF_COPY_EVENTS + 1];   // [0,64) input groups, [64,128) output groups, [128] start
+  bool pipe_in, pipe_out;                      // set for the duration of one ff_forward_host
+  void* pipe_out_host;                         // host destination of `out`
+  size_t pipe_head_bytes;                      // bytes of one (batch, head) slice of Q / K / V / out
   bool profiling;
   cudaEvent_t ev[FF_STAGE_COUNT + 1];
   long long stage_launches[FF_STAGE_COUNT];

@@ -684,6 +684,15 @@ static cudaError_t exchange_inverse_tc(ff_plan* p, void* out, cudaStream_t st) {
     p->launches += 1;
     e = ffk_inverse_transform_tc(p, h0, g, out, st);
     if (e != cudaSuccess) return e;
+    if (p->pipe_out) {                             // host-buffer entry point: hand this group of heads to the copy stream
+      cudaEvent_t ev = p->ev_copy[FF_COPY_EVENTS + h0 / G];
+      e = cudaEventRecord(ev, st);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(p->copy_stream, ev, 0);
+      if (e == cudaSuccess)
+        e = cudaMemcpyAsync((char*)p->pipe_out_host + (size_t)h0 * p->pipe_head_bytes, (const char*)out + (size_t)h0 * p->pipe_head_bytes,
+                            (size_t)g * p->pipe_head_bytes, cudaMemcpyDeviceToHost, p->copy_stream);
+      if (e != cudaSuccess) return e;
+    }
   }
   return cudaSuccess;
 }

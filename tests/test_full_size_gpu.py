@@ -101,3 +101,27 @@ def test_paper_reference_64k_full():
 def test_paper_reference_1m_full():
     """... at 1M tokens: N_low_bar = 32768 (dense low branch on the tensor cores), 1561 residue classes."""
     _run_full(C.PAPER_REF_1M, [0], per_band=1)
+
+
+def test_host_buffer_entry_point_64k_matches_device_path():
+    """Bench configuration of the end-to-end number: three copy groups in, one out; the result equals
+    the device-resident call's up to the last bits of the atomically accumulated summaries."""
+    import torch
+    from paper_2604_22808_b200 import binding as B
+    cfg = C.G64K
+    weights = I.router_weights(cfg)
+    q, k, v = _device_inputs(cfg)
+    out = torch.empty_like(q)
+    plan = B.Plan(cfg, weights, host_staging=True)
+    ts = [cfg.timesteps[0]] * cfg.batch
+    plan.forward(q, k, v, out, timesteps=ts)
+    torch.cuda.synchronize()
+    qh, kh, vh = (x.cpu().pin_memory() for x in (q, k, v))
+    oh = torch.empty_like(qh).pin_memory()
+    for _ in range(2):
+        oh.zero_()
+        plan.forward_host(qh, kh, vh, oh, timesteps=ts)
+        assert plan.device_status() == 0
+        diff = (oh.float() - out.cpu().float()).abs()
+        assert diff.max().item() <= 2e-2 and diff.mean().item() <= 1e-4
+    plan.destroy()

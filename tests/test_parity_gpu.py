@@ -316,3 +316,29 @@ def test_host_buffer_entry_point():
     plan.forward_host(qh, kh, vh, oh, alloc_host=np.array([7, 2], np.uint8))
     Hn.assert_close(oh.numpy()[0], res[0]["out"], "fp32", "host entry point")
     plan.destroy()
+
+
+def test_host_buffer_entry_point_pipelined():
+    """The host-buffer entry point on the tensor-core path (copies on a second stream, overlapped
+    with the transform groups) against the oracle, forced and routed allocation, twice in a row."""
+    import torch
+    from paper_2604_22808_b200 import binding as B
+    cfg = C.R128K                                        # batch 2
+    Q, K, V = Hn.host_inputs(cfg)
+    weights = I.router_weights(cfg)
+    U = I.summary_projection(cfg)
+    ts = [cfg.timesteps[0]] * cfg.batch
+    alloc = [PATTERN[i % 6] for i in range(cfg.batch * cfg.heads)]
+    plan = B.Plan(cfg, weights, host_staging=True)
+    qh, kh, vh = (torch.from_numpy(x).to(torch.bfloat16).pin_memory() for x in (Q, K, V))
+    oh = torch.empty_like(qh).pin_memory()
+    for forced in (True, False, True):
+        oh.zero_()
+        res = Hn.oracle_forward(cfg, Q, K, V, weights, U, ts, alloc=alloc if forced else None)
+        plan.forward_host(qh, kh, vh, oh, alloc_host=np.asarray(alloc, np.uint8) if forced else None, timesteps=ts)
+        assert plan.device_status() == 0
+        got = oh.float().numpy()
+        for bi in range(cfg.batch):
+            if forced or Hn.allocation_is_stable(res[bi]["pi"], cfg.heads):
+                Hn.assert_close(got[bi], res[bi]["out"], cfg.dtype, f"host entry point, sample {bi}")
+    plan.destroy()
