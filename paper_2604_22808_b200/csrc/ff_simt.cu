@@ -468,9 +468,15 @@ __global__ void summary_finalize_kernel(FFBuffers buf, const float* U, FFDims dm
 // tokens of the other two bands, and write the row at its coefficient position (fp32 grid).
 constexpr int EXC_WARPS = 8;
 
+// Coefficients per warp: up to 8, fewer when the launch would otherwise have too few blocks.
+static int exc_rounds(long long tokens, int g, int sm_count) {
+  long long r = tokens * g / ((long long)EXC_WARPS * 8 * sm_count);
+  return r < 1 ? 1 : (r > 8 ? 8 : (int)r);
+}
+
 template <typename ST, int DPL, typename OT>
 __global__ void __launch_bounds__(EXC_WARPS * 32) exchange_recombine_kernel(FFBuffers buf, FFDims dm, int bh0,
-                                                                             OT* grid_out, OT* grid_lo, int low_only) {
+                                                                             OT* grid_out, OT* grid_lo, int low_only, int rounds) {
   extern __shared__ float S[];   // [3][m][d]
   const int gi = blockIdx.y, bh = bh0 + gi;
   const int d = dm.d, m = dm.m;
@@ -478,9 +484,11 @@ __global__ void __launch_bounds__(EXC_WARPS * 32) exchange_recombine_kernel(FFBu
   __syncthreads();
   // low_only: the launch covers the low band's coefficients only (the other bands are exchanged
   // by the tensor-core kernel); the index is then a low rank, unravelled inside the low box.
-  long long f = (long long)blockIdx.x * EXC_WARPS + (threadIdx.x >> 5);
-  if (f >= (low_only ? dm.Nlow : dm.N)) return;
   const int lane = threadIdx.x & 31;
+  // a block stages the summaries once and then works through rounds x EXC_WARPS coefficients
+  for (int round = 0; round < rounds; ++round) {
+  long long f = ((long long)blockIdx.x * rounds + round) * EXC_WARPS + (threadIdx.x >> 5);
+  if (f >= (low_only ? dm.Nlow : dm.N)) return;
   int kw, kh, kt;
   if (low_only) {
     kw = (int)(f % dm.L[2]); kh = (int)((f / dm.L[2]) % dm.L[1]); kt = (int)(f / ((long long)dm.L[2] * dm.L[1]));
@@ -529,6 +537,7 @@ __global__ void __launch_bounds__(EXC_WARPS * 32) exchange_recombine_kernel(FFBu
     const float v = y[j] + acc[j];
     stf<OT>(dst + lane + 32 * j, v);
     if (grid_lo) stf<OT>(grid_lo + ((size_t)gi * dm.N + f) * d + lane + 32 * j, v - ldf<OT>(dst + lane + 32 * j));
+  }
   }
 }
 
@@ -651,12 +660,15 @@ cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st) {
 
 // Generic exchange + recombination into the hi/lo bf16 grids of the tensor-core inverse; DPL = d / 32.
 template <int DPL>
-static cudaError_t exchange_to_grids(ff_plan* p, dim3 grid, size_t smem, int h0, __nv_bfloat16* ghi, __nv_bfloat16* glo,
-                                     int low_only, cudaStream_t st) {
+static cudaError_t exchange_to_grids(ff_plan* p, long long tokens, int g, size_t smem, int h0, __nv_bfloat16* ghi,
+                                     __nv_bfloat16* glo, int low_only, cudaStream_t st) {
+  const int rounds = exc_rounds(tokens, g, p->sm_count);
+  const long long per_block = (long long)EXC_WARPS * rounds;
+  dim3 grid((unsigned)((tokens + per_block - 1) / per_block), (unsigned)g);
   cudaError_t e = cudaFuncSetAttribute(exchange_recombine_kernel<__nv_bfloat16, DPL, __nv_bfloat16>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  exchange_recombine_kernel<__nv_bfloat16, DPL, __nv_bfloat16><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, p->dm, h0, ghi, glo, low_only);
+  exchange_recombine_kernel<__nv_bfloat16, DPL, __nv_bfloat16><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, p->dm, h0, ghi, glo, low_only, rounds);
   return cudaGetLastError();
 }
 
@@ -668,17 +680,15 @@ static cudaError_t exchange_inverse_tc(ff_plan* p, void* out, cudaStream_t st) {
   cudaError_t e = cudaSuccess;
   for (int h0 = 0; h0 < dm.BH; h0 += G) {
     const int g = (dm.BH - h0 < G) ? dm.BH - h0 : G;
-    dim3 grid((unsigned)((dm.N + EXC_WARPS - 1) / EXC_WARPS), (unsigned)g);
     const size_t grid_bytes = ((size_t)G * dm.N * dm.d * 2 + 255) / 256 * 256;
     __nv_bfloat16* ghi = (__nv_bfloat16*)p->buf.scratchA;
     __nv_bfloat16* glo = (__nv_bfloat16*)((char*)p->buf.scratchA + grid_bytes);
     if (p->xtc_ok) {
       // mid and high bands on the tensor cores, the (small, fp32) low band with the generic kernel
-      dim3 lgrid((unsigned)((dm.Nlow + EXC_WARPS - 1) / EXC_WARPS), (unsigned)g);
-      e = dm.d == 128 ? exchange_to_grids<4>(p, lgrid, smem, h0, ghi, glo, 1, st) : exchange_to_grids<2>(p, lgrid, smem, h0, ghi, glo, 1, st);
+      e = dm.d == 128 ? exchange_to_grids<4>(p, dm.Nlow, g, smem, h0, ghi, glo, 1, st) : exchange_to_grids<2>(p, dm.Nlow, g, smem, h0, ghi, glo, 1, st);
       if (e == cudaSuccess) e = ffk_exchange_tc(p, h0, g, ghi, glo, st);
     } else {
-      e = dm.d == 128 ? exchange_to_grids<4>(p, grid, smem, h0, ghi, glo, 0, st) : exchange_to_grids<2>(p, grid, smem, h0, ghi, glo, 0, st);
+      e = dm.d == 128 ? exchange_to_grids<4>(p, dm.N, g, smem, h0, ghi, glo, 0, st) : exchange_to_grids<2>(p, dm.N, g, smem, h0, ghi, glo, 0, st);
     }
     if (e != cudaSuccess) return e;
     p->launches += 1;
@@ -706,11 +716,12 @@ static cudaError_t exchange_inverse_t(ff_plan* p, void* out, cudaStream_t st) {
   const size_t smem = (size_t)3 * dm.m * dm.d * sizeof(float);
   for (int h0 = 0; h0 < dm.BH; h0 += G) {
     const int g = (dm.BH - h0 < G) ? dm.BH - h0 : G;
-    dim3 grid((unsigned)((dm.N + EXC_WARPS - 1) / EXC_WARPS), (unsigned)g);
+    const int rounds = exc_rounds(dm.N, g, p->sm_count);
+    dim3 grid((unsigned)((dm.N + (long long)EXC_WARPS * rounds - 1) / ((long long)EXC_WARPS * rounds)), (unsigned)g);
     cudaError_t e = cudaSuccess;
 #define FF_EXC(DPL)                                                                                                   \
   e = cudaFuncSetAttribute(exchange_recombine_kernel<ST, DPL, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-  if (e == cudaSuccess) exchange_recombine_kernel<ST, DPL, float><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, dm, h0, p->buf.scratchA, (float*)nullptr, 0);
+  if (e == cudaSuccess) exchange_recombine_kernel<ST, DPL, float><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, dm, h0, p->buf.scratchA, (float*)nullptr, 0, rounds);
     switch (dm.d / 32) {
       case 1: FF_EXC(1) break;
       case 2: FF_EXC(2) break;
