@@ -234,7 +234,8 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     const int Lhw = dm.L[1] * dm.L[2], Mhw = dm.M[1] * dm.M[2];
     // (SPLIT) lane k of a warp accumulates the energies of channels 32 q + 2 (k % 16) + {0, 1} over the
     // warp's rows of parity k / 16: ea = mid + high rows, em = mid rows
-    float ea[NQ][2] = {}, em[NQ][2] = {}, el[NQ][2] = {};  // [chunk of the thread][channel of the pair]; el = low rows
+    float ea[NQ][2] = {}, em[NQ][2] = {};                 // [chunk of the thread][channel of the pair]
+    float el[NQ] = {};                                    // low rows, from the fp32 accumulators: lane k <-> channel 32 q + k
     int e_sample = -1;
     unsigned it = 0;
     bool ok = true;
@@ -247,9 +248,15 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
             const int c = (q_lo + qi) * 32 + 2 * (lane & 15) + e;
             atomicAdd(P.energy + ((size_t)e_sample * 3 + 1) * CH + c, (double)em[qi][e]);
             atomicAdd(P.energy + ((size_t)e_sample * 3 + 2) * CH + c, (double)(ea[qi][e] - em[qi][e]));
-            if (LOWACC) atomicAdd(P.energy + ((size_t)e_sample * 3 + 0) * CH + c, (double)el[qi][e]);
-            ea[qi][e] = em[qi][e] = el[qi][e] = 0.f;
+            ea[qi][e] = em[qi][e] = 0.f;
           }
+        if (LOWACC) {
+#pragma unroll
+          for (int qi = 0; qi < NQ; ++qi) {
+            atomicAdd(P.energy + ((size_t)e_sample * 3 + 0) * CH + (q_lo + qi) * 32 + lane, (double)el[qi]);
+            el[qi] = 0.f;
+          }
+        }
       }
     };
     for (int s = blockIdx.x; s < total_tiles && ok; s += gridDim.x, ++it) {
@@ -371,15 +378,23 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
                 if ((md >> (2 * i)) & 1) { m0 += s0; m1 += s1; }
               }
               ea[qi][0] += a0; ea[qi][1] += a1; em[qi][0] += m0; em[qi][1] += m1;
-              if (LOWACC && nonlow_rows != 0xffffffffu) {       // the warp holds low-band rows (rare)
-                float l0 = 0.f, l1 = 0.f;
+              if (LOWACC && nonlow_rows != 0xffffffffu) {
+                // The warp holds low-band rows (rare).  The low band has few coefficients per channel,
+                // so its energy is summed from the fp32 accumulators, not from the rounded staging
+                // copy: a halving butterfly over the warp's rows, after which lane k holds channel k.
+                float sa[32];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                  const uint32_t wd = *(const uint32_t*)(st_hi + (2 * i + par) * STG_PITCH + (((cp >> 2) ^ (i & 3)) << 4) + (cp & 3) * 4);
-                  const float v0 = __uint_as_float(wd << 16), v1 = __uint_as_float(wd & 0xffff0000u);
-                  if (!((nl >> (2 * i)) & 1)) { l0 = fmaf(v0, v0, l0); l1 = fmaf(v1, v1, l1); }
+                for (int i = 0; i < 32; ++i) { const float v = __uint_as_float(r[i]); sa[i] = band == 0 ? v * v : 0.f; }
+#pragma unroll
+                for (int step = 16; step >= 1; step >>= 1) {
+                  const bool upper = lane & step;
+#pragma unroll
+                  for (int i = 0; i < step; ++i) {
+                    const float keep = upper ? sa[i + step] : sa[i], send = upper ? sa[i] : sa[i + step];
+                    sa[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
+                  }
                 }
-                el[qi][0] += l0; el[qi][1] += l1;
+                el[qi] += sa[0];
               }
             }
 #pragma unroll
@@ -667,7 +682,7 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
   P.energy = want_energy ? p->buf.energy : nullptr;
   // A low box wider than a quarter of the w axis would make the fp32 side rows a large extra copy of the
   // data: take the low band from the tensor-core accumulators of the last pass instead.
-  P.low_from_acc = dm.L[2] * 4 > dm.W;
+  P.low_from_acc = true;
   P.spec_low = p->buf.spec_low;
   for (int g0 = 0; g0 < total; g0 += G) {
     const int g = total - g0 < G ? total - g0 : G;
