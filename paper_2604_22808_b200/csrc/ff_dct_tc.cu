@@ -24,13 +24,12 @@
 // bank conflicts) into its own staging area and one lane sends them out with a tensor store; the
 // area is reused when that store has read it.  SPLIT scatters rows to band positions: staged the
 // same way, then stored by all lanes with four lanes per 64-byte row piece.
-// Modes: FIRST  caller's Q/K/V -> hi/lo intermediate, plus an fp32 copy of the rows k_w < L_w
-//               from which the low band is computed at full precision
+// Modes: FIRST  caller's Q/K/V -> hi/lo intermediate
 //        MIDDLE hi/lo intermediate -> hi/lo intermediate
-//        SPLIT  intermediate -> band-major mid/high coefficient buffers (rank evaluated in
-//               registers) with the router's band energies accumulated from the stored (bf16) coefficients;
-//               for a low box wider than W/4 also the low band, in fp32 from the accumulators (the
-//               fp32 side rows and the low-band kernel are then skipped)
+//        SPLIT  intermediate -> band-major coefficient buffers (rank evaluated in registers): mid and
+//               high band in bf16, low band in fp32 straight from the accumulators (the hi/lo
+//               intermediates carry about 16 bits); the router's band energies are accumulated here,
+//               mid/high from the stored bf16 coefficients, low from the fp32 values
 //        LAST   intermediate -> the caller's out tensor
 #include <cuda.h>
 
@@ -63,10 +62,8 @@ struct DctTcParams {
   int group_start;         // index of the first one (tensor * BH + bh for the forward, bh for the inverse)
   int in_split;            // input is a hi/lo pair of grids (map0 = hi, map1 = lo)
   int nstage;              // ring depth
-  float* side;             // MODE_FIRST: [group][T][H][L_w][128] fp32
   __nv_bfloat16* spec_mid; __nv_bfloat16* spec_high;
-  float* spec_low;         // MODE_SPLIT with low_from_acc: [3 BH][N_low][d] fp32
-  int low_from_acc;        // the low band comes from the band-split pass's accumulators, not from the fp32 side rows
+  float* spec_low;         // MODE_SPLIT: [3 BH][N_low][d] fp32
   double* energy;          // [B][3][128]
   int* status;
 };
@@ -117,8 +114,7 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
 // Three source maps (Q, K, V) in MODE_FIRST; otherwise map0 (= hi) and, for split input, map1 (= lo).
 // map_oh / map_ol: destination hi / lo grids with the box of one epilogue warp (32 positions x 32
 // channels), all modes but SPLIT; MODE_LAST has no lo grid.
-// LOWACC: the low band comes from this kernel's band-split pass (see DctTcParams::low_from_acc).
-template <int CH, bool LOWACC>
+template <int CH>
 __global__ void __launch_bounds__(DCT_TC_THREADS, 1)
 dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
               const __grid_constant__ CUtensorMap map2, const __grid_constant__ CUtensorMap map_oh,
@@ -250,12 +246,10 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
             atomicAdd(P.energy + ((size_t)e_sample * 3 + 2) * CH + c, (double)(ea[qi][e] - em[qi][e]));
             ea[qi][e] = em[qi][e] = 0.f;
           }
-        if (LOWACC) {
 #pragma unroll
-          for (int qi = 0; qi < NQ; ++qi) {
-            atomicAdd(P.energy + ((size_t)e_sample * 3 + 0) * CH + (q_lo + qi) * 32 + lane, (double)el[qi]);
-            el[qi] = 0.f;
-          }
+        for (int qi = 0; qi < NQ; ++qi) {
+          atomicAdd(P.energy + ((size_t)e_sample * 3 + 0) * CH + (q_lo + qi) * 32 + lane, (double)el[qi]);
+          el[qi] = 0.f;
         }
       }
     };
@@ -284,8 +278,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
         const size_t th_slice = (size_t)tensor * dm.BH + bh;
         if (kt < dm.L[0] && hw_low) {
           band = 0;                                                                  // low band: fp32
-          if (LOWACC)
-            row_f32 = P.spec_low + (th_slice * dm.Nlow + (unsigned)((kt * dm.L[1] + h) * dm.L[2] + ww)) * CH;
+          row_f32 = P.spec_low + (th_slice * dm.Nlow + (unsigned)((kt * dm.L[1] + h) * dm.L[2] + ww)) * CH;
         } else if (kt < dm.M[0] && hw_mid) {
           const int offL = (h < dm.L[1] ? h : dm.L[1]) * dm.L[2] + (h < dm.L[1] ? (ww < dm.L[2] ? ww : dm.L[2]) : 0);
           const int cl = kt < dm.L[0] ? kt * Lhw + offL : (int)dm.Nlow;
@@ -295,8 +288,6 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
           band = 2;
           row_hi = P.spec_high + (th_slice * dm.Nhigh + (unsigned)(((kt * dm.H + h) * dm.W + ww) - cm)) * CH;
         }
-      } else if (P.mode == MODE_FIRST && a < dm.L[2] && !LOWACC) {
-        row_f32 = P.side + ((((size_t)gi * dm.T + t) * dm.H + h + l) * dm.L[2] + a) * CH;
       }
       // (SPLIT) lane L stores for rows 8 i + L/4 of its warp: fetch those rows' destinations
       __nv_bfloat16* dst_hi[4];
@@ -378,7 +369,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
                 if ((md >> (2 * i)) & 1) { m0 += s0; m1 += s1; }
               }
               ea[qi][0] += a0; ea[qi][1] += a1; em[qi][0] += m0; em[qi][1] += m1;
-              if (LOWACC && nonlow_rows != 0xffffffffu) {
+              if (nonlow_rows != 0xffffffffu) {
                 // The warp holds low-band rows (rare).  The low band has few coefficients per channel,
                 // so its energy is summed from the fp32 accumulators, not from the rounded staging
                 // copy: a halving butterfly over the warp's rows, after which lane k holds channel k.
@@ -423,95 +414,6 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     tc_fence_after();
     tmem_dealloc(tm, 512);
   }
-}
-
-// Low band at full precision from the fp32 copy of the w-transformed rows k_w < L_w:
-//   low[k_t][k_h][k_w][c] = sum_t C_T[k_t][t] sum_h C_H[k_h][h] side[t][h][k_w][c]
-// One CTA per (tensor-head, k_w) computes every (k_t, k_h) of the low box, in chunks of 8 x 8, so the
-// side buffer is read once per chunk pair; thread = (t group, channel); the t groups are combined
-// through shared memory.  Also accumulates the low band's energy.
-constexpr int LOW_CH = 8;        // k_h chunk
-constexpr int LOW_TG = 4;
-
-// LOW_CT = k_t chunk: the smallest of 2, 4, 8 that covers L_t keeps the accumulators (and with them
-// the registers per thread) small, so that more CTAs are resident and more loads in flight.
-// With few (k_w, tensor-head) pairs in a launch (large grids, small groups) the t axis is also split
-// over gridDim.z CTAs, which then add their parts into the zeroed output; the energy is summed by
-// low_energy_kernel afterwards.
-template <int LOW_CT, int CH>
-__global__ void __launch_bounds__(CH * LOW_TG) low_band_kernel(const float* side, const float* CT, const float* CHm,
-                                                               float* spec_low, double* energy, FFDims dm, int group_start) {
-  const int kw = blockIdx.x;
-  const int t_per = dm.T / (int)gridDim.z, t_lo = (int)blockIdx.z * t_per;   // this CTA's t range
-  const int gi = blockIdx.y, th = group_start + gi;
-  const int c = threadIdx.x % CH, tg = threadIdx.x / CH;     // threads = d x LOW_TG
-  __shared__ float ch_rows[LOW_CH][128];          // C_H rows of the current k_h chunk
-  __shared__ float red[LOW_CT * LOW_CH][CH];
-  float e = 0.f;
-  for (int kh0 = 0; kh0 < dm.L[1]; kh0 += LOW_CH) {
-    __syncthreads();
-    for (int i = threadIdx.x; i < LOW_CH * dm.H; i += CH * LOW_TG) {
-      const int q = i / dm.H, h = i % dm.H;
-      ch_rows[q][h] = kh0 + q < dm.L[1] ? CHm[(size_t)(kh0 + q) * dm.H + h] : 0.f;
-    }
-    for (int kt0 = 0; kt0 < dm.L[0]; kt0 += LOW_CT) {
-      for (int i = threadIdx.x; i < LOW_CT * LOW_CH * CH; i += CH * LOW_TG) red[i / CH][i % CH] = 0.f;
-      __syncthreads();
-      float acc[LOW_CT][LOW_CH];                    // [k_t][k_h]
-#pragma unroll
-      for (int i = 0; i < LOW_CT; ++i)
-#pragma unroll
-        for (int q = 0; q < LOW_CH; ++q) acc[i][q] = 0.f;
-      for (int t = t_lo + tg; t < t_lo + t_per; t += LOW_TG) {
-        const float* col = side + ((((size_t)gi * dm.T + t) * dm.H) * dm.L[2] + kw) * CH + c;
-        float s[LOW_CH];
-#pragma unroll
-        for (int q = 0; q < LOW_CH; ++q) s[q] = 0.f;
-        const size_t hs = (size_t)dm.L[2] * CH;
-        constexpr int NB = LOW_CT <= 4 ? 16 : 8;      // loads in flight (axis lengths are multiples of 16)
-        for (int h0 = 0; h0 < dm.H; h0 += NB) {
-          float x[NB];
-#pragma unroll
-          for (int u = 0; u < NB; ++u) x[u] = __ldg(col + (size_t)(h0 + u) * hs);
-#pragma unroll
-          for (int u = 0; u < NB; ++u)
-#pragma unroll
-            for (int q = 0; q < LOW_CH; ++q) s[q] = fmaf(ch_rows[q][h0 + u], x[u], s[q]);
-        }
-#pragma unroll
-        for (int i = 0; i < LOW_CT; ++i) {
-          const float ct = kt0 + i < dm.L[0] ? CT[(size_t)(kt0 + i) * dm.T + t] : 0.f;
-#pragma unroll
-          for (int q = 0; q < LOW_CH; ++q) acc[i][q] = fmaf(ct, s[q], acc[i][q]);
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < LOW_CT; ++i)
-#pragma unroll
-        for (int q = 0; q < LOW_CH; ++q)
-          if (kt0 + i < dm.L[0] && kh0 + q < dm.L[1]) atomicAdd(&red[i * LOW_CH + q][c], acc[i][q]);
-      __syncthreads();
-      for (int o = tg; o < LOW_CT * LOW_CH; o += LOW_TG) {
-        const int i = o / LOW_CH, q = o % LOW_CH;
-        if (kt0 + i >= dm.L[0] || kh0 + q >= dm.L[1]) continue;
-        const long long rank = ((long long)(kt0 + i) * dm.L[1] + kh0 + q) * dm.L[2] + kw;
-        const float v = red[o][c];
-        float* dst = spec_low + ((size_t)th * dm.Nlow + rank) * CH + c;
-        if (gridDim.z == 1) { *dst = v; e = fmaf(v, v, e); } else atomicAdd(dst, v);
-      }
-      __syncthreads();
-    }
-  }
-  if (energy && gridDim.z == 1) atomicAdd(energy + ((size_t)((th % dm.BH) / dm.heads) * 3) * CH + c, (double)e);
-}
-
-// Low-band energy of tensor-heads [group_start, group_start + gridDim.x): thread = channel.
-__global__ void low_energy_kernel(const float* spec_low, double* energy, FFDims dm, int group_start) {
-  const int th = group_start + blockIdx.x, c = threadIdx.x;
-  const float* v = spec_low + (size_t)th * dm.Nlow * dm.d + c;
-  float e = 0.f;
-  for (long long r = 0; r < dm.Nlow; ++r) { const float x = v[(size_t)r * dm.d]; e = fmaf(x, x, e); }
-  atomicAdd(energy + ((size_t)((th % dm.BH) / dm.heads) * 3) * dm.d + c, (double)e);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -583,13 +485,12 @@ cudaError_t launch_pass(ff_plan* p, const CUtensorMap& m0, const CUtensorMap& m1
   cudaError_t e = cudaSuccess;
   const int stages = (int)(P.group * (P.dm.N / TILE_ROWS));
   const int grid = stages < p->sm_count ? stages : p->sm_count;
-#define FF_DCT(D, LA)                                                                                              \
-  do {                                                                                                             \
-    e = cudaFuncSetAttribute(dct_tc_kernel<D, LA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
-    if (e == cudaSuccess) dct_tc_kernel<D, LA><<<grid, DCT_TC_THREADS, smem, st>>>(m0, m1, m2, moh, mol, P);       \
+#define FF_DCT(D)                                                                                              \
+  do {                                                                                                         \
+    e = cudaFuncSetAttribute(dct_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
+    if (e == cudaSuccess) dct_tc_kernel<D><<<grid, DCT_TC_THREADS, smem, st>>>(m0, m1, m2, moh, mol, P);       \
   } while (0)
-  if (P.dm.d == 128) { if (P.low_from_acc) FF_DCT(128, true); else FF_DCT(128, false); }
-  else { if (P.low_from_acc) FF_DCT(64, true); else FF_DCT(64, false); }
+  if (P.dm.d == 128) FF_DCT(128); else FF_DCT(64);
 #undef FF_DCT
   if (e != cudaSuccess) return e;
   p->launches += 1;
@@ -600,7 +501,7 @@ bool axis_ok(int n) { return n == 16 || n == 32 || n == 64 || n == 128; }
 
 }  // namespace
 
-// bf16, head_dim 128, power-of-two axis lengths 16..128, low box small enough for the fp32 side path.
+// bf16, head_dim 128 or 64, power-of-two axis lengths 16..128.
 bool ffk_dct_tc_supported(const FFDims& dm) {
   if (dm.fp32 || (dm.d != 128 && dm.d != 64) || !axis_ok(dm.T) || !axis_ok(dm.H) || !axis_ok(dm.W)) return false;
   // a tile groups 128/n lines: consecutive h for the w pass, consecutive w for the h and t passes
@@ -636,25 +537,22 @@ bool ffk_dct_tc_build_image(ff_plan* p, int axis, int inverse, const float* mat,
   return cudaMemcpy(p->dct_images + (size_t)2 * slot * TILE_BYTES, img.data(), 2 * TILE_BYTES, cudaMemcpyHostToDevice) == cudaSuccess;
 }
 
-// Scratch: two hi/lo pairs of bf16 grids and the fp32 side buffer for `group` tensor-heads.
+// Scratch: two hi/lo pairs of bf16 grids for `group` tensor-heads (and the fused w/h launch's ring).
 size_t ffk_dct_tc_scratch_bytes(const FFDims& dm, int group) {
   const size_t grid = (size_t)group * dm.N * dm.d * 2;
-  const size_t side = (size_t)group * dm.T * dm.H * dm.L[2] * dm.d * 4;
   const size_t ring = ffk_dct_wh_supported(dm) ? ffk_dct_wh_scratch_bytes(dm, group) : 0;
-  return 4 * ((grid + 255) / 256 * 256) + (side + 255) / 256 * 256 + (ring + 255) / 256 * 256;
+  return 4 * ((grid + 255) / 256 * 256) + (ring + 255) / 256 * 256;
 }
 
 namespace {
-struct Scratch { __nv_bfloat16 *a_hi, *a_lo, *b_hi, *b_lo; float* side; void* ring; };
+struct Scratch { __nv_bfloat16 *a_hi, *a_lo, *b_hi, *b_lo; void* ring; };
 Scratch carve(ff_plan* p) {
   const size_t grid_bytes = ((size_t)p->dct_group * p->dm.N * p->dm.d * 2 + 255) / 256 * 256;
   char* base = (char*)p->buf.scratchA;
   Scratch s;
   s.a_hi = (__nv_bfloat16*)base; s.a_lo = (__nv_bfloat16*)(base + grid_bytes);
   s.b_hi = (__nv_bfloat16*)(base + 2 * grid_bytes); s.b_lo = (__nv_bfloat16*)(base + 3 * grid_bytes);
-  s.side = (float*)(base + 4 * grid_bytes);
-  const size_t side_bytes = ((size_t)p->dct_group * p->dm.T * p->dm.H * p->dm.L[2] * p->dm.d * 4 + 255) / 256 * 256;
-  s.ring = base + 4 * grid_bytes + side_bytes;
+  s.ring = base + 4 * grid_bytes;
   return s;
 }
 }  // namespace
@@ -664,7 +562,6 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
   const FFDims& dm = p->dm;
   const int G = p->dct_group;
   const Scratch sc = carve(p);
-  float* side = sc.side;
   // mXh/mXl: load maps of a pass's input pair; oXh/oXl: store maps of a pass's output pair (the box
   // follows the axis of the pass that uses the map)
   CUtensorMap mq, mk, mv, m1h, m1l, m2h, m2l, o0h, o0l, o1h, o1l;
@@ -680,9 +577,6 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
   P.dm = dm; P.status = p->buf.status;
   P.spec_mid = (__nv_bfloat16*)p->buf.spec_mid; P.spec_high = (__nv_bfloat16*)p->buf.spec_high;
   P.energy = want_energy ? p->buf.energy : nullptr;
-  // A low box wider than a quarter of the w axis would make the fp32 side rows a large extra copy of the
-  // data: take the low band from the tensor-core accumulators of the last pass instead.
-  P.low_from_acc = true;
   P.spec_low = p->buf.spec_low;
   for (int g0 = 0; g0 < total; g0 += G) {
     const int g = total - g0 < G ? total - g0 : G;
@@ -694,11 +588,10 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
     }
     if ((p->attn_impl & 4) && ffk_dct_wh_usable(dm, g, p->sm_count)) {
       // w and h passes in one launch, the intermediate staying in L2
-      e = ffk_dct_wh_launch(p, 1, Q, K, V, g0, g, sc.ring, sc.b_hi, sc.b_lo, side, st);
+      e = ffk_dct_wh_launch(p, 1, Q, K, V, g0, g, sc.ring, sc.b_hi, sc.b_lo, nullptr, st);
       if (e != cudaSuccess) return e;
     } else {
       P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 2 + 0) * TILE_BYTES;
-      P.side = side;
       e = launch_pass(p, mq, mk, mv, o0h, o0l, P, st);
       if (e != cudaSuccess) return e;
       P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 1 + 0) * TILE_BYTES;
@@ -708,22 +601,6 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
     P.in_split = 1;
     P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 0 + 0) * TILE_BYTES;
     e = launch_pass(p, m2h, m2l, m2l, m2h, m2l, P, st);    // (no tensor stores in this mode)
-    if (e != cudaSuccess) return e;
-    if (P.low_from_acc) continue;                  // the band-split pass has written the low band already
-    int tz = 1;                                    // split t when the launch would not fill the GPU
-    while (dm.L[2] * g * tz < p->sm_count && tz * 2 * LOW_TG <= dm.T) tz *= 2;
-    dim3 lgrid((unsigned)dm.L[2], (unsigned)g, (unsigned)tz);
-    if (tz > 1) {
-      e = cudaMemsetAsync(p->buf.spec_low + (size_t)g0 * dm.Nlow * dm.d, 0, (size_t)g * dm.Nlow * dm.d * sizeof(float), st);
-      if (e != cudaSuccess) return e;
-    }
-#define FF_LOW(CT, D) low_band_kernel<CT, D><<<lgrid, D * LOW_TG, 0, st>>>(side, p->basis[0], p->basis[1], p->buf.spec_low, P.energy, dm, g0)
-    if (dm.d == 128) { if (dm.L[0] <= 2) FF_LOW(2, 128); else if (dm.L[0] <= 4) FF_LOW(4, 128); else FF_LOW(8, 128); }
-    else { if (dm.L[0] <= 2) FF_LOW(2, 64); else if (dm.L[0] <= 4) FF_LOW(4, 64); else FF_LOW(8, 64); }
-#undef FF_LOW
-    if (tz > 1 && P.energy) { low_energy_kernel<<<g, dm.d, 0, st>>>(p->buf.spec_low, P.energy, dm, g0); p->launches += 1; }
-    p->launches += 1;
-    e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;

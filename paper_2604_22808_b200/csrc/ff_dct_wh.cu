@@ -301,7 +301,7 @@ dct_wh_kernel(const __grid_constant__ CUtensorMap m0, const __grid_constant__ CU
       const int j0 = quarter * 32, a0 = j0 & (n - 1), l0 = j0 >> ln;
       const int bh0 = along_w ? x.u * kf + l0 : a0, bw0 = along_w ? a0 : x.u * kf + l0;
       float* row_f32 = nullptr;
-      if (!x.second && P.forward && a < dm.L[2]) row_f32 = P.side + ((((size_t)gi * dm.T + t) * dm.H + h) * dm.L[2] + a) * CH;
+      if (!x.second && P.forward && P.side && a < dm.L[2]) row_f32 = P.side + ((((size_t)gi * dm.T + t) * dm.H + h) * dm.L[2] + a) * CH;
       const CUtensorMap* mo_hi; const CUtensorMap* mo_lo;
       int c3, c4;
       uint64_t pol;
