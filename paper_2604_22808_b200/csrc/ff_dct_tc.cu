@@ -28,8 +28,9 @@
 //        MIDDLE hi/lo intermediate -> hi/lo intermediate
 //        SPLIT  intermediate -> band-major coefficient buffers (rank evaluated in registers): mid and
 //               high band in bf16, low band in fp32 straight from the accumulators (the hi/lo
-//               intermediates carry about 16 bits); the router's band energies are accumulated here,
-//               mid/high from the stored bf16 coefficients, low from the fp32 values
+//               intermediates carry about 16 bits); the router's mid and high band energies are
+//               accumulated here from the stored bf16 coefficients (the low band's, few values per
+//               channel, by low_energy_kernel from the fp32 coefficients)
 //        LAST   intermediate -> the caller's out tensor
 #include <cuda.h>
 
@@ -231,7 +232,6 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     // (SPLIT) lane k of a warp accumulates the energies of channels 32 q + 2 (k % 16) + {0, 1} over the
     // warp's rows of parity k / 16: ea = mid + high rows, em = mid rows
     float ea[NQ][2] = {}, em[NQ][2] = {};                 // [chunk of the thread][channel of the pair]
-    float el[NQ] = {};                                    // low rows, from the fp32 accumulators: lane k <-> channel 32 q + k
     int e_sample = -1;
     unsigned it = 0;
     bool ok = true;
@@ -246,11 +246,6 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
             atomicAdd(P.energy + ((size_t)e_sample * 3 + 2) * CH + c, (double)(ea[qi][e] - em[qi][e]));
             ea[qi][e] = em[qi][e] = 0.f;
           }
-#pragma unroll
-        for (int qi = 0; qi < NQ; ++qi) {
-          atomicAdd(P.energy + ((size_t)e_sample * 3 + 0) * CH + (q_lo + qi) * 32 + lane, (double)el[qi]);
-          el[qi] = 0.f;
-        }
       }
     };
     for (int s = blockIdx.x; s < total_tiles && ok; s += gridDim.x, ++it) {
@@ -369,24 +364,6 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
                 if ((md >> (2 * i)) & 1) { m0 += s0; m1 += s1; }
               }
               ea[qi][0] += a0; ea[qi][1] += a1; em[qi][0] += m0; em[qi][1] += m1;
-              if (nonlow_rows != 0xffffffffu) {
-                // The warp holds low-band rows (rare).  The low band has few coefficients per channel,
-                // so its energy is summed from the fp32 accumulators, not from the rounded staging
-                // copy: a halving butterfly over the warp's rows, after which lane k holds channel k.
-                float sa[32];
-#pragma unroll
-                for (int i = 0; i < 32; ++i) { const float v = __uint_as_float(r[i]); sa[i] = band == 0 ? v * v : 0.f; }
-#pragma unroll
-                for (int step = 16; step >= 1; step >>= 1) {
-                  const bool upper = lane & step;
-#pragma unroll
-                  for (int i = 0; i < step; ++i) {
-                    const float keep = upper ? sa[i + step] : sa[i], send = upper ? sa[i] : sa[i + step];
-                    sa[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
-                  }
-                }
-                el[qi] += sa[0];
-              }
             }
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -414,6 +391,23 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
     tc_fence_after();
     tmem_dealloc(tm, 512);
   }
+}
+
+// Low-band energy for the router: sum of squares of the fp32 low-band coefficients per channel,
+// over Q~, K~, V~ and the heads of a sample.  grid = (row chunks, 3 BH); thread = channel.
+__global__ void low_energy_kernel(const float* spec_low, double* energy, FFDims dm) {
+  const int th = blockIdx.y, c = threadIdx.x;
+  const long long per = (dm.Nlow + gridDim.x - 1) / gridDim.x;
+  const long long r0 = (long long)blockIdx.x * per, r1 = r0 + per < dm.Nlow ? r0 + per : dm.Nlow;
+  const float* v = spec_low + ((size_t)th * dm.Nlow) * dm.d + c;
+  float e0 = 0.f, e1 = 0.f;
+  long long r = r0;
+  for (; r + 1 < r1; r += 2) {
+    const float x0 = v[(size_t)r * dm.d], x1 = v[(size_t)(r + 1) * dm.d];
+    e0 = fmaf(x0, x0, e0); e1 = fmaf(x1, x1, e1);
+  }
+  if (r < r1) { const float x0 = v[(size_t)r * dm.d]; e0 = fmaf(x0, x0, e0); }
+  if (r0 < r1) atomicAdd(energy + ((size_t)((th % dm.BH) / dm.heads) * 3) * dm.d + c, (double)(e0 + e1));
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -601,6 +595,14 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
     P.in_split = 1;
     P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 0 + 0) * TILE_BYTES;
     e = launch_pass(p, m2h, m2l, m2l, m2h, m2l, P, st);    // (no tensor stores in this mode)
+    if (e != cudaSuccess) return e;
+  }
+  if (want_energy) {
+    long long chunks = (dm.Nlow + 511) / 512;             // about 512 rows per block
+    if (chunks > 256) chunks = 256;
+    low_energy_kernel<<<dim3((unsigned)chunks, (unsigned)total), dm.d, 0, st>>>(p->buf.spec_low, p->buf.energy, dm);
+    p->launches += 1;
+    const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
