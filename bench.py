@@ -32,7 +32,7 @@ METRIC = "freqformer_attn_layer_tokens_per_s"
 # capture summarised in profiles/dct_tc_kernel_64k_6heads.md (forward: three passes over Q, K and V;
 # inverse: three passes over one tensor).
 FP32_FMA_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 74.5: plain fp32 FMA rate of the GPU (unit counts x max clock)
-NCU_DRAM_BYTES_PER_TOKEN_HEAD = {"transform": 7532.0, "inverse": 3111.0}
+NCU_DRAM_BYTES_PER_TOKEN_HEAD = {"transform": 7330.0, "inverse": 3110.0}
 
 
 def measured_peaks():
