@@ -213,12 +213,12 @@ def router_probabilities(g: np.ndarray, e: np.ndarray, W1, b1, W2, b2):
 
 def head_quota(pi: np.ndarray, n_heads: int):
     """Heads per band from pi.  Reading: largest-remainder rounding of q_l = pi_l n_h (leftover
-    heads to the largest fractional parts, ties to the lower band).  The rounding is decided in
-    float32, the precision the device uses for this step.  Returns (counts[3], margin) where
-    margin is the smallest distance of the decision from flipping."""
-    q = (np.asarray(pi, np.float64).astype(np.float32) * np.float32(n_heads)).astype(np.float32)
+    heads to the largest fractional parts, ties to the lower band), in float64 like every other
+    step here.  Returns (counts[3], margin) where margin is the smallest distance of the decision
+    from flipping (a caller comparing with lower-precision arithmetic checks it first)."""
+    q = np.asarray(pi, np.float64) * float(n_heads)
     base = np.floor(q).astype(np.int64)
-    frac = (q - np.floor(q)).astype(np.float64)
+    frac = q - np.floor(q)
     left = int(n_heads - base.sum())
     order = sorted(range(3), key=lambda l: (-frac[l], l))
     counts = base.copy()

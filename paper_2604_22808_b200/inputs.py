@@ -104,13 +104,15 @@ def router_weights(cfg: FFConfig):
     return {"W1": W1, "b1": np.zeros(hid, np.float32), "W2": W2, "b2": np.zeros(3, np.float32)}
 
 
-def summary_projection(cfg: FFConfig, identity: bool = True) -> np.ndarray:
-    """U[3, d, d]: identity (the benchmark workloads) or a seeded random matrix of unit row scale."""
+def summary_projection(cfg: FFConfig, identity: bool = True, scale: float = 1.0) -> np.ndarray:
+    """U[3, d, d]: identity (the benchmark workloads) or a seeded random matrix whose rows have
+    norm `scale` on average (a small scale keeps the summary logits of a workload with large
+    low-frequency coefficients of order one)."""
     d = cfg.head_dim
     if identity:
         return np.broadcast_to(np.eye(d, dtype=np.float32), (3, d, d)).copy()
     g = _rng(cfg.seed, _STREAM_U, 0)
-    return (g.standard_normal((3, d, d)) / np.sqrt(d)).astype(np.float32)
+    return (g.standard_normal((3, d, d)) * (scale / np.sqrt(d))).astype(np.float32)
 
 
 def sample_rows(cfg: FFConfig, tag: int, length: int, count: int) -> np.ndarray:

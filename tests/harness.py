@@ -6,18 +6,64 @@ import numpy as np
 from oracle import freqformer_oracle as O
 from paper_2604_22808_b200 import inputs as I
 
-# Tolerances of the benchmark definition.  bf16 in / fp32 accumulate: max-abs 2e-2, max-rel 1e-2,
-# read elementwise as |g - o| <= max(2e-2, 1e-2 |o|) (an absolute bound alone cannot hold for a
-# bf16 result of magnitude > 8, whose own rounding step exceeds 2e-2).  fp32 workload: 5e-5.
+# Tolerances of the benchmark definition.  bf16 in / fp32 accumulate: "max-abs 2e-2 and max-rel 1e-2".
+# Two figures state that contract for a whole tensor: max|g - o| and max|g - o| / max(1, max|o|);
+# parity_report computes both.  What is asserted is an elementwise bound that implies the first
+# figure wherever a bf16 result can meet it and says what "relative" means where it cannot:
+#   |o| <  4:  |g - o| <= 2e-2  (a bf16 value below 4 has a rounding half-step <= 0.0078)
+#   |o| >= 4:  |g - o| <= max(2e-2, 1e-2 |o|)  and  |g - bf16(o)| <= one bf16 step of o: g is the
+#              oracle value rounded to the storage type, or its neighbour (the step is 0.031 from
+#              4 on and 0.0625 from 8 on, so no bf16 result can promise 2e-2 there)
+# fp32 workload: |g - o| <= 5e-5 max(1, |o|).
 BF16_ATOL, BF16_RTOL = 2e-2, 1e-2
 FP32_TOL = 5e-5
+BINS = ((0.0, 2.0), (2.0, 4.0), (4.0, 8.0), (8.0, np.inf))
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """float64 -> nearest bf16 (ties to even), as float64.  (Input generation's rounding helper,
+    applied to oracle values: storage rounding, no arithmetic of the method.)"""
+    return I.round_to_bf16(np.asarray(x, np.float32)).astype(np.float64)
+
+
+def bf16_step(o: np.ndarray) -> np.ndarray:
+    """Spacing of bf16 values at |o| (8 significand bits): 2^(floor(log2 |o|) - 7)."""
+    a = np.maximum(np.abs(np.asarray(o, np.float64)), 2.0 ** -126)
+    return 2.0 ** (np.floor(np.log2(a)) - 7.0)
 
 
 def tolerance(o: np.ndarray, dtype: str) -> np.ndarray:
     a = np.abs(o)
     if dtype == "fp32":
         return FP32_TOL * np.maximum(1.0, a)
-    return np.maximum(BF16_ATOL, BF16_RTOL * a)
+    return np.where(a < 4.0, BF16_ATOL, np.maximum(BF16_ATOL, BF16_RTOL * a))
+
+
+def parity_report(g, o) -> dict:
+    """The contract's two figures, the number of elements whose error exceeds 2e-2 binned by |o|,
+    and the same against the oracle value rounded to bf16 (separates the storage rounding of the
+    result from the error of the computation)."""
+    g = np.asarray(g, np.float64); o = np.asarray(o, np.float64)
+    err = np.abs(g - o)
+    errb = np.abs(g - bf16_round(o))
+    a = np.abs(o)
+    rep = {"max_abs": float(err.max()), "max_abs_over_scale": float(err.max() / max(1.0, a.max())),
+           "max_abs_vs_bf16_oracle": float(errb.max()), "max_oracle": float(a.max()), "n": int(err.size)}
+    over, overb = [], []
+    for lo, hi in BINS:
+        sel = (a >= lo) & (a < hi)
+        over.append(int((err[sel] > BF16_ATOL).sum()))
+        overb.append(int((errb[sel] > BF16_ATOL).sum()))
+    rep["over_2e-2_by_|o|_bin"] = over
+    rep["over_2e-2_vs_bf16_oracle_by_bin"] = overb
+    return rep
+
+
+def format_report(rep: dict) -> str:
+    return ("max|g-o| = %.3g, max|g-o|/max(1,max|o|) = %.3g (max|o| = %.3g), max|g-bf16(o)| = %.3g, "
+            "elements over 2e-2 for |o| in [0,2) [2,4) [4,8) [8,inf): %s; against bf16(o): %s; n = %d"
+            % (rep["max_abs"], rep["max_abs_over_scale"], rep["max_oracle"], rep["max_abs_vs_bf16_oracle"],
+               rep["over_2e-2_by_|o|_bin"], rep["over_2e-2_vs_bf16_oracle_by_bin"], rep["n"]))
 
 
 def assert_close(g, o, dtype: str, what: str = ""):
@@ -27,10 +73,14 @@ def assert_close(g, o, dtype: str, what: str = ""):
     err = np.abs(g - o)
     tol = tolerance(o, dtype)
     bad = err > tol
+    if dtype != "fp32":
+        # from 4 on: the oracle value rounded to bf16, or the neighbouring bf16 value
+        bad |= (np.abs(o) >= 4.0) & (np.abs(g - bf16_round(o)) > bf16_step(o) * (1 + 1e-9))
     if bad.any():
-        i = np.unravel_index(np.argmax(err - tol), err.shape)
+        i = np.unravel_index(np.argmax(np.where(bad, err - tol, -np.inf)), err.shape)
         raise AssertionError(f"{what}: {bad.sum()} of {bad.size} outside tolerance; worst at {i}: "
-                             f"gpu={g[i]:.6g} oracle={o[i]:.6g} err={err[i]:.3g} tol={tol[i]:.3g}")
+                             f"gpu={g[i]:.6g} oracle={o[i]:.6g} err={err[i]:.3g} tol={tol[i]:.3g}; "
+                             + (format_report(parity_report(g, o)) if dtype != "fp32" else ""))
     return float(err.max())
 
 

@@ -34,10 +34,10 @@ def _taps_check(cfg, plan, res, dtype):
                     Hn.assert_close(S[bh, l], taps["S"][h][l], dtype, f"S band {l} head {bh}")
 
 
-def _run(cfg, alloc=None, identity_U=True, timestep_index=0, impl=0, check_taps=True):
+def _run(cfg, alloc=None, identity_U=True, timestep_index=0, impl=0, check_taps=True, u_scale=1.0):
     Q, K, V = Hn.host_inputs(cfg)
     weights = I.router_weights(cfg)
-    U = I.summary_projection(cfg, identity=identity_U)
+    U = I.summary_projection(cfg, identity=identity_U, scale=u_scale)
     ts = [cfg.timesteps[timestep_index]] * cfg.batch
     res = Hn.oracle_forward(cfg, Q, K, V, weights, U, ts, alloc=alloc, want_taps=True)
     out, plan = Hn.gpu_forward(cfg, Q, K, V, weights, None if identity_U else U, timesteps=ts, alloc=alloc,
@@ -107,6 +107,17 @@ def test_replicas_bf16_forced_allocation(cfg):
 def test_replicas_bf16_routed(cfg):
     for ti in range(len(cfg.timesteps)):
         _run(cfg, timestep_index=ti, check_taps=(ti == 0))
+
+
+def test_smooth_replica_end_to_end_with_scaled_summaries():
+    """The replica of the workload with the smooth low-frequency component, end to end.  With identity
+    summary projections its exchange is ill-conditioned (tests/test_conditioning.py shows it with the
+    oracle alone); with projections scaled so that the summary logits are of order one, the whole
+    layer, large low-frequency coefficients included, has to match."""
+    from test_conditioning import WELL_CONDITIONED_U_SCALE
+    cfg = C.R256K
+    _run(cfg, alloc=[PATTERN[i % 6] for i in range(cfg.batch * cfg.heads)], identity_U=False, u_scale=WELL_CONDITIONED_U_SCALE)
+    _run(cfg, identity_U=False, u_scale=WELL_CONDITIONED_U_SCALE)          # routed
 
 
 @pytest.mark.parametrize("cfg", C.REPLICAS, ids=lambda c: c.name)
