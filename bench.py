@@ -29,10 +29,13 @@ from paper_2604_22808_b200 import inputs as I           # noqa: E402
 METRIC = "freqformer_attn_layer_tokens_per_s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the transform kernels per token and head, from the ncu
-# capture summarised in profiles/dct_tc_kernel_64k_6heads.md (forward: three passes over Q, K and V;
-# inverse: three passes over one tensor).
+# capture of the 6-head 64K case (forward: the passes over Q, K and V; inverse: the passes over one tensor).
 FP32_FMA_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 74.5: plain fp32 FMA rate of the GPU (unit counts x max clock)
 NCU_DRAM_BYTES_PER_TOKEN_HEAD = {"transform": 7330.0, "inverse": 3110.0}
+TRANSFORM_KERNELS = {"transform": "dct_tc_kernel (transform stage)", "inverse": "dct_tc_kernel (inverse stage)"}
+# Reported beside the 64K line by the default run: the larger workloads with the router's allocation and the
+# 64K grid with every band operator present.
+EXTRA_WORKLOADS = {"256k": ("256k", ""), "1m": ("1m", ""), "64k_forced_8_8_8": ("64k", "8,8,8")}
 
 
 def measured_peaks():
@@ -105,7 +108,12 @@ def layer_work(cfg, alloc):
                 bytes_attn += 4 * n_l * d * e
     heads = len(alloc)
     exch_pairs = heads * 2 * cfg.m * cfg.N
+    # forward transform, counted strictly: read Q, K, V, write V~ in full but Q~, K~ only for the bands the
+    # head's mask executes (what the band operators go on to read)
+    frac_exec = [sum(n_l for l, n_l in enumerate((n_low, n_mid, n_high)) if mask >> l & 1) / cfg.N for mask in alloc]
+    bytes_transform_strict = sum((4 + 2 * f) * u for f in frac_exec)
     return {
+        "bytes_transform_strict": bytes_transform_strict,
         "attn_flops": flops,
         "exchange_flops": 4 * d * exch_pairs,
         "transform_flops": heads * 4 * 2 * cfg.N * (cfg.T + cfg.H + cfg.W) * d,
@@ -123,14 +131,24 @@ class ClockSampler:
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, index: int):
+        """`index` is the CUDA device index; NVML numbers devices differently when CUDA_VISIBLE_DEVICES
+        is set, so the handle is looked up by the device's UUID (read-only queries throughout)."""
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
         self._thread = None
         try:
             import pynvml
+            import torch
             pynvml.nvmlInit()
             self._nv = pynvml
-            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            uuid = "GPU-" + str(torch.cuda.get_device_properties(index).uuid)
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                try:
+                    self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+                except Exception:
+                    self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
             self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
         except Exception:
             self._nv = None
@@ -145,7 +163,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            self._stop.wait(0.05)
+            self._stop.wait(0.01)
 
     def start(self):
         if self._nv is not None:
@@ -190,12 +208,34 @@ def oracle_sample_time(cfg, alloc):
     return cfg.batch * cfg.N / total, spent, cores, text
 
 
+# Head allocation the seeded random-init router produces at each workload's first timestep (heads per band and
+# sample), so that the reference arm times the same configuration as the CUDA arm without a GPU.  The fp64 oracle
+# yields the same counts (the full-size parity tests compare them).
+ROUTER_HEADS_PER_BAND = {"64k": (8, 0, 16), "256k": (0, 24, 0), "1m": (9, 6, 1), "paper_ref_64k": (0, 12, 4),
+                         "paper_ref_1m": (16, 0, 0)}
+
+
+def config_record(cfg, timestep, forced: bool, alloc):
+    io_mb = 3 * cfg.batch * cfg.heads * cfg.N * cfg.head_dim * (4 if cfg.dtype == "fp32" else 2) / 1e6
+    return {"workload": cfg.name, "grid": list(cfg.grid), "batch": cfg.batch, "heads": cfg.heads,
+            "head_dim": cfg.head_dim, "timestep": timestep, "allocation": "forced" if forced else "router",
+            "heads_per_band": [alloc.count(1), alloc.count(2), alloc.count(4)],
+            "l2": "inputs (%.0f MB) larger than L2" % io_mb}
+
+
 def run_reference(args, cfg):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     n = cfg.heads
-    alloc = [1] * (n // 3) + [2] * (n // 3) + [4] * (n - 2 * (n // 3))
+    forced = forced_allocation(cfg, args.alloc)
+    if forced is not None:
+        alloc = forced
+    elif cfg.name in ROUTER_HEADS_PER_BAND and args.timestep_index == 0:
+        c = ROUTER_HEADS_PER_BAND[cfg.name]
+        alloc = ([1] * c[0] + [2] * c[1] + [4] * c[2]) * cfg.batch
+    else:
+        alloc = ([1] * (n // 3) + [2] * (n // 3) + [4] * (n - 2 * (n // 3))) * cfg.batch
     vals = []
     t_all = time.perf_counter()
     for i in range(args.warmup + args.steps):
@@ -207,9 +247,10 @@ def run_reference(args, cfg):
     value = float(np.mean(vals))
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
             "steps": len(vals), "warmup": args.warmup, "ms_per_step": 1e3 * cfg.batch * cfg.N / value,
+            "ms_per_step_is": "extrapolated: each step times one head per allocated band type on the full grid "
+                              "(%.1f s of host work) and scales by the allocation" % spent,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "grid": list(cfg.grid), "heads": cfg.heads, "head_dim": cfg.head_dim,
-                       "allocation": "even split low/mid/high"},
+            "config": config_record(cfg, cfg.timesteps[args.timestep_index], forced is not None, alloc),
             "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": text},
             "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -259,6 +300,88 @@ def aggregate_tokens_per_s(cfg, world: int, ms_step_max: float) -> float:
 # ---------------------------------------------------------------------------------------------
 # The CUDA arm
 # ---------------------------------------------------------------------------------------------
+def stage_rooflines(cfg, alloc, stage_ms, peaks):
+    """Per stage: achieved algorithmic rate and its fraction of the measured peak that bounds it."""
+    work = layer_work(cfg, alloc)
+    ms = lambda name: max(stage_ms[name], 1e-9) * 1e-3
+    tc = tensor_core_path_any(cfg)
+    low_tc = band_sizes(cfg)[1] >= 128
+    issued = 4 * cfg.head_dim * sum(sum(p for l, p in enumerate(issued_pairs(cfg)) if (mk >> l & 1) and (l > 0 or low_tc))
+                                    for mk in alloc)
+    peak_t = peaks["bf16_tflops_sustained"]
+    out = {
+        "transform": {"bound": "hbm", "gbs": work["bytes_transform_strict"] / ms("transform") / 1e9,
+                      "gbs_all_bands_written": work["bytes_transform"] / ms("transform") / 1e9},
+        "inverse": {"bound": "hbm", "gbs": work["bytes_inverse"] / ms("inverse") / 1e9},
+        "attention": {"bound": "tensor" if tc else "alu", "useful_tflops": work["attn_flops"] / ms("attention") / 1e12,
+                      "issued_tflops": issued / ms("attention") / 1e12 if tc else None},
+    }
+    out["transform"]["frac"] = out["transform"]["gbs"] / peaks["hbm_gbs"]
+    out["inverse"]["frac"] = out["inverse"]["gbs"] / peaks["hbm_gbs"]
+    out["attention"]["frac"] = out["attention"]["useful_tflops"] / (peak_t if tc else FP32_FMA_TFLOPS)
+    out["attention"]["frac_of_nominal_2250"] = out["attention"]["useful_tflops"] / 2250.0 if tc else None
+    return out, work
+
+
+def time_forward(plan, q, k, v, out, alloc_dev, ts, steps, warmup, B, sampler=None):
+    """W untimed forwards, then K timed ones (CUDA events on the launching stream).  Returns the mean
+    ms per step, the sorted per-step times, the mean stage times and the launches per stage."""
+    import torch
+    for _ in range(warmup):
+        plan.forward(q, k, v, out, alloc=alloc_dev, timesteps=ts)
+    torch.cuda.synchronize()
+    if sampler is not None:
+        sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    stage_ms = {name: 0.0 for name in B.STAGES}
+    stage_launches = {}
+    ev[0].record()
+    for i in range(steps):
+        plan.forward(q, k, v, out, alloc=alloc_dev, timesteps=ts)
+        ev[i + 1].record()
+        for name, (ms, n) in plan.stage_times().items():       # waits for this step's last event
+            stage_ms[name] += ms / steps
+            stage_launches[name] = n
+    torch.cuda.synchronize()
+    per_step = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(steps))
+    return ev[0].elapsed_time(ev[-1]) / steps, per_step, stage_ms, stage_launches
+
+
+def extra_workload(name, alloc_text, args, dev, local, peaks):
+    """One more workload of the metric's 64K-1M range, device-timed only: inputs drawn on the GPU,
+    router-driven or forced allocation, stage times and per-stage roofline fractions."""
+    import torch
+    from paper_2604_22808_b200 import binding as B
+    cfg = C.BY_NAME[name]
+    q, k, v = (I.qkv_full_device(cfg, t, dev) for t in range(3))
+    out = torch.empty_like(q)
+    plan = B.Plan(cfg, I.router_weights(cfg), device=dev)
+    plan.set_profiling(True)
+    ts = [cfg.timesteps[0]] * cfg.batch
+    forced = forced_allocation(cfg, alloc_text)
+    alloc_dev = None if forced is None else torch.tensor(forced, dtype=torch.uint8, device=dev)
+    sampler = ClockSampler(local)
+    steps = max(3, min(args.steps, 10))
+    ms_step, per_step, stage_ms, stage_launches = time_forward(plan, q, k, v, out, alloc_dev, ts, steps, 3, B, sampler)
+    clocks = sampler.stop()
+    if plan.device_status() != 0:
+        raise RuntimeError(B.library().ff_last_error(plan.handle).decode())
+    alloc = forced if forced is not None else plan.tap(B.TAP_ALLOC).cpu().numpy().tolist()
+    stages, work = stage_rooflines(cfg, alloc, stage_ms, peaks)
+    res = {"grid": list(cfg.grid), "batch": cfg.batch, "heads": cfg.heads, "head_dim": cfg.head_dim,
+           "allocation": "router" if forced is None else "forced", "timestep": ts[0],
+           "heads_per_band": [alloc.count(1), alloc.count(2), alloc.count(4)],
+           "inputs": "drawn on the device (torch CUDA generator), same distribution as the parity tests' host inputs",
+           "steps": steps, "warmup": 3, "ms_per_step": ms_step, "ms_per_step_best": per_step[0],
+           "tokens_per_s": cfg.batch * cfg.N / (ms_step * 1e-3), "stages_ms": stage_ms, "stage_launches": stage_launches,
+           "stage_roofline": stages, "useful_attention_tflops_whole_step": work["attn_flops"] / (ms_step * 1e-3) / 1e12,
+           "clocks": clocks}
+    plan.destroy()
+    del q, k, v, out, plan
+    torch.cuda.empty_cache()
+    return res
+
+
 def run_cuda(args, cfg):
     import torch
     import torch.distributed as dist
@@ -274,12 +397,17 @@ def run_cuda(args, cfg):
 
     dt = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
     cfg_r = replica_config(cfg, rank)
-    host = [torch.from_numpy(I.qkv_full(cfg_r, t)).to(dt).pin_memory() for t in range(3)]
-    q, k, v = (x.to(dev, non_blocking=True) for x in host)
+    big = cfg.N * cfg.heads * cfg.batch > 3 * 2 ** 20            # drawing on the host would take minutes
+    if big:
+        q, k, v = (I.qkv_full_device(cfg_r, t, dev) for t in range(3))
+        host = None
+    else:
+        host = [torch.from_numpy(I.qkv_full(cfg_r, t)).to(dt).pin_memory() for t in range(3)]
+        q, k, v = (x.to(dev, non_blocking=True) for x in host)
     out = torch.empty_like(q)
-    out_host = torch.empty_like(host[0]).pin_memory()
     weights = I.router_weights(cfg)
-    plan = B.Plan(cfg, weights, host_staging=True, device=dev)
+    do_e2e = not args.no_e2e and host is not None
+    plan = B.Plan(cfg, weights, host_staging=do_e2e, device=dev)
     plan.set_profiling(True)
     plan.set_attention_impl(args.kernel_select)
     ts = [cfg.timesteps[args.timestep_index]] * cfg.batch
@@ -302,21 +430,10 @@ def run_cuda(args, cfg):
         plan.forward(q, k, v, out, alloc=alloc_dev, timesteps=ts)
     barrier()
     sampler = ClockSampler(local)
-    sampler.start()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    stage_ms = {name: 0.0 for name in B.STAGES}
-    stage_launches = {}
-    ev[0].record()
-    for i in range(args.steps):
-        plan.forward(q, k, v, out, alloc=alloc_dev, timesteps=ts)
-        ev[i + 1].record()
-        for name, (ms, n) in plan.stage_times().items():       # waits for this step's last event
-            stage_ms[name] += ms / args.steps
-            stage_launches[name] = n
+    ms_local, per_step, stage_ms, stage_launches = time_forward(plan, q, k, v, out, alloc_dev, ts, args.steps, 0, B, sampler)
     barrier()
     clocks = sampler.stop()
-    ms_step = reduce_max_(ev[0].elapsed_time(ev[-1]) / args.steps)
-    per_step = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps))     # this rank's steps
+    ms_step = reduce_max_(ms_local)
     launches = plan.last_launches()
     if plan.device_status() != 0:
         raise RuntimeError(B.library().ff_last_error(plan.handle).decode())
@@ -325,7 +442,8 @@ def run_cuda(args, cfg):
 
     # end to end through the host-buffer entry point (pinned host memory, copies inside the call)
     e2e_ms = float("nan")
-    if not args.no_e2e:
+    if do_e2e:
+        out_host = torch.empty_like(host[0]).pin_memory()
         for _ in range(min(2, args.warmup)):
             plan.forward_host(host[0], host[1], host[2], out_host, alloc_host=alloc_np, timesteps=ts)
         barrier()
@@ -336,36 +454,37 @@ def run_cuda(args, cfg):
         e2e_ms = reduce_max_((time.perf_counter() - t0) * 1e3 / e2e_steps)
         barrier()
 
+    io_bytes = q.numel() * q.element_size()
+    plan.destroy()
+    del q, k, v, out, plan
+    torch.cuda.empty_cache()
+
     if rank == 0:
         peaks = measured_peaks()
         tokens = cfg.batch * cfg.N * world
-        work = layer_work(cfg, alloc)
+        stages, work = stage_rooflines(cfg, alloc, stage_ms, peaks)
         # roofline of the dominant stage (achieved and traffic are per launch of the stage's kernel)
         top = max(stage_ms, key=stage_ms.get)
         n_launch = max(1, stage_launches.get(top) or 1)
         heads_total = cfg.batch * cfg.heads
         tensor_core_path = tensor_core_path_any(cfg)                         # otherwise the generic fp32 kernels run
-        if top == "attention" and tensor_core_path:
-            achieved = work["attn_flops"] / (stage_ms[top] * 1e-3) / 1e12
-            roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                    "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
-                    "kernel": "attention_tc_kernel"}
-        elif top == "attention":
-            # generic attention kernel: fp32 FMAs; peak = 148 SMs x 128 lanes x 2 FLOP x 1.965 GHz
-            achieved = work["attn_flops"] / (stage_ms[top] * 1e-3) / 1e12
-            roof = {"bound": "alu", "achieved": achieved, "peak": FP32_FMA_TFLOPS, "unit": "TFLOP/s",
-                    "frac": achieved / FP32_FMA_TFLOPS, "traffic": None, "kernel": "attention_simt_kernel"}
+        if top == "attention":
+            st = stages["attention"]
+            roof = {"bound": st["bound"], "achieved": st["useful_tflops"], "unit": "TFLOP/s", "frac": st["frac"],
+                    "peak": peaks["bf16_tflops_sustained"] if tensor_core_path else FP32_FMA_TFLOPS, "traffic": None,
+                    "kernel": "attention_tc_kernel" if tensor_core_path else "attention_simt_kernel"}
         else:
-            nbytes = work["bytes_transform"] if top == "transform" else work["bytes_inverse"]
-            achieved = nbytes / (stage_ms[top] * 1e-3) / 1e9
-            # DRAM bytes per token-head and stage from the ncu capture of the 6-head 64K case
-            # (profiles/dct_tc_kernel_64k_6heads.md); traffic is proportional to tokens x heads.
-            per_token_head = NCU_DRAM_BYTES_PER_TOKEN_HEAD[top]
-            roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"],
+            st = stages["transform" if top == "transform" else "inverse"]
+            nbytes = work["bytes_transform_strict"] if top == "transform" else work["bytes_inverse"]
+            # DRAM bytes per token-head and stage from the ncu capture of the 6-head 64K case; the traffic is
+            # proportional to tokens x heads
+            per_token_head = NCU_DRAM_BYTES_PER_TOKEN_HEAD[top] * cfg.head_dim / 128.0
+            roof = {"bound": "hbm", "achieved": st["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": st["frac"],
                     "traffic": per_token_head * cfg.N * heads_total / n_launch if tensor_core_path else None,
-                    "kernel": ("dct_tc_kernel (%s stage)" if tensor_core_path else "dct_pass_kernel (%s stage)") % top,
-                    "algorithmic_bytes_per_launch": nbytes / n_launch}
+                    "kernel": (TRANSFORM_KERNELS[top] if tensor_core_path else "dct_pass_kernel (%s stage)" % top),
+                    "algorithmic_bytes_per_launch": nbytes / n_launch,
+                    "algorithmic_bytes": "read Q,K,V, write V~ and the executed band of Q~,K~" if top == "transform"
+                                         else "read the band outputs once, write out once"}
         roof.update({"stage": top, "launches_per_step": stage_launches.get(top), "ms_per_step": stage_ms[top],
                      "ms_per_launch": stage_ms[top] / n_launch, "peak_source": peaks["source"]})
         cpu = None
@@ -373,38 +492,39 @@ def run_cuda(args, cfg):
             v_cpu, spent, cores, text = oracle_sample_time(cfg, alloc)
             cpu = {"value": v_cpu, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": text,
                    "seconds": spent}
-        io_bytes = q.numel() * q.element_size()
         line = {
             "metric": METRIC, "value": aggregate_tokens_per_s(cfg, world, ms_step), "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-            "config": {"workload": cfg.name, "grid": list(cfg.grid), "batch": cfg.batch, "heads": cfg.heads,
-                       "head_dim": cfg.head_dim, "timestep": ts[0], "allocation": "router" if forced is None else "forced",
-                       "heads_per_band": [alloc.count(1), alloc.count(2), alloc.count(4)], "pi": pi[0],
-                       "l2": "inputs (%.0f MB) larger than L2" % (3 * io_bytes / 1e6)},
+            "config": config_record(cfg, ts[0], forced is not None, alloc),
+            "router_pi": pi[0],
             "roofline": roof,
             "cpu_baseline": cpu,
-            "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 3 * io_bytes,
-                    "d2h_bytes_per_step": io_bytes, "ms_per_step": e2e_ms},
+            "e2e": ({"value": tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 3 * io_bytes,
+                     "d2h_bytes_per_step": io_bytes, "ms_per_step": e2e_ms} if do_e2e else None),
             "gpu_launches": launches * args.steps,
             "clocks": clocks,
             "stages_ms": stage_ms,
+            "stage_roofline": stages,
             "ms_per_step_median": per_step[len(per_step) // 2], "ms_per_step_best": per_step[0],
+            "ms_x_sm_mhz": ms_step * clocks["sm_mhz"] if clocks.get("sm_mhz") else None,
             "useful_attention_tflops": work["attn_flops"] / (ms_step * 1e-3) / 1e12,
-            # whole tiles the tensor-core kernel computes (masked parts included); the pooled low band only from 128 tokens on
-            "attention_stage_issued_tflops": (4 * cfg.head_dim * sum(
-                sum(p for l, p in enumerate(issued_pairs(cfg)) if (mk >> l & 1) and (l > 0 or band_sizes(cfg)[1] >= 128))
-                for mk in alloc) / (max(stage_ms["attention"], 1e-9) * 1e-3) / 1e12) if tensor_core_path_any(cfg) else None,
-            "attention_stage_tflops": work["attn_flops"] / (max(stage_ms["attention"], 1e-9) * 1e-3) / 1e12,
-            "transform_stage_gbs": work["bytes_transform"] / (max(stage_ms["transform"], 1e-9) * 1e-3) / 1e9,
-            "inverse_stage_gbs": work["bytes_inverse"] / (max(stage_ms["inverse"], 1e-9) * 1e-3) / 1e9,
+            "attention_stage_issued_tflops": stages["attention"]["issued_tflops"],
+            "attention_stage_tflops": stages["attention"]["useful_tflops"],
+            "transform_stage_gbs": stages["transform"]["gbs"],
+            "inverse_stage_gbs": stages["inverse"]["gbs"],
             "paper_context": "simulated estimates only: 9.3-27.3x attention-FLOP and 8.8-20.9x score-traffic reduction vs dense",
             # the same ratio for this workload and allocation, from the interaction counts (exchange included)
             "interaction_reduction_vs_dense": (len(alloc) * cfg.N * cfg.N) / max(1, work["attn_flops"] // (4 * cfg.head_dim)
                                                                               + len(alloc) * 2 * cfg.m * cfg.N),
         }
+        # The other workloads of the metric's range, device-timed in the same run (default invocation only)
+        if world == 1 and args.workload == "64k" and not args.alloc and not args.heads and not args.no_extra:
+            extra = {}
+            for key, (name, alloc_text) in EXTRA_WORKLOADS.items():
+                extra[key] = extra_workload(name, alloc_text, args, dev, local, peaks)
+            line["workloads"] = extra
         print(json.dumps(line))
-    plan.destroy()
     if world > 1:
         dist.destroy_process_group()
 
@@ -421,8 +541,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--heads", type=int, default=0, help="override the number of heads (profiling on a small case)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling)")
+    ap.add_argument("--no-extra", action="store_true", help="skip the additional workloads of the default run")
     ap.add_argument("--kernel-select", type=int, default=0,
-                    help="ff_plan_set_attention_impl bits: 1 generic attention, 2 generic transform, 4 fused w/h passes")
+                    help="ff_plan_set_attention_impl bits: 1 generic attention, 2 generic transform, 4 separate axis passes")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     cfg = C.BY_NAME[args.workload]

@@ -113,6 +113,10 @@ ff_status_t ff_plan_create(const ff_config_t *cfg, const ff_weights_t *weights, 
 
 ff_status_t ff_plan_workspace_bytes(const ff_plan_t *plan, size_t *bytes);
 
+/* Band sizes of the plan's configuration, as ff_band_sizes: N_low, ceil(N_low / r), N_mid, N_high
+ * ("Frequency band partitioning"). */
+ff_status_t ff_band_info(const ff_plan_t *plan, int64_t sizes[4]);
+
 /* Hand the plan its workspace (device memory owned by the caller, >= the size above, base
  * aligned to 256 bytes).  Must precede ff_route / ff_forward; may be called again. */
 ff_status_t ff_plan_set_workspace(ff_plan_t *plan, void *dev_ptr, size_t bytes);
@@ -213,9 +217,9 @@ enum {
 ff_status_t ff_get_tap(const ff_plan_t *plan, int32_t which, const void **dev_ptr, size_t *bytes);
 
 /* Kernel selection, a bit mask (0 = the defaults): 1 = generic SIMT attention instead of the
- * tensor-core kernel, 2 = generic SIMT transform instead of the tensor-core passes, 4 = w and h
- * passes fused in one launch with the intermediate kept in L2 (measured level with the separate
- * passes on B200; kept for experiments).  For tests and benchmarks.
+ * tensor-core kernel, 2 = generic SIMT transform instead of the tensor-core passes, 4 = the three
+ * axes of the tensor-core transform as separate passes (instead of two of them fused in one launch
+ * with the intermediate kept in shared memory).  For tests and benchmarks.
  * The tensor-core kernels cover bf16 storage with head_dim 128 or 64, axis lengths 16, 32, 64 or 128
  * and mid block sizes that tile 128 ranks; the pooled low band joins the tensor-core attention launch
  * from 128 pooled tokens on.  Every other configuration runs on the generic fp32 kernels. */
@@ -234,14 +238,18 @@ ff_status_t ff_plan_set_attention_impl(ff_plan_t *plan, int32_t impl);
  * an allocation implies, or a plug-in that is only ever given pointers.
  *
  *   q, k, v   device, bf16, contiguous [heads][n][128]: the band's tokens in band order
- *   y         device, bf16, [heads][n][128]: the operator's output (written by the call)
- *   heads     1 .. 1024;  n  1 .. 2^31-257;  larger sizes are rejected with FF_ERR_UNSUPPORTED
+ *   y         device, bf16, [heads][n][128]: the operator's output (written by the call); it must
+ *             not overlap q, k or v (other query tiles still read them while y is written)
+ *   heads     1 .. 1024;  n  1 .. 2^31-257;  heads * ceil(n / 256) < 2^31;  larger sizes are
+ *             rejected with FF_ERR_UNSUPPORTED
  *   sync      non-zero: synchronise the stream before returning and report a device-side
- *             FF_ERR_TIMEOUT; zero: return right after the launches
+ *             FF_ERR_TIMEOUT; zero: return right after the launches -- a device-side time-out is
+ *             then not reported at all (the next call clears the status word), so use zero only
+ *             where the caller synchronises and validates by its own means
  *
- * The kernel's scratch (worklist, per-head masks, status word: 16 KB) lives in a fixed array inside
- * the library image, so every GPU on which the library is loaded carries those 16 KB until the
- * process ends.  The first call on a device looks up the array's device address and sets the
+ * The kernel's scratch (worklist, per-head masks, status word: 13,824 bytes) lives in a fixed array
+ * inside the library image, so every GPU on which the library is loaded carries those bytes until
+ * the process ends.  The first call on a device looks up the array's device address and sets the
  * kernel's shared-memory limit; make that first call before starting any stream capture.  All calls
  * on a device share the one array, and it keeps what the previous call left: the call rewrites the
  * masks and the worklist and clears the status word itself, but two calls whose kernels overlap on

@@ -26,7 +26,7 @@ FF_BAND_LOW, FF_BAND_MID, FF_BAND_HIGH = 1, 2, 4
  TAP_ENERGY, TAP_ALLOC, TAP_PI) = range(11)
 
 EXPORTS = ("ff_config_validate", "ff_band_sizes", "ff_band_rank", "ff_workspace_bytes", "ff_workspace_bytes_host",
-           "ff_plan_create", "ff_plan_workspace_bytes", "ff_plan_set_workspace", "ff_destroy", "ff_last_error",
+           "ff_plan_create", "ff_plan_workspace_bytes", "ff_band_info", "ff_plan_set_workspace", "ff_destroy", "ff_last_error",
            "ff_route", "ff_forward", "ff_forward_host", "ff_plan_device_status", "ff_plan_last_launches",
            "ff_get_tap", "ff_plan_set_attention_impl", "ff_plan_set_profiling", "ff_plan_stage_times", "ff_high_attention_noalloc",
            "ff_plan_selftest_bounded_wait")
@@ -67,6 +67,7 @@ def library() -> C.CDLL:
         lib.ff_plan_create.argtypes = [C.POINTER(ff_config_t), C.POINTER(ff_weights_t), C.POINTER(C.c_void_p)]
         lib.ff_plan_workspace_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
         lib.ff_plan_set_workspace.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
+        lib.ff_band_info.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
         lib.ff_destroy.argtypes = [C.c_void_p]
         lib.ff_route.argtypes = [C.c_void_p] + [C.c_void_p] * 3 + [C.c_void_p] * 4 + [C.c_void_p]
         lib.ff_forward.argtypes = [C.c_void_p] + [C.c_void_p] * 3 + [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -147,6 +148,8 @@ class Plan:
         self.cfg = cfg
         self._torch = torch
         self.device = torch.device(device)
+        if self.device.index is None:
+            self.device = torch.device("cuda", torch.cuda.current_device())
         self.handle = C.c_void_p()
         lib = library()
         w = ff_weights_t()
@@ -178,6 +181,12 @@ class Plan:
         except Exception:
             pass
 
+    def band_info(self):
+        """(N_low, ceil(N_low / r), N_mid, N_high) of the plan's configuration."""
+        out = (C.c_int64 * 4)()
+        _check(library().ff_band_info(self.handle, out), self.handle)
+        return tuple(int(x) for x in out)
+
     def _stream(self):
         return C.c_void_p(self._torch.cuda.current_stream(self.device).cuda_stream)
 
@@ -190,6 +199,8 @@ class Plan:
         for t in tensors:
             if tuple(t.shape) != shape or t.dtype != self.torch_dtype or not t.is_contiguous():
                 raise FFError(1, f"expected a contiguous {self.torch_dtype} tensor of shape {shape}")
+            if not t.is_cuda or t.device != self.device:
+                raise FFError(1, f"expected a tensor on {self.device}, got one on {t.device}")
 
     # -- the path
     def route(self, Q, K, V, timesteps: Sequence[float], alloc_out=None, want_host: bool = True):
@@ -293,8 +304,9 @@ def ff_high_attention_noalloc(q, k, v, y, radius: int, sync: bool = True):
     synchronisation of an allocation.  Calls on one device share that scratch: do not overlap them."""
     import torch
     for t in (q, k, v, y):
-        if t.dtype != torch.bfloat16 or not t.is_contiguous() or t.dim() != 3 or t.shape[2] != 128 or t.shape != q.shape:
-            raise FFError(1, "expected contiguous bf16 CUDA tensors of one shape [heads][n][128]")
+        if (not t.is_cuda or t.device != q.device or t.dtype != torch.bfloat16 or not t.is_contiguous() or t.dim() != 3
+                or t.shape[2] != 128 or t.shape != q.shape):
+            raise FFError(1, "expected contiguous bf16 CUDA tensors of one shape [heads][n][128] on one device")
     stream = C.c_void_p(torch.cuda.current_stream(q.device).cuda_stream)
     with torch.cuda.device(q.device):
         _check(library().ff_high_attention_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), y.data_ptr(), q.shape[0],

@@ -167,7 +167,7 @@ extern "C" ff_status_t ff_destroy(ff_plan_t* p) {
     for (int i = 0; i <= 2 * FF_COPY_EVENTS; ++i) cudaEventDestroy(p->ev_copy[i]);
     cudaStreamDestroy(p->copy_stream);
   }
-  cudaFree(p->dct_images); cudaFree(p->pos_table);
+  cudaFree(p->dct_images); cudaFree(p->dct2_images); cudaFree(p->pos_table);
   cudaFree(p->W1); cudaFree(p->b1); cudaFree(p->W2); cudaFree(p->b2); cudaFree(p->U);
   delete p;
   return FF_OK;
@@ -206,7 +206,11 @@ extern "C" ff_status_t ff_plan_create(const ff_config_t* c, const ff_weights_t* 
     if (s == FF_OK && ffk_dct_tc_supported(p->dm) &&
         !(ffk_dct_tc_build_image(p, a, 0, C.data(), n[a]) && ffk_dct_tc_build_image(p, a, 1, Ct.data(), n[a])))
       s = fail(p, FF_ERR_CUDA, "could not upload the transform matrix images%s");
+    if (s == FF_OK && ffk_dct2_supported(p->dm, nullptr, nullptr) &&
+        !(ffk_dct2_build_image(p, a, 0, C.data(), n[a]) && ffk_dct2_build_image(p, a, 1, Ct.data(), n[a])))
+      s = fail(p, FF_ERR_CUDA, "could not upload the transform matrix images%s");
   }
+  p->dct2_ok = s == FF_OK && p->dct2_images && ffk_dct2_supported(p->dm, &p->dct2_axis2, nullptr);
   const size_t d = c->head_dim, hid = c->router_hidden, nin = 3 * d + c->t_embed_dim;
   if (s == FF_OK && w && w->W1 && w->b1 && w->W2 && w->b2) {
     s = upload(p, &p->W1, w->W1, hid * nin);
@@ -237,6 +241,12 @@ extern "C" ff_status_t ff_plan_create(const ff_config_t* c, const ff_weights_t* 
 extern "C" ff_status_t ff_plan_workspace_bytes(const ff_plan_t* p, size_t* bytes) {
   if (!p || !bytes) return fail(nullptr, FF_ERR_INVALID_ARG, "plan or bytes is NULL%s");
   *bytes = p->lay.total;
+  return FF_OK;
+}
+
+extern "C" ff_status_t ff_band_info(const ff_plan_t* p, int64_t sizes[4]) {
+  if (!p || !sizes) return fail(nullptr, FF_ERR_INVALID_ARG, "plan or sizes is NULL%s");
+  sizes[0] = p->dm.Nlow; sizes[1] = p->dm.Nbar; sizes[2] = p->dm.Nmid; sizes[3] = p->dm.Nhigh;
   return FF_OK;
 }
 

@@ -637,7 +637,7 @@ attention_tc_qkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
 }
 
 // Scratch of ff_high_attention_noalloc: the worklist, one band mask per head and a status word.
-// 16 KB in every GPU context that loads this library, held until the process exits.
+// 13,824 bytes in every GPU context that loads this library, held until the process exits.
 constexpr int NOALLOC_MAX_HEADS = MAX_UNITS;
 constexpr size_t NOALLOC_WORK_BYTES = ((2 + 3 * MAX_UNITS + 1) * sizeof(int) + 255) / 256 * 256;
 constexpr size_t NOALLOC_BYTES = NOALLOC_WORK_BYTES + NOALLOC_MAX_HEADS + 256;
@@ -736,6 +736,11 @@ extern "C" ff_status_t ff_high_attention_noalloc(const void* q, const void* k, c
   }
   if (heads > NOALLOC_MAX_HEADS || n >= (1LL << 31) - 256) {
     ff_set_thread_error("ff_high_attention_noalloc: the built-in scratch covers at most 1024 heads and 2^31-257 tokens per head");
+    return FF_ERR_UNSUPPORTED;
+  }
+  // the worklist counts items (pairs of 128-row query tiles) of all heads in 32 bits
+  if ((long long)heads * ((n + 2 * TILE - 1) / (2 * TILE)) >= (1LL << 31)) {
+    ff_set_thread_error("ff_high_attention_noalloc: heads x ceil(n / 256) must stay below 2^31");
     return FF_ERR_UNSUPPORTED;
   }
   // Device address of the scratch array, looked up once per device with that device current: in host

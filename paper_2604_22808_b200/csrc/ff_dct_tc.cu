@@ -263,25 +263,28 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
       if (P.mode == MODE_SPLIT) {
         const int sample = bh / dm.heads;
         if (sample != e_sample) { flush_energy(); e_sample = sample; }
-        // Band and rank of coefficient (k_t = a, h, w + l): the counts of box members below it are
-        // piecewise linear in the coordinates.
-        const int kt = a, ww = w + l;
-        const bool hw_low = h < dm.L[1] && ww < dm.L[2], hw_mid = h < dm.M[1] && ww < dm.M[2];
-        const int offM = (h < dm.M[1] ? h : dm.M[1]) * dm.M[2] + (h < dm.M[1] ? (ww < dm.M[2] ? ww : dm.M[2]) : 0);
+        // Band and rank of this row's coefficient: the pass axis supplies index a, the tile origin the
+        // other two (lines of a tile are neighbours along w for the t and h passes, along h for the w
+        // pass).  The counts of box members below a coefficient are piecewise linear in the coordinates.
+        const int kt = P.axis == 0 ? a : t;
+        const int h_ = P.axis == 1 ? a : (P.axis == 2 ? h + l : h);
+        const int ww = P.axis == 2 ? a : w + l;
+        const bool hw_low = h_ < dm.L[1] && ww < dm.L[2], hw_mid = h_ < dm.M[1] && ww < dm.M[2];
+        const int offM = (h_ < dm.M[1] ? h_ : dm.M[1]) * dm.M[2] + (h_ < dm.M[1] ? (ww < dm.M[2] ? ww : dm.M[2]) : 0);
         // (axis lengths are at most 128, so every count fits 32 bits)
         const int cm = kt < dm.M[0] ? kt * Mhw + offM : dm.M[0] * Mhw;
         const size_t th_slice = (size_t)tensor * dm.BH + bh;
         if (kt < dm.L[0] && hw_low) {
           band = 0;                                                                  // low band: fp32
-          row_f32 = P.spec_low + (th_slice * dm.Nlow + (unsigned)((kt * dm.L[1] + h) * dm.L[2] + ww)) * CH;
+          row_f32 = P.spec_low + (th_slice * dm.Nlow + (unsigned)((kt * dm.L[1] + h_) * dm.L[2] + ww)) * CH;
         } else if (kt < dm.M[0] && hw_mid) {
-          const int offL = (h < dm.L[1] ? h : dm.L[1]) * dm.L[2] + (h < dm.L[1] ? (ww < dm.L[2] ? ww : dm.L[2]) : 0);
+          const int offL = (h_ < dm.L[1] ? h_ : dm.L[1]) * dm.L[2] + (h_ < dm.L[1] ? (ww < dm.L[2] ? ww : dm.L[2]) : 0);
           const int cl = kt < dm.L[0] ? kt * Lhw + offL : (int)dm.Nlow;
           band = 1;
           row_hi = P.spec_mid + (th_slice * dm.Nmid + (unsigned)(cm - cl)) * CH;
         } else {
           band = 2;
-          row_hi = P.spec_high + (th_slice * dm.Nhigh + (unsigned)(((kt * dm.H + h) * dm.W + ww) - cm)) * CH;
+          row_hi = P.spec_high + (th_slice * dm.Nhigh + (unsigned)(((kt * dm.H + h_) * dm.W + ww) - cm)) * CH;
         }
       }
       // (SPLIT) lane L stores for rows 8 i + L/4 of its warp: fetch those rows' destinations
@@ -531,22 +534,20 @@ bool ffk_dct_tc_build_image(ff_plan* p, int axis, int inverse, const float* mat,
   return cudaMemcpy(p->dct_images + (size_t)2 * slot * TILE_BYTES, img.data(), 2 * TILE_BYTES, cudaMemcpyHostToDevice) == cudaSuccess;
 }
 
-// Scratch: two hi/lo pairs of bf16 grids for `group` tensor-heads (and the fused w/h launch's ring).
+// Scratch: two hi/lo pairs of bf16 grids for `group` tensor-heads.
 size_t ffk_dct_tc_scratch_bytes(const FFDims& dm, int group) {
   const size_t grid = (size_t)group * dm.N * dm.d * 2;
-  const size_t ring = ffk_dct_wh_supported(dm) ? ffk_dct_wh_scratch_bytes(dm, group) : 0;
-  return 4 * ((grid + 255) / 256 * 256) + (ring + 255) / 256 * 256;
+  return 4 * ((grid + 255) / 256 * 256);
 }
 
 namespace {
-struct Scratch { __nv_bfloat16 *a_hi, *a_lo, *b_hi, *b_lo; void* ring; };
+struct Scratch { __nv_bfloat16 *a_hi, *a_lo, *b_hi, *b_lo; };
 Scratch carve(ff_plan* p) {
   const size_t grid_bytes = ((size_t)p->dct_group * p->dm.N * p->dm.d * 2 + 255) / 256 * 256;
   char* base = (char*)p->buf.scratchA;
   Scratch s;
   s.a_hi = (__nv_bfloat16*)base; s.a_lo = (__nv_bfloat16*)(base + grid_bytes);
   s.b_hi = (__nv_bfloat16*)(base + 2 * grid_bytes); s.b_lo = (__nv_bfloat16*)(base + 3 * grid_bytes);
-  s.ring = base + 4 * grid_bytes;
   return s;
 }
 }  // namespace
@@ -556,15 +557,21 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
   const FFDims& dm = p->dm;
   const int G = p->dct_group;
   const Scratch sc = carve(p);
+  // Default: w and the shorter of h, t in one launch (intermediate on chip), then the band-split pass
+  // along the remaining axis.  Kernel-select bit 4: the three axes as separate passes w, h, t.
+  const bool fused = p->dct2_ok && !(p->attn_impl & 4);
+  const int last_axis = fused ? (p->dct2_axis2 == 1 ? 0 : 1) : 0;
+  const int last_n = last_axis == 0 ? dm.T : dm.H;
   // mXh/mXl: load maps of a pass's input pair; oXh/oXl: store maps of a pass's output pair (the box
   // follows the axis of the pass that uses the map)
-  CUtensorMap mq, mk, mv, m1h, m1l, m2h, m2l, o0h, o0l, o1h, o1l;
+  CUtensorMap mq, mk, mv, m1h, m1l, m2h, m2l, o0h, o0l, o1h, o1l, m3h, m3l;
   if (!encode_grid_map(&mq, Q, dm, dm.BH, 2) || !encode_grid_map(&mk, K, dm, dm.BH, 2) ||
       !encode_grid_map(&mv, V, dm, dm.BH, 2) || !encode_grid_map(&m1h, sc.a_hi, dm, G, 1) ||
       !encode_grid_map(&m1l, sc.a_lo, dm, G, 1) || !encode_grid_map(&m2h, sc.b_hi, dm, G, 0) ||
       !encode_grid_map(&m2l, sc.b_lo, dm, G, 0) || !encode_store_map(&o0h, sc.a_hi, dm, G, 2) ||
       !encode_store_map(&o0l, sc.a_lo, dm, G, 2) || !encode_store_map(&o1h, sc.b_hi, dm, G, 1) ||
-      !encode_store_map(&o1l, sc.b_lo, dm, G, 1))
+      !encode_store_map(&o1l, sc.b_lo, dm, G, 1) || !encode_grid_map(&m3h, sc.a_hi, dm, G, last_axis) ||
+      !encode_grid_map(&m3l, sc.a_lo, dm, G, last_axis))
     return cudaErrorInvalidValue;
   const int total = 3 * dm.BH;
   DctTcParams P{};
@@ -580,18 +587,21 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
       e = cudaStreamWaitEvent(st, p->ev_copy[g0 / G], 0);
       if (e != cudaSuccess) return e;
     }
-    if ((p->attn_impl & 4) && ffk_dct_wh_usable(dm, g, p->sm_count)) {
-      // w and h passes in one launch, the intermediate staying in L2
-      e = ffk_dct_wh_launch(p, 1, Q, K, V, g0, g, sc.ring, sc.b_hi, sc.b_lo, nullptr, st);
+    if (fused) {
+      e = ffk_dct2_forward(p, Q, K, V, g0, g, sc.a_hi, sc.a_lo, st);
       if (e != cudaSuccess) return e;
-    } else {
-      P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 2 + 0) * TILE_BYTES;
-      e = launch_pass(p, mq, mk, mv, o0h, o0l, P, st);
+      P.in_split = 1;
+      P.mode = MODE_SPLIT; P.axis = last_axis; P.n = last_n; P.image = p->dct_images + (size_t)(2 * last_axis + 0) * TILE_BYTES;
+      e = launch_pass(p, m3h, m3l, m3l, m3h, m3l, P, st);    // (no tensor stores in this mode)
       if (e != cudaSuccess) return e;
-      P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 1 + 0) * TILE_BYTES;
-      e = launch_pass(p, m1h, m1l, m1l, o1h, o1l, P, st);
-      if (e != cudaSuccess) return e;
+      continue;
     }
+    P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 2 + 0) * TILE_BYTES;
+    e = launch_pass(p, mq, mk, mv, o0h, o0l, P, st);
+    if (e != cudaSuccess) return e;
+    P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 1 + 0) * TILE_BYTES;
+    e = launch_pass(p, m1h, m1l, m1l, o1h, o1l, P, st);
+    if (e != cudaSuccess) return e;
     P.in_split = 1;
     P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 0 + 0) * TILE_BYTES;
     e = launch_pass(p, m2h, m2l, m2l, m2h, m2l, P, st);    // (no tensor stores in this mode)
@@ -613,21 +623,24 @@ cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaS
   const FFDims& dm = p->dm;
   const int G = p->dct_group;
   const Scratch sc = carve(p);
+  const bool fused = p->dct2_ok && !(p->attn_impl & 4);
+  const int first_axis = fused ? (p->dct2_axis2 == 1 ? 0 : 1) : 0;       // the axis the fused launch leaves out
+  const int first_n = first_axis == 0 ? dm.T : dm.H;
   CUtensorMap m_in, m_inl, mbh, mbl, mah, mal, obh, obl, oah, oal, mout;
-  if (!encode_grid_map(&m_in, sc.a_hi, dm, G, 0) || !encode_grid_map(&m_inl, sc.a_lo, dm, G, 0) ||
+  if (!encode_grid_map(&m_in, sc.a_hi, dm, G, first_axis) || !encode_grid_map(&m_inl, sc.a_lo, dm, G, first_axis) ||
       !encode_grid_map(&mbh, sc.b_hi, dm, G, 1) ||
       !encode_grid_map(&mbl, sc.b_lo, dm, G, 1) || !encode_grid_map(&mah, sc.a_hi, dm, G, 2) ||
-      !encode_grid_map(&mal, sc.a_lo, dm, G, 2) || !encode_store_map(&obh, sc.b_hi, dm, G, 0) ||
-      !encode_store_map(&obl, sc.b_lo, dm, G, 0) || !encode_store_map(&oah, sc.a_hi, dm, G, 1) ||
+      !encode_grid_map(&mal, sc.a_lo, dm, G, 2) || !encode_store_map(&obh, sc.b_hi, dm, G, first_axis) ||
+      !encode_store_map(&obl, sc.b_lo, dm, G, first_axis) || !encode_store_map(&oah, sc.a_hi, dm, G, 1) ||
       !encode_store_map(&oal, sc.a_lo, dm, G, 1) || !encode_store_map(&mout, out, dm, dm.BH, 2))
     return cudaErrorInvalidValue;
   DctTcParams P{};
   P.dm = dm; P.status = p->buf.status; P.group = g; P.group_start = h0;
-  P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 3 + 0) * TILE_BYTES;
+  P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = first_axis; P.n = first_n;
+  P.image = p->dct_images + (size_t)(2 * (3 + first_axis) + 0) * TILE_BYTES;
   cudaError_t e = launch_pass(p, m_in, m_inl, m_inl, obh, obl, P, st);
   if (e != cudaSuccess) return e;
-  if ((p->attn_impl & 4) && ffk_dct_wh_usable(dm, g, p->sm_count))
-    return ffk_dct_wh_launch(p, 0, sc.b_hi, sc.b_lo, nullptr, h0, g, sc.ring, out, nullptr, nullptr, st);
+  if (fused) return ffk_dct2_inverse(p, sc.b_hi, sc.b_lo, h0, g, out, st);
   P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 4 + 0) * TILE_BYTES;
   e = launch_pass(p, mbh, mbl, mbl, oah, oal, P, st);
   if (e != cudaSuccess) return e;

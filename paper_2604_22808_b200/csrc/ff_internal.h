@@ -104,6 +104,10 @@ struct ff_plan {
   int* pos_table;                              // rank -> flat coefficient index of the mid, then the high band (plan-owned)
   alignas(64) unsigned char tmap_x[4][128];    // CUtensorMaps of the exchange kernel (Y / V~ of the mid and high bands)
   uint8_t* dct_images;                         // 6 x (hi, lo) matrix images of the tensor-core transform (plan-owned)
+  uint32_t* dct2_images;                       // the same matrices as tensor-memory operands of the fused two-axis launch
+  bool dct2_ok;                                // the fused two-axis launch covers this configuration
+  int dct2_axis2;                              // its second axis (1 = h, 0 = t); the remaining axis gets a pass of its own
+  int dct2_clusters;                           // clusters of that launch the device runs at once (0 = not yet asked)
   alignas(64) unsigned char tmap_mid[128];     // CUtensorMap over the mid-band / high-band coefficient buffers
   alignas(64) unsigned char tmap_high[128];
   alignas(64) unsigned char tmap_low[128];     // ... over the pooled low band (bf16 copy), when low_tc_ok
@@ -150,12 +154,11 @@ size_t ffk_dct_tc_scratch_bytes(const FFDims& dm, int group);
 cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, const void* V, bool want_energy,
                                      cudaStream_t st);
 cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaStream_t st);
-// ---- fused w/h passes (ff_dct_wh.cu) ---------------------------------------------------------------
-bool ffk_dct_wh_supported(const FFDims& dm);
-void ffk_dct_wh_shape(const FFDims& dm, int* ring, int* lag);
-bool ffk_dct_wh_usable(const FFDims& dm, int g, int sm_count);
-size_t ffk_dct_wh_scratch_bytes(const FFDims& dm, int group);
-cudaError_t ffk_dct_wh_launch(ff_plan* p, int forward, const void* src0, const void* src1, const void* src2, int g0, int g,
-                              void* ring, void* out_hi, void* out_lo, float* side, cudaStream_t st);
+// ---- two axis passes in one launch, intermediate in shared memory (ff_dct2_tc.cu) --------------------
+bool ffk_dct2_supported(const FFDims& dm, int* axis2, int* cs);
+bool ffk_dct2_build_image(ff_plan* p, int axis, int inverse, const float* mat_host, int n);
+cudaError_t ffk_dct2_forward(ff_plan* p, const void* Q, const void* K, const void* V, int g0, int g, void* out_hi, void* out_lo,
+                             cudaStream_t st);
+cudaError_t ffk_dct2_inverse(ff_plan* p, const void* in_hi, const void* in_lo, int h0, int g, void* out, cudaStream_t st);
 cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st);
 cudaError_t ffk_exchange_inverse(ff_plan* p, void* out, cudaStream_t st);

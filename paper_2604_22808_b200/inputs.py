@@ -93,6 +93,36 @@ def qkv_full(cfg: FFConfig, tensor: int) -> np.ndarray:
     return out
 
 
+def qkv_full_device(cfg: FFConfig, tensor: int, device):
+    """[B, heads, T, H, W, d] for one of Q, K, V, drawn on the GPU: the same distribution as
+    qkv_full (i.i.d. N(0,1) plus the workload's smooth component, rounded to the storage type)
+    from torch's counter-based CUDA generator, seeded by (workload seed, tensor).  For benchmark
+    runs at sizes where drawing on the host would take minutes; the values differ from qkv_full's,
+    so parity tests keep to the host generator."""
+    import torch
+    dt = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
+    out = torch.empty((cfg.batch, cfg.heads, cfg.T, cfg.H, cfg.W, cfg.head_dim), dtype=dt, device=device)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(1000003 * cfg.seed + 101 * tensor + 7)
+    axes = None
+    if cfg.smooth_cosines:
+        freqs = smooth_frequencies(cfg)
+        axes = []
+        for n, col in zip(cfg.grid, range(3)):
+            i = np.arange(n, dtype=np.float64)
+            a = np.cos(np.pi * (2.0 * i[:, None] + 1.0) * freqs[None, :, col] / (2.0 * n))
+            axes.append(torch.from_numpy(a.astype(np.float32)).to(device))
+        wave = torch.einsum("tj,hj,wj->thwj", axes[0], axes[1], axes[2]).reshape(cfg.N, -1)      # [N, J]
+    for bi in range(cfg.batch):
+        for h in range(cfg.heads):
+            x = torch.randn((cfg.N, cfg.head_dim), generator=gen, device=device, dtype=torch.float32)
+            if cfg.smooth_cosines:
+                sig = torch.from_numpy(smooth_signs(cfg, tensor, bi, h)).to(device)                 # [d, J]
+                x += cfg.smooth_amplitude * (wave @ sig.T)
+            out[bi, h].copy_(x.view(cfg.T, cfg.H, cfg.W, cfg.head_dim))
+    return out
+
+
 def router_weights(cfg: FFConfig):
     """Random-init router MLP: W1 ~ N(0, 1/in), W2 ~ N(0, 16/hidden), zero biases.
     Drawn in a fixed order (W1 row-major, then W2) from the workload's seed."""

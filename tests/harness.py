@@ -66,14 +66,17 @@ def format_report(rep: dict) -> str:
                rep["over_2e-2_by_|o|_bin"], rep["over_2e-2_vs_bf16_oracle_by_bin"], rep["n"]))
 
 
-def assert_close(g, o, dtype: str, what: str = ""):
+def assert_close(g, o, dtype: str, what: str = "", stored_bf16: bool = True):
+    """`stored_bf16`: the compared values were rounded to bf16 by the device (the mid and high
+    bands' buffers and the output of a bf16 workload); False for what it keeps in fp32 (low band,
+    summary tokens), where the neighbour rule of the storage type does not apply."""
     g = np.asarray(g, np.float64); o = np.asarray(o, np.float64)
     assert g.shape == o.shape, (what, g.shape, o.shape)
     assert np.all(np.isfinite(g)), f"{what}: non-finite values"
     err = np.abs(g - o)
     tol = tolerance(o, dtype)
     bad = err > tol
-    if dtype != "fp32":
+    if dtype != "fp32" and stored_bf16:
         # from 4 on: the oracle value rounded to bf16, or the neighbouring bf16 value
         bad |= (np.abs(o) >= 4.0) & (np.abs(g - bf16_round(o)) > bf16_step(o) * (1 + 1e-9))
     if bad.any():
@@ -189,7 +192,8 @@ def stagewise_check(cfg, plan, Q, K, V, out_gpu, weights, U, timesteps, routed: 
                     rows = I.sample_rows(cfg, 1000 * bh + 10 * t + l, sizes[l], n_rows)
                     g = spec_taps[l][t, bh][rows].float().cpu().numpy()
                     dt = "fp32" if cfg.dtype == "fp32" else "bf16"
-                    errs["spectral"] = max(errs["spectral"], assert_close(g, ob[l][rows], dt, f"spectral t{t} band {l} head {bh}"))
+                    errs["spectral"] = max(errs["spectral"], assert_close(g, ob[l][rows], dt, f"spectral t{t} band {l} head {bh}",
+                                                                          stored_bf16=l > 0))
             if not checked:
                 continue
             Qo, Ko, Vo = bands
@@ -209,12 +213,14 @@ def stagewise_check(cfg, plan, Q, K, V, out_gpu, weights, U, timesteps, routed: 
                     op = O.mid_operator if l == 1 else O.high_operator
                     args = (cfg.b, cfg.s) if l == 1 else (cfg.R,)
                     ref, _ = op(Qo[l], Ko[l], Vo[l], *args, rows=rows)
-                errs["attention"] = max(errs["attention"], assert_close(Yg[l][rows], ref, cfg.dtype, f"Y band {l} head {bh}"))
+                errs["attention"] = max(errs["attention"], assert_close(Yg[l][rows], ref, cfg.dtype, f"Y band {l} head {bh}",
+                                                                        stored_bf16=l > 0))
             # summaries of the working outputs the device holds
             if m > 0:
                 for l in range(3):
                     ref = O.summary_tokens(Yg[l], Uo[l], m)
-                    errs["summary"] = max(errs["summary"], assert_close(S_tap[bh, l], ref, cfg.dtype, f"S band {l} head {bh}"))
+                    errs["summary"] = max(errs["summary"], assert_close(S_tap[bh, l], ref, cfg.dtype, f"S band {l} head {bh}",
+                                                                        stored_bf16=False))
             # exchange + recombination + inverse transform from the device's Y and S
             if bh in inverse_heads:
                 spec = np.zeros((cfg.N, d))

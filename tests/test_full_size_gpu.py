@@ -35,6 +35,32 @@ def _pick_heads(alloc, per_band=2):
     return sorted(set(picked))
 
 
+def _run_forced(cfg, heads_per_band, per_band=1):
+    """Full size with a forced allocation (heads [0,L) low, next M mid, rest high, per sample): the
+    seeded router gives some workloads no head of one band type, so every (workload, band) pair is
+    also run -- and compared on sampled rows -- under a mask that has it."""
+    import torch
+    from paper_2604_22808_b200 import binding as B
+    assert sum(heads_per_band) == cfg.heads
+    masks = ([1] * heads_per_band[0] + [2] * heads_per_band[1] + [4] * heads_per_band[2]) * cfg.batch
+    weights = I.router_weights(cfg)
+    U = I.summary_projection(cfg)
+    q, k, v = _device_inputs(cfg)
+    out = torch.empty_like(q)
+    plan = B.Plan(cfg, weights)
+    plan.forward(q, k, v, out, alloc=torch.tensor(masks, dtype=torch.uint8, device="cuda"))
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    assert plan.tap(B.TAP_ALLOC).cpu().numpy().tolist() == masks
+    heads = _pick_heads(masks, per_band)
+    source = lambda t, bi, h: (q, k, v)[t][bi, h].float().cpu().numpy()
+    errs = Hn.stagewise_check(cfg, plan, None, None, None, lambda bi, h: out[bi, h].float().cpu().numpy(), weights, U,
+                              [cfg.timesteps[0]] * cfg.batch, routed=False, check_heads=heads, inverse_heads=heads,
+                              head_source=source)
+    print(cfg.name, "forced", heads_per_band, "checked heads", heads, errs)
+    plan.destroy()
+
+
 def _run_full(cfg, timestep_indices, per_band=2):
     import torch
     from paper_2604_22808_b200 import binding as B
@@ -91,6 +117,18 @@ def test_1m_full():
 
 def test_128k_sweep_full():
     _run_full(C.G128K, [0, 1, 2, 3, 4], per_band=1)
+
+
+def test_64k_full_forced_allocation():
+    _run_forced(C.G64K, (8, 8, 8))
+
+
+def test_256k_full_forced_allocation():
+    _run_forced(C.G256K, (8, 8, 8))
+
+
+def test_128k_full_forced_allocation():
+    _run_forced(C.G128K, (8, 8, 8))
 
 
 def test_paper_reference_64k_full():
