@@ -38,6 +38,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", os.path.join(PKG, "csrc"),
            "-o", LIB] + sources()
+    cmd[1:1] = os.environ.get("FF_NVCC_FLAGS", "").split()      # e.g. -DFF_DEBUG: the build with device-side range checks
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
