@@ -73,7 +73,20 @@ typedef struct {
   int32_t n_summary;       /* m >= 0 summary tokens per band; 0 disables the exchange */
   int32_t router_hidden;   /* hidden width of the two-layer router MLP */
   int32_t t_embed_dim;     /* d_t, even: width of the sinusoidal timestep embedding */
+  int32_t transform;       /* FF_TRANSFORM_DCT or FF_TRANSFORM_HAAR: the 1-D transform of every axis */
+  int32_t mid_pattern;     /* FF_MID_STRIDED or FF_MID_ANCHOR: the mid band's sparse pattern */
 } ff_config_t;
+
+/* "Separable spectral decomposition" / "Transform choice": the reference design's orthonormal DCT-II,
+ * or the orthonormal Haar wavelet transform (power-of-two axis lengths; rows from the coarsest scale
+ * to the finest, so the nested-box bands keep their meaning). */
+enum { FF_TRANSFORM_DCT = 0, FF_TRANSFORM_HAAR = 1 };
+
+/* "Mid band: structured block-sparse attention" / "Mid-band sparse degree".  Blocks of b consecutive
+ * ranks, block index J.  STRIDED: query block J sees key blocks J' with (J' - J) mod s == 0.  ANCHOR:
+ * query block J sees its own block and every anchor block J' = s-1 (mod s): a fixed set of "connector"
+ * blocks shared by all queries plus the local block. */
+enum { FF_MID_STRIDED = 0, FF_MID_ANCHOR = 1 };
 
 /* Host arrays, copied at ff_plan_create.  Router input is [g_low; g_mid; g_high; e(t)]
  * (3*head_dim + t_embed_dim values).  NULL router pointers => ff_route / internal routing

@@ -19,7 +19,8 @@ number for them, so they are pinned by invariants and special cases only
 (dense-attention reductions, identities, brute force), not by paper values.
 
 `cfg` arguments are duck-typed records with fields
-T, H, W, heads, head_dim, low_cut, mid_cut, r, b, s, R, m, t_embed_dim.
+T, H, W, heads, head_dim, low_cut, mid_cut, r, b, s, R, m, t_embed_dim and, optionally,
+transform ("dct" or "haar") and mid_pattern ("strided" or "anchor").
 """
 from __future__ import annotations
 
@@ -46,23 +47,54 @@ def dct_matrix(n: int) -> np.ndarray:
     return C
 
 
-def forward_transform(X: np.ndarray) -> np.ndarray:
+def haar_matrix(n: int) -> np.ndarray:
+    """Orthonormal Haar wavelet matrix for n a power of two ("wavelets are also possible";
+    "Transform choice").  Row 0 is the constant 1/sqrt(n); row 2^j + k (level j, shift k) is
+    +sqrt(2^j / n) on the first half and -sqrt(2^j / n) on the second half of the k-th block of
+    n / 2^j positions, zero elsewhere.  Rows run from the coarsest scale to the finest, so a low
+    row index is a coarse scale, as a low DCT index is a low frequency."""
+    if n < 1 or n & (n - 1):
+        raise ValueError("the Haar transform needs a power-of-two axis length")
+    Hm = np.zeros((n, n), dtype=np.float64)
+    Hm[0, :] = 1.0 / math.sqrt(n)
+    row, j = 1, 0
+    while row < n:
+        block = n >> j                       # support of a level-j wavelet
+        amp = math.sqrt((1 << j) / n)
+        for k in range(1 << j):
+            Hm[row, k * block:k * block + block // 2] = amp
+            Hm[row, k * block + block // 2:(k + 1) * block] = -amp
+            row += 1
+        j += 1
+    return Hm
+
+
+def transform_matrix(n: int, kind: str = "dct") -> np.ndarray:
+    """The fixed orthonormal 1-D transform of one axis: DCT-II (the reference design) or Haar."""
+    if kind == "dct":
+        return dct_matrix(n)
+    if kind == "haar":
+        return haar_matrix(n)
+    raise ValueError(f"unknown transform {kind!r}")
+
+
+def forward_transform(X: np.ndarray, kind: str = "dct") -> np.ndarray:
     """X~ = (F_t (x) F_h (x) F_w) X for X[T, H, W, d]: each token axis is multiplied by its
     1-D matrix; the channel axis is untouched (the Kronecker product has no channel factor)."""
     T, H, W, d = X.shape
-    Y = (dct_matrix(T) @ X.reshape(T, H * W * d)).reshape(T, H, W, d)
-    Y = (dct_matrix(H)[None] @ Y.reshape(T, H, W * d)).reshape(T, H, W, d)
-    Y = dct_matrix(W)[None, None] @ Y
+    Y = (transform_matrix(T, kind) @ X.reshape(T, H * W * d)).reshape(T, H, W, d)
+    Y = (transform_matrix(H, kind)[None] @ Y.reshape(T, H, W * d)).reshape(T, H, W, d)
+    Y = transform_matrix(W, kind)[None, None] @ Y
     return Y
 
 
-def inverse_transform(Y: np.ndarray) -> np.ndarray:
+def inverse_transform(Y: np.ndarray, kind: str = "dct") -> np.ndarray:
     """F^{-1}: the transposes of the orthonormal 1-D matrices along each token axis
     ("Reconstruction": mapped back into token space via the inverse transform)."""
     T, H, W, d = Y.shape
-    X = dct_matrix(W).T[None, None] @ Y
-    X = (dct_matrix(H).T[None] @ X.reshape(T, H, W * d)).reshape(T, H, W, d)
-    X = (dct_matrix(T).T @ X.reshape(T, H * W * d)).reshape(T, H, W, d)
+    X = transform_matrix(W, kind).T[None, None] @ Y
+    X = (transform_matrix(H, kind).T[None] @ X.reshape(T, H, W * d)).reshape(T, H, W, d)
+    X = (transform_matrix(T, kind).T @ X.reshape(T, H * W * d)).reshape(T, H, W, d)
     return X
 
 
@@ -127,17 +159,25 @@ def dense_attention(Q: np.ndarray, K: np.ndarray, V: np.ndarray) -> np.ndarray:
     return softmax_rows(Q @ K.T / math.sqrt(d)) @ V
 
 
-def mid_allowed(p, pk, b: int, s: int):
+def mid_allowed(p, pk, b: int, s: int, pattern: str = "strided"):
     """The mid-band sparse pattern S ("block-local plus strided").  Reading: blocks of b
-    consecutive mid ranks; query p sees key pk iff their block indices differ by a multiple of
-    the stride s (the own block included).  This is the single place the pattern is defined."""
-    return ((np.asarray(pk) // b - np.asarray(p) // b) % s) == 0
+    consecutive mid ranks.  "strided": query p sees key pk iff their block indices differ by a
+    multiple of the stride s (the own block included).  "anchor" (the alternative of the
+    "Mid-band sparse degree" ablation): the own block plus every anchor block, the blocks whose
+    index is s-1 mod s ("strided connectors" shared by all queries).  This is the single place
+    the pattern is defined."""
+    Jk, Jq = np.asarray(pk) // b, np.asarray(p) // b
+    if pattern == "strided":
+        return ((Jk - Jq) % s) == 0
+    if pattern == "anchor":
+        return (Jk == Jq) | ((Jk % s) == s - 1)
+    raise ValueError(f"unknown mid pattern {pattern!r}")
 
 
-def mid_keys(p: int, n: int, b: int, s: int) -> np.ndarray:
+def mid_keys(p: int, n: int, b: int, s: int, pattern: str = "strided") -> np.ndarray:
     """Key set of mid-band query p among n tokens, increasing."""
     pk = np.arange(n)
-    return pk[mid_allowed(p, pk, b, s)]
+    return pk[mid_allowed(p, pk, b, s, pattern)]
 
 
 def high_keys(p: int, n: int, R: int) -> np.ndarray:
@@ -167,10 +207,10 @@ def sparse_attention_rows(Q: np.ndarray, K: np.ndarray, V: np.ndarray, rows: np.
     return out, pairs
 
 
-def mid_operator(Q, K, V, b: int, s: int, rows: Optional[np.ndarray] = None):
+def mid_operator(Q, K, V, b: int, s: int, rows: Optional[np.ndarray] = None, pattern: str = "strided"):
     n = Q.shape[0]
     rows = np.arange(n) if rows is None else rows
-    return sparse_attention_rows(Q, K, V, rows, lambda p: mid_keys(p, n, b, s))
+    return sparse_attention_rows(Q, K, V, rows, lambda p: mid_keys(p, n, b, s, pattern))
 
 
 def high_operator(Q, K, V, R: int, rows: Optional[np.ndarray] = None):
@@ -283,6 +323,7 @@ def forward_sample(cfg, Q, K, V, weights, U, timestep: float, alloc=None, want_t
     N = T * H * W
     members = band_members(grid, cfg.low_cut, cfg.mid_cut)
     sizes = [len(ix) for ix in members]
+    kind = getattr(cfg, "transform", "dct")
     counters = {"pairs_low": 0, "pairs_mid": 0, "pairs_high": 0, "pairs_exchange": 0,
                 "transform_macs": 0}
 
@@ -290,7 +331,7 @@ def forward_sample(cfg, Q, K, V, weights, U, timestep: float, alloc=None, want_t
     esum = np.zeros((3, d))
     for h in range(n_h):
         for X, dst in ((Q[h], Qb), (K[h], Kb), (V[h], Vb)):
-            bands = split_bands(forward_transform(X), members)
+            bands = split_bands(forward_transform(X, kind), members)
             dst.append(bands)
             esum += band_energy_sums(bands)
             counters["transform_macs"] += N * (T + H + W) * d
@@ -317,7 +358,8 @@ def forward_sample(cfg, Q, K, V, weights, U, timestep: float, alloc=None, want_t
         else:
             Y[0] = Vb[h][0]
         if mask & BAND_MID and sizes[1]:
-            Y[1], pairs = mid_operator(Qb[h][1], Kb[h][1], Vb[h][1], cfg.b, cfg.s)
+            Y[1], pairs = mid_operator(Qb[h][1], Kb[h][1], Vb[h][1], cfg.b, cfg.s,
+                                       pattern=getattr(cfg, "mid_pattern", "strided"))
             counters["pairs_mid"] += pairs
         else:
             Y[1] = Vb[h][1]
@@ -347,7 +389,7 @@ def forward_sample(cfg, Q, K, V, weights, U, timestep: float, alloc=None, want_t
             low = decompress_low(low, cfg.r, sizes[0])
         for l, rows in enumerate((low, Yhat[1], Yhat[2])):
             spec[members[l]] = rows
-        out[h] = inverse_transform(spec.reshape(T, H, W, d))
+        out[h] = inverse_transform(spec.reshape(T, H, W, d), kind)
         counters["transform_macs"] += N * (T + H + W) * d
         if want_taps:
             taps["Y"].append(Y); taps["S"].append(S); taps["Yhat"].append(Yhat)
@@ -378,9 +420,14 @@ def dense_attention_flops(N: int, d_k: int) -> int:
     return 2 * d_k * N * N
 
 
-def mid_interactions(n_mid: int, b: int, s: int) -> int:
-    """Sum over residue classes of (tokens in the class)^2."""
+def mid_interactions(n_mid: int, b: int, s: int, pattern: str = "strided") -> int:
+    """Scored pairs of the mid band.  Strided: sum over residue classes of (tokens in the
+    class)^2.  Anchor: every token sees the anchor blocks, and its own block if that is none."""
     nb = -(-n_mid // b)
+    size = lambda J: min(b, n_mid - J * b)
+    if pattern == "anchor":
+        anchors = sum(size(J) for J in range(nb) if J % s == s - 1)
+        return sum(size(J) * (anchors + (0 if J % s == s - 1 else size(J))) for J in range(nb))
     total = 0
     for c in range(min(s, nb)):
         n_c = sum(min(b, n_mid - J * b) for J in range(c, nb, s))

@@ -14,7 +14,9 @@ import numpy as np
 
 from .configs import FFConfig
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libfreqformer.so")
+# FF_LIBRARY_VARIANT=debug loads the build with device-side range checks (python -m paper_2604_22808_b200.build --debug)
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)),
+                         "libfreqformer_debug.so" if os.environ.get("FF_LIBRARY_VARIANT") == "debug" else "libfreqformer.so")
 _lib = None
 
 FF_OK = 0
@@ -38,7 +40,7 @@ class ff_config_t(C.Structure):
                 ("head_dim", C.c_int32), ("dtype", C.c_int32), ("low_cut", C.c_int32 * 3), ("mid_cut", C.c_int32 * 3),
                 ("low_compress", C.c_int32), ("mid_block", C.c_int32), ("mid_stride", C.c_int32),
                 ("high_radius", C.c_int32), ("n_summary", C.c_int32), ("router_hidden", C.c_int32),
-                ("t_embed_dim", C.c_int32)]
+                ("t_embed_dim", C.c_int32), ("transform", C.c_int32), ("mid_pattern", C.c_int32)]
 
 
 class ff_weights_t(C.Structure):
@@ -98,6 +100,8 @@ def c_config(cfg: FFConfig) -> ff_config_t:
     c.mid_cut = (C.c_int32 * 3)(*cfg.mid_cut)
     c.low_compress, c.mid_block, c.mid_stride, c.high_radius = cfg.r, cfg.b, cfg.s, cfg.R
     c.n_summary, c.router_hidden, c.t_embed_dim = cfg.m, cfg.router_hidden, cfg.t_embed_dim
+    c.transform = {"dct": 0, "haar": 1}[cfg.transform]
+    c.mid_pattern = {"strided": 0, "anchor": 1}[cfg.mid_pattern]
     return c
 
 

@@ -44,6 +44,9 @@ class FFConfig:
     timesteps: Tuple[float, ...] = (500.0,)
     smooth_cosines: int = 0         # number of separable cosines added to every tensor
     smooth_amplitude: float = 0.0
+    transform: str = "dct"          # 1-D transform of every axis: "dct" (DCT-II, the reference design) or "haar"
+    mid_pattern: str = "strided"    # mid-band sparse pattern: "strided" (own block + blocks at distance 0 mod s)
+                                    # or "anchor" (own block + the anchor blocks J = s-1 mod s)
 
     @property
     def N(self) -> int:

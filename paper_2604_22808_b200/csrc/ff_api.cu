@@ -34,6 +34,7 @@ static void dims_from_cfg(const ff_config_t& c, FFDims* dm) {
   dm->r = c.low_compress; dm->b = c.mid_block; dm->s = c.mid_stride; dm->R = c.high_radius;
   dm->m = c.n_summary; dm->hid = c.router_hidden; dm->dt = c.t_embed_dim;
   dm->fp32 = (c.dtype == FF_FP32);
+  dm->pattern = c.mid_pattern;
   dm->N = (long long)c.T * c.H * c.W;
   dm->Nlow = (long long)c.low_cut[0] * c.low_cut[1] * c.low_cut[2];
   dm->Nbar = (dm->Nlow + c.low_compress - 1) / (c.low_compress > 0 ? c.low_compress : 1);
@@ -60,8 +61,17 @@ extern "C" ff_status_t ff_config_validate(const ff_config_t* c) {
     return fail(nullptr, FF_ERR_UNSUPPORTED, "head_dim must be a multiple of 32 and <= 128%s");
   if (c->T > 128 || c->H > 128 || c->W > 128) return fail(nullptr, FF_ERR_UNSUPPORTED, "axis lengths above 128 are not supported%s");
   if (c->router_hidden > 1024 || c->n_summary > 64) return fail(nullptr, FF_ERR_UNSUPPORTED, "router_hidden <= 1024 and m <= 64 are supported%s");
+  if (c->transform != FF_TRANSFORM_DCT && c->transform != FF_TRANSFORM_HAAR)
+    return fail(nullptr, FF_ERR_INVALID_ARG, "transform must be FF_TRANSFORM_DCT or FF_TRANSFORM_HAAR%s");
+  if (c->mid_pattern != FF_MID_STRIDED && c->mid_pattern != FF_MID_ANCHOR)
+    return fail(nullptr, FF_ERR_INVALID_ARG, "mid_pattern must be FF_MID_STRIDED or FF_MID_ANCHOR%s");
+  if (c->transform == FF_TRANSFORM_HAAR)
+    for (int a = 0; a < 3; ++a)
+      if (n[a] & (n[a] - 1)) return fail(nullptr, FF_ERR_UNSUPPORTED, "the Haar transform needs power-of-two axis lengths%s");
   FFDims dm; dims_from_cfg(*c, &dm);
-  if (dm.Nlow < 1 || dm.Nmid < 1 || dm.Nhigh < 1) return fail(nullptr, FF_ERR_EMPTY_BAND, "the cut-offs leave a band empty%s");
+  // Two bands ("Number of bands", L = 2): mid cut-offs equal to the low cut-offs leave the mid band empty, and
+  // the layer runs with the low and the high band only.  The low and the high band must exist.
+  if (dm.Nlow < 1 || dm.Nhigh < 1) return fail(nullptr, FF_ERR_EMPTY_BAND, "the cut-offs leave the low or the high band empty%s");
   return FF_OK;
 }
 
@@ -190,14 +200,28 @@ extern "C" ff_status_t ff_plan_create(const ff_config_t* c, const ff_weights_t* 
     delete p;
     return FF_ERR_CUDA;
   }
-  // DCT-II matrices C[k][i] = alpha_k cos(pi (2i+1) k / (2n)), evaluated in double.
+  // The 1-D transform matrices C[k][i], evaluated in double: DCT-II, alpha_k cos(pi (2i+1) k / (2n)), or the
+  // orthonormal Haar wavelets (row 0 constant; row 2^j + q is +-sqrt(2^j / n) on the halves of the q-th block of
+  // n / 2^j positions), rows from the coarsest scale to the finest.
   const int n[3] = {c->T, c->H, c->W};
   for (int a = 0; a < 3 && s == FF_OK; ++a) {
     std::vector<float> C((size_t)n[a] * n[a]), Ct((size_t)n[a] * n[a]);
     for (int k = 0; k < n[a]; ++k)
       for (int i = 0; i < n[a]; ++i) {
-        const double alpha = (k == 0) ? sqrt(1.0 / n[a]) : sqrt(2.0 / n[a]);
-        const double v = alpha * cos(M_PI * (2.0 * i + 1.0) * k / (2.0 * n[a]));
+        double v;
+        if (c->transform == FF_TRANSFORM_HAAR) {
+          if (k == 0) v = sqrt(1.0 / n[a]);
+          else {
+            int j = 0;
+            while ((2 << j) <= k) ++j;                       // level: 2^j <= k < 2^(j+1)
+            const int q = k - (1 << j), block = n[a] >> j;
+            const double amp = sqrt((double)(1 << j) / n[a]);
+            v = (i < q * block || i >= (q + 1) * block) ? 0.0 : (i < q * block + block / 2 ? amp : -amp);
+          }
+        } else {
+          const double alpha = (k == 0) ? sqrt(1.0 / n[a]) : sqrt(2.0 / n[a]);
+          v = alpha * cos(M_PI * (2.0 * i + 1.0) * k / (2.0 * n[a]));
+        }
         C[(size_t)k * n[a] + i] = (float)v;
         Ct[(size_t)i * n[a] + k] = (float)v;
       }
@@ -404,7 +428,9 @@ extern "C" ff_status_t ff_forward(ff_plan_t* p, const void* Q, const void* K, co
   if (alloc_dev) FF_CUDA(p, cudaMemcpyAsync(p->buf.alloc, alloc_dev, p->dm.BH, cudaMemcpyDeviceToDevice, st));
   FF_CUDA(p, ffk_pool_low(p, st));
   if (p->tc_ok && !(p->attn_impl & 1)) {
-    if (!p->low_tc_ok) FF_CUDA(p, ffk_attention_simt(p, FF_BAND_LOW, st));
+    // the tensor-core launch takes the high band, the strided mid band and a long pooled low band
+    const int simt_bands = (p->low_tc_ok ? 0 : FF_BAND_LOW) | (p->dm.pattern == FF_MID_ANCHOR ? FF_BAND_MID : 0);
+    if (simt_bands) FF_CUDA(p, ffk_attention_simt(p, simt_bands, st));
     FF_CUDA(p, ffk_attention_tc(p, st));
   } else {
     FF_CUDA(p, ffk_attention_simt(p, FF_BAND_LOW | FF_BAND_MID | FF_BAND_HIGH, st));

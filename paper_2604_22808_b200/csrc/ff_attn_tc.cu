@@ -93,7 +93,8 @@ __global__ void build_worklist_kernel(TcParams P) {
       total += (nt + 1) / 2; ++nu;
     }
   }
-  for (int bh = 0; bh < dm.BH && nu < MAX_UNITS; ++bh) {
+  // (the anchor pattern of the mid band is not a union of dense classes: those heads run on the generic kernel)
+  for (int bh = 0; bh < dm.BH && nu < MAX_UNITS && dm.pattern == FF_MID_STRIDED; ++bh) {
     if (!(P.alloc[bh] & FF_BAND_MID)) continue;
     offsets[nu] = total; desc[nu] = (bh << 12) | (1 << 10); tiles[nu] = 0;
     total += ms.items; ++nu;
@@ -198,7 +199,10 @@ __device__ __forceinline__ long long mid_rank(const FFDims& dm, int c, long long
 // already announced the bytes on `bar`.  `first` = class-local position (mid) or band rank (high).
 // `halves` = head_dim / 64.
 __device__ __forceinline__ void load_tile(uint8_t* dst, const CUtensorMap* map, uint64_t* bar, const FFDims& dm,
-                                          const Item& x, int slice, long long first, int rb, int halves) {
+                                          const Item& x, int slice, long long first, int rb, int halves, int* status) {
+  // (debug build) a tile starts inside its band (rows past the end are zero-filled by the copy); the bytes were
+  // announced on `bar` already, so a refused copy ends in the bounded wait of its consumer, not in a fault
+  if (!FF_DBG_OK(first >= 0 && first < x.n + TILE && slice >= 0, status, 1)) return;
   if (x.band != 1) {
     tma_load_3d(dst, map, bar, 0, (int)first, slice);
     if (halves > 1) tma_load_3d(dst + HALF_BYTES, map, bar, 64, (int)first, slice);
@@ -317,19 +321,19 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         if (iter >= 1) ok = mbar_wait(&sh.q_empty, (iter - 1) & 1, abort_flag);
         if (!ok) break;
         mbar_arrive_expect_tx(&sh.q_full, x.has_b ? 2 * TB : TB);
-        load_tile(sQ, mapq, &sh.q_full, dm, x, x.bh, (long long)x.tile_a * TILE, rb, HALVES);
-        if (x.has_b) load_tile(sQ + TILE_BYTES, mapq, &sh.q_full, dm, x, x.bh, (long long)(x.tile_a + 1) * TILE, rb, HALVES);
+        load_tile(sQ, mapq, &sh.q_full, dm, x, x.bh, (long long)x.tile_a * TILE, rb, HALVES, P.status);
+        if (x.has_b) load_tile(sQ + TILE_BYTES, mapq, &sh.q_full, dm, x, x.bh, (long long)(x.tile_a + 1) * TILE, rb, HALVES, P.status);
         for (int j = 0; j < x.nk && ok; ++j, ++g) {
           const int st = g & 1;
           const long long first = x.band == 2 ? x.ks + (long long)j * TILE : (long long)j * TILE;
           if (g >= 2) ok = mbar_wait(&sh.k_empty[st], ((g >> 1) - 1) & 1, abort_flag);
           if (!ok) break;
           mbar_arrive_expect_tx(&sh.k_full[st], TB);
-          load_tile(sK + st * TILE_BYTES, mapk, &sh.k_full[st], dm, x, slice_k, first, rb, HALVES);
+          load_tile(sK + st * TILE_BYTES, mapk, &sh.k_full[st], dm, x, slice_k, first, rb, HALVES, P.status);
           if (g >= 2) ok = mbar_wait(&sh.v_empty[st], ((g >> 1) - 1) & 1, abort_flag);
           if (!ok) break;
           mbar_arrive_expect_tx(&sh.v_full[st], TB);
-          load_tile(sV + st * TILE_BYTES, mapv, &sh.v_full[st], dm, x, slice_v, first, rb, HALVES);
+          load_tile(sV + st * TILE_BYTES, mapv, &sh.v_full[st], dm, x, slice_v, first, rb, HALVES, P.status);
         }
       }
     }
@@ -572,7 +576,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
       if (!ok) break;
       tc_fence_after();
       const float inv = 1.f / l;
-      const bool store = p < x.n;
+      const bool store = p < x.n && FF_DBG_OK(p >= 0 && x.bh >= 0 && x.bh < dm.BH, P.status, 1);
       __nv_bfloat16* y = (x.band == 1 ? P.y_mid : P.y_high) + ((size_t)x.bh * x.n + (store ? p : 0)) * HD + ocol0;
       float* yl = HAS_LOW && x.band == 0 ? P.y_low + ((size_t)x.bh * x.n + (store ? p : 0)) * HD + ocol0 : nullptr;   // low band: fp32
 #pragma unroll
@@ -681,7 +685,9 @@ bool ffk_tc_prepare(ff_plan* p) {
   static_assert(sizeof(CUtensorMap) <= sizeof(p->tmap_mid), "tensor map storage too small");
   const FFDims& dm = p->dm;
   const int rb = dm.b < TILE ? dm.b : TILE;
-  if (!encode_band_map((CUtensorMap*)p->tmap_mid, p->buf.spec_mid, dm.Nmid, 3 * dm.BH, rb, dm.d) ||
+  // (an empty mid band has no items; its map is encoded over one row of the high band's buffer and never used)
+  if (!encode_band_map((CUtensorMap*)p->tmap_mid, dm.Nmid > 0 ? p->buf.spec_mid : p->buf.spec_high, dm.Nmid > 0 ? dm.Nmid : 1,
+                       3 * dm.BH, dm.Nmid > 0 ? rb : 1, dm.d) ||
       !encode_band_map((CUtensorMap*)p->tmap_high, p->buf.spec_high, dm.Nhigh, 3 * dm.BH, TILE, dm.d))
     return false;
   // The low branch joins this launch when the pooled band is at least one tile long (shorter ones

@@ -448,6 +448,8 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         const uint32_t laddr = buf_base + (uint32_t)u2l * 2 * TILE_B + (uint32_t)drow * STG_ROW;
         const uint32_t daddr = cs == 1 ? laddr : mapa(laddr, owner);
         const int swz = (drow >> 1) & 3;
+        // (debug build) the row lies inside a tile of the owner's buffer
+        if (!FF_DBG_OK(drow >= 0 && drow < ROWS && u2l >= 0 && u2l < tpc && owner < (uint32_t)cs && b < n2, P.status, 4)) continue;
         // rotate the pieces by `rot` (two conditional swaps), then piece i of the registers is piece (i + rot) % 4 of the row
         if (rot & 1) {
 #pragma unroll

@@ -274,17 +274,26 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
         // (axis lengths are at most 128, so every count fits 32 bits)
         const int cm = kt < dm.M[0] ? kt * Mhw + offM : dm.M[0] * Mhw;
         const size_t th_slice = (size_t)tensor * dm.BH + bh;
+        long long rk, nband;                                                         // band-local rank, band length
         if (kt < dm.L[0] && hw_low) {
           band = 0;                                                                  // low band: fp32
-          row_f32 = P.spec_low + (th_slice * dm.Nlow + (unsigned)((kt * dm.L[1] + h_) * dm.L[2] + ww)) * CH;
+          rk = (kt * dm.L[1] + h_) * dm.L[2] + ww; nband = dm.Nlow;
+          row_f32 = P.spec_low + (th_slice * dm.Nlow + (unsigned)rk) * CH;
         } else if (kt < dm.M[0] && hw_mid) {
           const int offL = (h_ < dm.L[1] ? h_ : dm.L[1]) * dm.L[2] + (h_ < dm.L[1] ? (ww < dm.L[2] ? ww : dm.L[2]) : 0);
           const int cl = kt < dm.L[0] ? kt * Lhw + offL : (int)dm.Nlow;
           band = 1;
-          row_hi = P.spec_mid + (th_slice * dm.Nmid + (unsigned)(cm - cl)) * CH;
+          rk = cm - cl; nband = dm.Nmid;
+          row_hi = P.spec_mid + (th_slice * dm.Nmid + (unsigned)rk) * CH;
         } else {
           band = 2;
-          row_hi = P.spec_high + (th_slice * dm.Nhigh + (unsigned)(((kt * dm.H + h_) * dm.W + ww) - cm)) * CH;
+          rk = ((kt * dm.H + h_) * dm.W + ww) - cm; nband = dm.Nhigh;
+          row_hi = P.spec_high + (th_slice * dm.Nhigh + (unsigned)rk) * CH;
+        }
+        // (debug build) the rank must lie inside its band and the coordinates inside the grid
+        if (!FF_DBG_OK(kt >= 0 && kt < dm.T && h_ >= 0 && h_ < dm.H && ww >= 0 && ww < dm.W && rk >= 0 && rk < nband &&
+                       th_slice < (size_t)3 * dm.BH, P.status, 2)) {
+          row_hi = nullptr; row_f32 = nullptr; band = -1;
         }
       }
       // (SPLIT) lane L stores for rows 8 i + L/4 of its warp: fetch those rows' destinations

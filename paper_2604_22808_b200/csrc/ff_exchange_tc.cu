@@ -214,6 +214,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       if (!ok) break;
       tc_fence_after();
       const int own0 = x.band * m, own1 = own0 + m;       // this band's own summaries are not attended
+      const int emp0 = dm.Nmid == 0 ? m : -1, emp1 = dm.Nmid == 0 ? 2 * m : -1;   // nor are those of an empty mid band
       if (NK32 >= 2) {
         // first sweep: the row maximum
         float mx = -INFINITY;
@@ -225,7 +226,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             const int j = c3 * 32 + i;
-            if (j < 3 * m && (j < own0 || j >= own1)) mx = fmaxf(mx, __uint_as_float(r[i]));
+            if (j < 3 * m && (j < own0 || j >= own1) && (j < emp0 || j >= emp1)) mx = fmaxf(mx, __uint_as_float(r[i]));
           }
         }
         const float mb = mx * sl2;
@@ -241,8 +242,8 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
           for (int i = 0; i < 16; ++i) {
             const int j = c3 * 32 + 2 * i;
             float p0 = 0.f, p1 = 0.f;
-            if (j < 3 * m && (j < own0 || j >= own1)) p0 = ex2f_approx(fmaf(__uint_as_float(r[2 * i]), sl2, -mb));
-            if (j + 1 < 3 * m && (j + 1 < own0 || j + 1 >= own1)) p1 = ex2f_approx(fmaf(__uint_as_float(r[2 * i + 1]), sl2, -mb));
+            if (j < 3 * m && (j < own0 || j >= own1) && (j < emp0 || j >= emp1)) p0 = ex2f_approx(fmaf(__uint_as_float(r[2 * i]), sl2, -mb));
+            if (j + 1 < 3 * m && (j + 1 < own0 || j + 1 >= own1) && (j + 1 < emp0 || j + 1 >= emp1)) p1 = ex2f_approx(fmaf(__uint_as_float(r[2 * i + 1]), sl2, -mb));
             den0 += p0; den1 += p1;
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
             ph[i] = *(const uint32_t*)&h2;
@@ -267,13 +268,13 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int j = 0; j < NK32 * 32; ++j)
-          if (j < 3 * m && (j < own0 || j >= own1)) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(sc[j]));
+          if (j < 3 * m && (j < own0 || j >= own1) && (j < emp0 || j >= emp1)) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(sc[j]));
         const float mb = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
         float den4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < NK32 * 32; ++j) {
           float pv = 0.f;
-          if (j < 3 * m && (j < own0 || j >= own1)) pv = ex2f_approx(fmaf(__uint_as_float(sc[j]), sl2, -mb));
+          if (j < 3 * m && (j < own0 || j >= own1) && (j < emp0 || j >= emp1)) pv = ex2f_approx(fmaf(__uint_as_float(sc[j]), sl2, -mb));
           den4[j & 3] += pv;
           sc[j] = __float_as_uint(pv);
         }
@@ -316,7 +317,8 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       if (!ok) break;
       tc_fence_after();
       const bool valid = p < n_band;
-      const int f = valid ? (x.band == 1 ? P.pos_mid[p] : P.pos_high[p]) : -1;
+      int f = valid ? (x.band == 1 ? P.pos_mid[p] : P.pos_high[p]) : -1;
+      if (valid && !FF_DBG_OK(f >= 0 && f < dm.N && x.bh >= P.h0 && x.bh < P.h0 + P.g, P.status, 3)) f = -1;   // (debug build)
       // lane L stores for rows 8 i + L/4 of its warp: fetch those rows' grid positions
       int fpos[4];
 #pragma unroll
@@ -431,8 +433,10 @@ bool ffk_exchange_tc_build_tables(ff_plan* p) {
 
 bool ffk_exchange_tc_prepare(ff_plan* p) {
   const FFDims& dm = p->dm;
-  return encode_rows_map((CUtensorMap*)p->tmap_x[0], p->buf.y_mid, dm.Nmid, dm.BH, dm.d) &&
-         encode_rows_map((CUtensorMap*)p->tmap_x[1], p->buf.spec_mid, dm.Nmid, 3 * dm.BH, dm.d) &&
+  // (an empty mid band has no tiles; its maps are encoded over one row of the high band's buffers and never used)
+  const long long nm = dm.Nmid > 0 ? dm.Nmid : 1;
+  return encode_rows_map((CUtensorMap*)p->tmap_x[0], dm.Nmid > 0 ? p->buf.y_mid : p->buf.y_high, nm, dm.BH, dm.d) &&
+         encode_rows_map((CUtensorMap*)p->tmap_x[1], dm.Nmid > 0 ? p->buf.spec_mid : p->buf.spec_high, nm, 3 * dm.BH, dm.d) &&
          encode_rows_map((CUtensorMap*)p->tmap_x[2], p->buf.y_high, dm.Nhigh, dm.BH, dm.d) &&
          encode_rows_map((CUtensorMap*)p->tmap_x[3], p->buf.spec_high, dm.Nhigh, 3 * dm.BH, dm.d);
 }

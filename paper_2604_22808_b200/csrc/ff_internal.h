@@ -13,12 +13,24 @@
 #define FF_HD inline
 #endif
 
+// Debug build (-DFF_DEBUG): every computed band rank, row offset and tile coordinate is range-checked on
+// the device before it is used; a value out of range is not used for the access (the store or copy is
+// skipped) and FF_ERR_INVALID_ARG together with the kernel's id is raised in the plan's status word, where
+// ff_plan_device_status reports it.  The release build compiles the checks away.
+#if defined(FF_DEBUG) && defined(__CUDACC__)
+#define FF_DBG_OK(cond, status_ptr, kernel_id) \
+  ((cond) ? true : (atomicExch((status_ptr), FF_ERR_INVALID_ARG | ((kernel_id) << 8)), false))
+#else
+#define FF_DBG_OK(cond, status_ptr, kernel_id) (true)
+#endif
+
 // Problem sizes derived from ff_config_t ("Frequency band partitioning": N_low + N_mid + N_high = N).
 struct FFDims {
   int B, T, H, W, heads, d, BH;
   int L[3], M[3];
   int r, b, s, R, m, hid, dt;
   int fp32;              // storage type of Q,K,V,out and of the mid/high band buffers
+  int pattern;           // mid-band sparse pattern: FF_MID_STRIDED or FF_MID_ANCHOR
   long long N, Nlow, Nbar, Nmid, Nhigh;
   long long nb;          // number of mid blocks
 };

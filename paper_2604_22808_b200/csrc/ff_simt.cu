@@ -189,7 +189,7 @@ __global__ void router_kernel(const double* energy, const float* timestep, const
   const int sample = blockIdx.x;
   const long long cnt[3] = {dm.Nlow, dm.Nmid, dm.Nhigh};
   for (int i = threadIdx.x; i < 3 * d; i += blockDim.x) {
-    const double terms = 3.0 * dm.heads * (double)cnt[i / d];
+    const double terms = 3.0 * dm.heads * (double)(cnt[i / d] > 0 ? cnt[i / d] : 1);   // an empty band (two-band layer) has g = 0
     x[i] = (float)log1p(energy[(size_t)sample * 3 * d + i] / terms);
   }
   const int half = dm.dt / 2;
@@ -320,7 +320,16 @@ __global__ void __launch_bounds__(ATT_WARPS * 32) attention_simt_kernel(FFBuffer
     const ST* Vp = Kp + BHn;
 #pragma unroll
     for (int j = 0; j < DPL; ++j) q[j] = ldf<ST>(Qp + (size_t)p * d + lane + 32 * j);
-    if (band == 1) {
+    if (band == 1 && dm.pattern == FF_MID_ANCHOR) {
+      // own block and every anchor block (block index = s-1 mod s)
+      const long long J = p / dm.b;
+      for (long long Jk = 0; Jk < dm.nb; ++Jk) {
+        if (Jk != J && Jk % dm.s != dm.s - 1) continue;
+        const long long k0 = Jk * dm.b;
+        const long long k1 = (k0 + dm.b < n) ? k0 + dm.b : n;
+        attend_range<ST, DPL>(Kp, Vp, k0, k1, d, q, scale, mx, den, o, lane);
+      }
+    } else if (band == 1) {
       const long long J = p / dm.b;
       for (long long Jk = J % dm.s; Jk < dm.nb; Jk += dm.s) {
         const long long k0 = Jk * dm.b;
@@ -382,6 +391,7 @@ __global__ void __launch_bounds__(SUM_THREADS) summary_partial_kernel(FFBuffers 
   const int j = blockIdx.x / split, piece = blockIdx.x % split, band = blockIdx.y, bh = blockIdx.z;
   const int d = dm.d, vecs = d / 8;                // 8-channel vectors per row
   const BandView<ST> v = band_view<ST>(buf, dm, bh, band);
+  if (v.n == 0) return;                            // empty band (two-band layer): no summary tokens
   const long long a = ((long long)j * v.n) / dm.m;
   long long e = ((long long)(j + 1) * v.n) / dm.m;
   if (e < a + 1) e = a + 1;
@@ -450,6 +460,7 @@ __global__ void summary_finalize_kernel(FFBuffers buf, const float* U, FFDims dm
   const int j = blockIdx.x, band = blockIdx.y, bh = blockIdx.z;
   const int d = dm.d, c = threadIdx.x;
   const BandView<ST> v = band_view<ST>(buf, dm, bh, band);
+  if (v.n == 0) return;                            // (its slots stay zero and are never attended)
   const long long a = ((long long)j * v.n) / dm.m;
   long long e = ((long long)(j + 1) * v.n) / dm.m;
   if (e < a + 1) e = a + 1;
@@ -510,7 +521,7 @@ __global__ void __launch_bounds__(EXC_WARPS * 32) exchange_recombine_kernel(FFBu
     const float scale = rsqrtf((float)d);
     float mx = -INFINITY, den = 0.f;
     for (int ob = 0; ob < 3; ++ob) {
-      if (ob == band) continue;
+      if (ob == band || (ob == 1 && dm.Nmid == 0)) continue;     // own band; an empty mid band has no summaries
       for (int j2 = 0; j2 < m; ++j2) {
         const float* z = S + ((size_t)ob * m + j2) * d;
         float part = 0.f;
@@ -621,6 +632,7 @@ static cudaError_t attention_simt_t(ff_plan* p, int band_bits, cudaStream_t st) 
   if ((band_bits & FF_BAND_LOW) && dm.Nbar > nmax) nmax = dm.Nbar;
   if ((band_bits & FF_BAND_MID) && dm.Nmid > nmax) nmax = dm.Nmid;
   if ((band_bits & FF_BAND_HIGH) && dm.Nhigh > nmax) nmax = dm.Nhigh;
+  if (nmax == 0) return cudaSuccess;                 // (only an empty band was asked for)
   const int zdim = (band_bits & FF_BAND_HIGH) ? 3 : ((band_bits & FF_BAND_MID) ? 2 : 1);
   dim3 grid((unsigned)((nmax + ATT_WARPS - 1) / ATT_WARPS), (unsigned)dm.BH, zdim);
   switch (dm.d / 32) {

@@ -14,8 +14,13 @@ from paper_2604_22808_b200 import inputs as I
 #   |o| >= 4:  |g - o| <= max(2e-2, 1e-2 |o|)  and  |g - bf16(o)| <= one bf16 step of o: g is the
 #              oracle value rounded to the storage type, or its neighbour (the step is 0.031 from
 #              4 on and 0.0625 from 8 on, so no bf16 result can promise 2e-2 there)
+# Both bounds widen to 2^-15 max|o| of the compared tensor where that is larger: a stage whose values
+# reach 3e4 (the exchanged low band of the workload with the smooth component, identity summaries) and
+# whose intermediates carry 16 bits (bf16 hi + lo) cannot resolve 2e-2 on the small outputs of the same
+# transform line; for every tensor of magnitude up to 650 the term is below 2e-2 and changes nothing.
 # fp32 workload: |g - o| <= 5e-5 max(1, |o|).
 BF16_ATOL, BF16_RTOL = 2e-2, 1e-2
+BF16_SCALE_RTOL = 2.0 ** -15
 FP32_TOL = 5e-5
 BINS = ((0.0, 2.0), (2.0, 4.0), (4.0, 8.0), (8.0, np.inf))
 
@@ -36,7 +41,8 @@ def tolerance(o: np.ndarray, dtype: str) -> np.ndarray:
     a = np.abs(o)
     if dtype == "fp32":
         return FP32_TOL * np.maximum(1.0, a)
-    return np.where(a < 4.0, BF16_ATOL, np.maximum(BF16_ATOL, BF16_RTOL * a))
+    scale_term = BF16_SCALE_RTOL * (float(a.max()) if a.size else 0.0)
+    return np.maximum(np.where(a < 4.0, BF16_ATOL, np.maximum(BF16_ATOL, BF16_RTOL * a)), scale_term)
 
 
 def parity_report(g, o) -> dict:
@@ -72,13 +78,15 @@ def assert_close(g, o, dtype: str, what: str = "", stored_bf16: bool = True):
     summary tokens), where the neighbour rule of the storage type does not apply."""
     g = np.asarray(g, np.float64); o = np.asarray(o, np.float64)
     assert g.shape == o.shape, (what, g.shape, o.shape)
+    if g.size == 0:                                  # (an empty band)
+        return 0.0
     assert np.all(np.isfinite(g)), f"{what}: non-finite values"
     err = np.abs(g - o)
     tol = tolerance(o, dtype)
     bad = err > tol
     if dtype != "fp32" and stored_bf16:
         # from 4 on: the oracle value rounded to bf16, or the neighbouring bf16 value
-        bad |= (np.abs(o) >= 4.0) & (np.abs(g - bf16_round(o)) > bf16_step(o) * (1 + 1e-9))
+        bad |= (np.abs(o) >= 4.0) & (np.abs(g - bf16_round(o)) > np.maximum(bf16_step(o) * (1 + 1e-9), BF16_SCALE_RTOL * np.abs(o).max()))
     if bad.any():
         i = np.unravel_index(np.argmax(np.where(bad, err - tol, -np.inf)), err.shape)
         raise AssertionError(f"{what}: {bad.sum()} of {bad.size} outside tolerance; worst at {i}: "
@@ -160,6 +168,7 @@ def stagewise_check(cfg, plan, Q, K, V, out_gpu, weights, U, timesteps, routed: 
     members = O.band_members(cfg.grid, cfg.low_cut, cfg.mid_cut)
     sizes = [len(x) for x in members]
     n_bar = -(-sizes[0] // cfg.r)
+    kind = getattr(cfg, "transform", "dct")
     alloc = plan.tap(B.TAP_ALLOC).cpu().numpy().reshape(cfg.batch, cfg.heads)
     spec_taps = [plan.tap(w) for w in (B.TAP_SPEC_LOW, B.TAP_SPEC_MID, B.TAP_SPEC_HIGH)]
     y_taps = [plan.tap(w) for w in (B.TAP_Y_LOW, B.TAP_Y_MID, B.TAP_Y_HIGH)]
@@ -183,7 +192,7 @@ def stagewise_check(cfg, plan, Q, K, V, out_gpu, weights, U, timesteps, routed: 
             mask = int(alloc[bi, h])
             bands = []
             for t in range(3):
-                ob = O.split_bands(O.forward_transform(np.asarray(head_source(t, bi, h), np.float64)), members)
+                ob = O.split_bands(O.forward_transform(np.asarray(head_source(t, bi, h), np.float64), kind), members)
                 esum += O.band_energy_sums(ob)
                 bands.append(ob)
                 for l in range(3):
@@ -212,7 +221,8 @@ def stagewise_check(cfg, plan, Q, K, V, out_gpu, weights, U, timesteps, routed: 
                     rows = np.arange(sizes[l]) if full else I.sample_rows(cfg, 77000 + 10 * bh + l, sizes[l], n_rows)
                     op = O.mid_operator if l == 1 else O.high_operator
                     args = (cfg.b, cfg.s) if l == 1 else (cfg.R,)
-                    ref, _ = op(Qo[l], Ko[l], Vo[l], *args, rows=rows)
+                    kw = {"pattern": getattr(cfg, "mid_pattern", "strided")} if l == 1 else {}
+                    ref, _ = op(Qo[l], Ko[l], Vo[l], *args, rows=rows, **kw)
                 errs["attention"] = max(errs["attention"], assert_close(Yg[l][rows], ref, cfg.dtype, f"Y band {l} head {bh}",
                                                                         stored_bf16=l > 0))
             # summaries of the working outputs the device holds
@@ -233,7 +243,7 @@ def stagewise_check(cfg, plan, Q, K, V, out_gpu, weights, U, timesteps, routed: 
                     if l == 0 and yh.shape[0] != sizes[0]:
                         yh = O.decompress_low(yh, cfg.r, sizes[0])
                     spec[members[l]] = yh
-                ref = O.inverse_transform(spec.reshape(cfg.T, cfg.H, cfg.W, d))
+                ref = O.inverse_transform(spec.reshape(cfg.T, cfg.H, cfg.W, d), kind)
                 errs["output"] = max(errs["output"], assert_close(out_of(bi, h), ref, cfg.dtype, f"out head {bh}"))
         if routed:
             g = O.pooled_statistics(esum, [3.0 * cfg.heads * n for n in sizes])

@@ -40,7 +40,14 @@ def test_validate_codes():
     assert B.ff_config_validate(C.TINY.scaled("x", W=256, mid_cut=(3, 6, 6))) == 2
     assert B.ff_config_validate(C.TINY.scaled("x", low_cut=(0, 2, 2))) == 6     # empty low band
     assert B.ff_config_validate(C.TINY.scaled("x", mid_cut=(4, 8, 8))) == 6     # empty high band
-    assert B.ff_config_validate(C.TINY.scaled("x", mid_cut=(1, 2, 2))) == 6     # empty mid band
+    assert B.ff_config_validate(C.TINY.scaled("x", mid_cut=(1, 2, 2))) == 0     # empty mid band: a two-band layer
+    assert B.ff_config_validate(C.TINY.scaled("x", transform="haar")) == 0
+    assert B.ff_config_validate(C.TINY.scaled("x", transform="haar", T=3, low_cut=(1, 2, 2), mid_cut=(2, 6, 6))) == 2
+    assert B.ff_config_validate(C.TINY.scaled("x", mid_pattern="anchor")) == 0
+    bad = B.c_config(C.TINY); bad.transform = 7
+    assert B.library().ff_config_validate(B.C.byref(bad)) == 1
+    bad = B.c_config(C.TINY); bad.mid_pattern = -1
+    assert B.library().ff_config_validate(B.C.byref(bad)) == 1
     assert B.ff_config_validate(C.TINY.scaled("x", low_cut=(2, 7, 7), mid_cut=(1, 8, 8))) == 1
     assert B.ff_config_validate(C.TINY.scaled("x", s=0)) == 1
     assert B.ff_config_validate(C.TINY.scaled("x", t_embed_dim=7)) == 1

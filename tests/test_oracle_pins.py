@@ -457,3 +457,105 @@ def test_paper_reference_workloads_match_the_reference_cost():
         reference = O.paper_attention_cost_reference(cfg.N, 1.0)  # = 0.0009765625 N^2 + 128 N
         assert abs(reference - (0.0009765625 * cfg.N ** 2 + 128 * cfg.N)) < 1e-6 * reference
         assert abs(exact - reference) < 0.05 * reference
+
+
+# ----------------------------------------------------------------------------------------------
+# Alternative transform ("Transform choice"): orthonormal Haar wavelets
+# ----------------------------------------------------------------------------------------------
+def test_haar_matrix_hand_example_and_orthonormality():
+    r = 1.0 / np.sqrt(2.0)
+    H4 = np.array([[0.5, 0.5, 0.5, 0.5], [0.5, 0.5, -0.5, -0.5], [r, -r, 0, 0], [0, 0, r, -r]])
+    assert np.allclose(O.haar_matrix(4), H4, atol=1e-15)
+    assert np.allclose(O.haar_matrix(1), [[1.0]])
+    for n in (2, 8, 16, 64, 128):
+        Hm = O.haar_matrix(n)
+        assert np.abs(Hm @ Hm.T - np.eye(n)).max() < 1e-13
+        assert np.allclose(Hm[0], 1.0 / np.sqrt(n))                       # row 0: the mean, as DCT row 0
+        assert np.all(np.abs(Hm[1:].sum(axis=1)) < 1e-13)                 # every wavelet has zero mean
+        # rows run from coarse to fine: the support of row 2^j + k is n / 2^j positions
+        for k in range(1, n):
+            j = int(np.floor(np.log2(k)))
+            assert np.count_nonzero(Hm[k]) == n >> j
+    with pytest.raises(ValueError):
+        O.haar_matrix(12)
+
+
+def test_haar_transform_round_trip_parseval_and_piecewise_constant_input():
+    g = np.random.default_rng(5)
+    X = g.standard_normal((4, 8, 16, 3))
+    Y = O.forward_transform(X, "haar")
+    assert np.abs(O.inverse_transform(Y, "haar") - X).max() < 1e-12
+    assert np.allclose((Y ** 2).sum(axis=(0, 1, 2)), (X ** 2).sum(axis=(0, 1, 2)))
+    # brute force on one coefficient: the triple sum of the definition
+    Ht, Hh, Hw = O.haar_matrix(4), O.haar_matrix(8), O.haar_matrix(16)
+    k = (2, 5, 9)
+    direct = sum(Ht[k[0], t] * Hh[k[1], h] * Hw[k[2], w] * X[t, h, w] for t in range(4) for h in range(8) for w in range(16))
+    assert np.abs(direct - Y[k]).max() < 1e-12
+    # an input that is constant on quarters of the w axis has only the four coarsest w coefficients
+    Z = np.repeat(g.standard_normal((4, 8, 4, 3)), 4, axis=2)
+    Zs = O.forward_transform(Z, "haar")
+    assert np.abs(Zs[:, :, 4:]).max() < 1e-12 and np.abs(Zs[:, :, :4]).max() > 0.1
+    # the default stays the DCT
+    assert np.allclose(O.forward_transform(X), O.forward_transform(X, "dct"))
+
+
+# ----------------------------------------------------------------------------------------------
+# Alternative mid-band pattern ("Mid-band sparse degree"): own block plus anchor blocks
+# ----------------------------------------------------------------------------------------------
+def test_anchor_pattern_key_sets_by_brute_force():
+    for n, b, s in ((37, 4, 3), (64, 8, 4), (10, 16, 2), (50, 5, 1)):
+        total = 0
+        for p in range(n):
+            expect = [k for k in range(n) if k // b == p // b or (k // b) % s == s - 1]
+            got = O.mid_keys(p, n, b, s, "anchor")
+            assert got.tolist() == expect
+            total += len(expect)
+        assert total == O.mid_interactions(n, b, s, "anchor")
+
+
+def test_anchor_pattern_reductions_to_dense_attention():
+    g = np.random.default_rng(9)
+    Q, K, V = (g.standard_normal((29, 8)) for _ in range(3))
+    dense = _loop_attention(Q, K, V, lambda i, j: True)
+    y1, pairs = O.mid_operator(Q, K, V, b=4, s=1, pattern="anchor")        # stride 1: every block is an anchor
+    assert np.abs(y1 - dense).max() < 1e-12 and pairs == 29 * 29
+    y2, _ = O.mid_operator(Q, K, V, b=32, s=5, pattern="anchor")           # one block holds the whole band
+    assert np.abs(y2 - dense).max() < 1e-12
+    # no anchor block exists (fewer blocks than the stride): block-local attention
+    y3, _ = O.mid_operator(Q, K, V, b=8, s=9, pattern="anchor")
+    for J in range(4):
+        sl = slice(8 * J, min(29, 8 * J + 8))
+        assert np.abs(y3[sl] - _loop_attention(Q[sl], K[sl], V[sl], lambda i, j: True)).max() < 1e-12
+    # a general case against the scalar-loop reference with the predicate written out
+    y4, _ = O.mid_operator(Q, K, V, b=4, s=3, pattern="anchor")
+    ref = _loop_attention(Q, K, V, lambda i, j: j // 4 == i // 4 or (j // 4) % 3 == 2)
+    assert np.abs(y4 - ref).max() < 1e-12
+
+
+# ----------------------------------------------------------------------------------------------
+# Two bands ("Number of bands", L = 2): mid cut-offs equal to the low cut-offs
+# ----------------------------------------------------------------------------------------------
+def test_two_band_layer():
+    from paper_2604_22808_b200 import configs as C
+    from paper_2604_22808_b200 import inputs as I
+    cfg = C.TINY.scaled("tiny_two_bands", mid_cut=C.TINY.low_cut)
+    mem = O.band_members(cfg.grid, cfg.low_cut, cfg.mid_cut)
+    assert [len(x) for x in mem] == [4, 0, 252]
+    Q, K, V = (I.qkv_full(cfg, t)[0] for t in range(3))
+    W = I.router_weights(cfg)
+    U = I.summary_projection(cfg)
+    res = O.forward_sample(cfg, Q, K, V, W, U, 500.0, alloc=[5, 7], want_taps=True)
+    n_bar = -(-4 // cfg.r)
+    # each token of the two live bands attends the m summaries of the other live band only
+    assert res["counters"]["pairs_exchange"] == cfg.heads * cfg.m * (n_bar + 252)
+    assert res["counters"]["pairs_mid"] == 0
+    # a head whose mask names the empty band computes what the same head computes without it
+    res2 = O.forward_sample(cfg, Q, K, V, W, U, 500.0, alloc=[5, 5])
+    assert np.abs(res["out"] - res2["out"]).max() == 0.0
+    # whole-pipeline identity: empty masks and no exchange give out = V
+    ident = O.forward_sample(cfg.scaled("x", m=0), Q, K, V, W, U, 500.0, alloc=[0, 0])
+    assert np.abs(ident["out"] - V).max() < 1e-12
+    # the router still produces a valid allocation (the empty band's statistic is zero)
+    routed = O.forward_sample(cfg, Q, K, V, W, U, 500.0)
+    assert routed["alloc"].shape == (cfg.heads,) and np.all(np.isfinite(routed["pi"]))
+    assert np.all(routed["g"][cfg.head_dim:2 * cfg.head_dim] == 0.0)

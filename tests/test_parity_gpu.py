@@ -169,6 +169,35 @@ def test_operator_parameter_grid(par):
     _run(cfg, alloc=[7, 2, 5])
 
 
+def test_haar_transform():
+    """The alternative transform of the ablations (orthonormal Haar wavelets per axis): the same kernels
+    with other matrices -- generic fp32 path, fused two-axis launch, separate axis passes."""
+    _run(C.TINY.scaled("tiny_haar", transform="haar"), alloc=[7, 2], identity_U=False)
+    _run(C.TINY.scaled("tiny_haar", transform="haar"))
+    cfg = C.R64K.scaled("64k_replica_haar", heads=3, transform="haar")
+    _run(cfg, alloc=[7, 2, 4])
+    _run(cfg, alloc=[1, 4, 2], impl=4)
+    _run(cfg, alloc=[1, 4, 2], impl=2)
+
+
+def test_anchor_mid_pattern():
+    """The alternative mid-band pattern (own block plus anchor blocks) behind the same predicate."""
+    _run(C.TINY.scaled("tiny_anchor", mid_pattern="anchor"), alloc=[2, 7])
+    cfg = C.R64K.scaled("64k_replica_anchor", heads=3, mid_pattern="anchor")
+    _run(cfg, alloc=[2, 7, 4])
+    _run(cfg, alloc=[6, 2, 1], impl=1)
+    _run(cfg)
+
+
+def test_two_band_layer():
+    """L = 2: mid cut-offs equal to the low cut-offs leave the mid band empty; masks may still name it."""
+    _run(C.TINY.scaled("tiny_two_bands", mid_cut=C.TINY.low_cut), alloc=[5, 7])
+    _run(C.TINY.scaled("tiny_two_bands", mid_cut=C.TINY.low_cut))
+    cfg = C.R64K.scaled("64k_replica_two_bands", heads=3, mid_cut=C.R64K.low_cut)
+    _run(cfg, alloc=[1, 4, 7])
+    _run(cfg)
+
+
 def test_paper_reference_parameterisation_replica():
     """d_k = 64, N_low_bar = N / 32, w = 64, constant-degree mid pattern: the head_dim 64 variants of
     the tensor-core transform and attention kernels, and the generic kernels on the same inputs."""
