@@ -178,6 +178,21 @@ ff_status_t ff_forward_host(ff_plan_t *plan, const void *Q_host, const void *K_h
                             void *out_host, void *cuda_stream);
 ff_status_t ff_workspace_bytes_host(const ff_config_t *cfg, size_t *bytes);
 
+/* The layer with its projections ("Setup and notation": linear projections of the layer input produce
+ * Q_h, K_h, V_h; "Reconstruction": the head outputs are concatenated and projected):
+ *     [Q | K | V] = X [W_q | W_k | W_v],   A = ff_forward(Q, K, V),   out = concat_h(A_h) W_o
+ *   X      device, bf16, [batch][T*H*W][D], token-major, D = heads * head_dim
+ *   Wqkv   device, bf16, [3][D][D]: W_q, W_k, W_v with y = x W (row k of W multiplies input channel k;
+ *          output column h * head_dim + c is channel c of head h)
+ *   Wo     device, bf16, [D][D], same convention (input row h * head_dim + c = channel c of head h)
+ *   out    device, bf16, [batch][T*H*W][D]
+ * Q, K, V and the attention output live in the workspace's staging area (size the workspace with
+ * ff_workspace_bytes_host); Q, K, V are rounded to bf16, the storage type of the path.  bf16 plans with
+ * head_dim 64 or 128, T*H*W a multiple of 128 and D a multiple of 256; otherwise FF_ERR_UNSUPPORTED.
+ * alloc_dev / timestep as for ff_forward.  Asynchronous on the stream. */
+ff_status_t ff_forward_projected(ff_plan_t *plan, const void *X, const void *Wqkv, const void *Wo,
+                                 const uint8_t *alloc_dev, const float *timestep, void *out, void *cuda_stream);
+
 /* Synchronises the stream and returns the device status word (FF_OK or FF_ERR_TIMEOUT), then
  * clears it. */
 ff_status_t ff_plan_device_status(ff_plan_t *plan, void *cuda_stream);

@@ -402,6 +402,55 @@ def forward_sample(cfg, Q, K, V, weights, U, timestep: float, alloc=None, want_t
 
 
 # ----------------------------------------------------------------------------------------------
+# The layer with its projections ("Setup and notation", "Reconstruction")
+# ----------------------------------------------------------------------------------------------
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """Nearest bf16 (ties to even) of float64 values, as float64: the storage type of Q, K, V."""
+    x32 = np.ascontiguousarray(x, dtype=np.float32)
+    u = x32.view(np.uint32)
+    u = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return u.view(np.float32).astype(np.float64)
+
+
+def project_qkv(X: np.ndarray, Wqkv: np.ndarray, heads: int, grid, bf16_storage: bool = True):
+    """"Linear projections produce Q_h, K_h, V_h": X[N, D] (token-major, D = heads d) times
+    W_q, W_k, W_v [D, D] (y = x W); output column h d + c is channel c of head h.  Returns Q, K, V as
+    [heads, T, H, W, d].  With bf16_storage the results are rounded to bf16, the type in which the
+    attention path receives them (reading: the benchmark fixes bf16 Q/K/V)."""
+    X = np.asarray(X, np.float64)
+    N, D = X.shape
+    d = D // heads
+    T, H, W = grid
+    out = []
+    for l in range(3):
+        Y = X @ np.asarray(Wqkv[l], np.float64)                       # [N, D]
+        if bf16_storage:
+            Y = round_bf16(Y)
+        out.append(Y.reshape(N, heads, d).transpose(1, 0, 2).reshape(heads, T, H, W, d))
+    return out
+
+
+def project_out(A: np.ndarray, Wo: np.ndarray) -> np.ndarray:
+    """"Head outputs are concatenated and projected": A[heads, T, H, W, d] -> [N, D] (column h d + c
+    = channel c of head h) times W_o [D, D]."""
+    heads, T, H, W, d = A.shape
+    cat = np.asarray(A, np.float64).reshape(heads, T * H * W, d).transpose(1, 0, 2).reshape(T * H * W, heads * d)
+    return cat @ np.asarray(Wo, np.float64)
+
+
+def forward_projected_sample(cfg, X, Wqkv, Wo, weights, U, timestep: float, alloc=None, bf16_storage: bool = True):
+    """The attention layer of one sample from its input X[N, D]: projections, forward_sample, output
+    projection.  The attention output is rounded to bf16 before the output projection when the path
+    stores it in bf16."""
+    Q, K, V = project_qkv(X, Wqkv, cfg.heads, (cfg.T, cfg.H, cfg.W), bf16_storage)
+    res = forward_sample(cfg, Q, K, V, weights, U, timestep, alloc=alloc)
+    A = round_bf16(res["out"]) if bf16_storage else res["out"]
+    res["attention_out"] = res["out"]
+    res["out"] = project_out(A, Wo)
+    return res
+
+
+# ----------------------------------------------------------------------------------------------
 # Cost model ("Complexity Analysis")
 # ----------------------------------------------------------------------------------------------
 def paper_interactions(n_low_bar: float, n_mid: float, k_mid: float, n_high: float, w: float) -> float:

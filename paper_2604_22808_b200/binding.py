@@ -29,7 +29,7 @@ FF_BAND_LOW, FF_BAND_MID, FF_BAND_HIGH = 1, 2, 4
 
 EXPORTS = ("ff_config_validate", "ff_band_sizes", "ff_band_rank", "ff_workspace_bytes", "ff_workspace_bytes_host",
            "ff_plan_create", "ff_plan_workspace_bytes", "ff_band_info", "ff_plan_set_workspace", "ff_destroy", "ff_last_error",
-           "ff_route", "ff_forward", "ff_forward_host", "ff_plan_device_status", "ff_plan_last_launches",
+           "ff_route", "ff_forward", "ff_forward_host", "ff_forward_projected", "ff_plan_device_status", "ff_plan_last_launches",
            "ff_get_tap", "ff_plan_set_attention_impl", "ff_plan_set_profiling", "ff_plan_stage_times", "ff_high_attention_noalloc",
            "ff_plan_selftest_bounded_wait")
 STAGES = ("transform", "router", "attention", "summary", "inverse")
@@ -74,6 +74,7 @@ def library() -> C.CDLL:
         lib.ff_route.argtypes = [C.c_void_p] + [C.c_void_p] * 3 + [C.c_void_p] * 4 + [C.c_void_p]
         lib.ff_forward.argtypes = [C.c_void_p] + [C.c_void_p] * 3 + [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.ff_forward_host.argtypes = [C.c_void_p] + [C.c_void_p] * 3 + [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.ff_forward_projected.argtypes = [C.c_void_p] + [C.c_void_p] * 3 + [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.ff_plan_device_status.argtypes = [C.c_void_p, C.c_void_p]
         lib.ff_plan_last_launches.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
         lib.ff_get_tap.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
@@ -236,6 +237,22 @@ class Plan:
                                          out_h.data_ptr(), self._stream()), self.handle)
         return out_h
 
+    def forward_projected(self, X, Wqkv, Wo, out, alloc=None, timesteps: Optional[Sequence[float]] = None):
+        """X, out: bf16 CUDA tensors [batch][T*H*W][heads*head_dim]; Wqkv [3][D][D], Wo [D][D] (y = x W).
+        The plan must have been created with host_staging=True (Q, K, V and the attention output live there)."""
+        torch = self._torch
+        cfg = self.cfg
+        D = cfg.heads * cfg.head_dim
+        for t, shape in ((X, (cfg.batch, cfg.N, D)), (out, (cfg.batch, cfg.N, D)), (Wqkv, (3, D, D)), (Wo, (D, D))):
+            if (tuple(t.shape) != shape or t.dtype != torch.bfloat16 or not t.is_contiguous() or not t.is_cuda
+                    or t.device != self.device):
+                raise FFError(1, f"expected a contiguous bf16 tensor of shape {shape} on {self.device}")
+        ts = None if timesteps is None else np.ascontiguousarray(timesteps, dtype=np.float32)
+        _check(library().ff_forward_projected(self.handle, X.data_ptr(), Wqkv.data_ptr(), Wo.data_ptr(),
+                                              None if alloc is None else alloc.data_ptr(), _ptr(ts), out.data_ptr(),
+                                              self._stream()), self.handle)
+        return out
+
     def device_status(self) -> int:
         return library().ff_plan_device_status(self.handle, self._stream())
 
@@ -299,6 +316,10 @@ def ff_forward(plan: Plan, Q, K, V, out, alloc=None, timesteps=None):
 
 def ff_forward_host(plan: Plan, Qh, Kh, Vh, out_h, alloc_host=None, timesteps=None):
     return plan.forward_host(Qh, Kh, Vh, out_h, alloc_host, timesteps)
+
+
+def ff_forward_projected(plan: Plan, X, Wqkv, Wo, out, alloc=None, timesteps=None):
+    return plan.forward_projected(X, Wqkv, Wo, out, alloc, timesteps)
 
 
 def ff_high_attention_noalloc(q, k, v, y, radius: int, sync: bool = True):

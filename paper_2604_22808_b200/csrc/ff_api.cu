@@ -443,6 +443,26 @@ extern "C" ff_status_t ff_forward(ff_plan_t* p, const void* Q, const void* K, co
   return FF_OK;
 }
 
+extern "C" ff_status_t ff_forward_projected(ff_plan_t* p, const void* X, const void* Wqkv, const void* Wo,
+                                            const uint8_t* alloc_dev, const float* timestep, void* out, void* stream) {
+  if (!p) return fail(nullptr, FF_ERR_INVALID_ARG, "plan is NULL%s");
+  if (!X || !Wqkv || !Wo || !out) return fail(p, FF_ERR_INVALID_ARG, "X, Wqkv, Wo or out is NULL%s");
+  if ((((uintptr_t)X) | ((uintptr_t)Wqkv) | ((uintptr_t)Wo) | ((uintptr_t)out)) & 15)
+    return fail(p, FF_ERR_INVALID_ARG, "X, Wqkv, Wo and out must be 16-byte aligned%s");
+  if (!p->ws) return fail(p, FF_ERR_WORKSPACE, "ff_plan_set_workspace has not been called%s");
+  if (!p->ws_has_staging) return fail(p, FF_ERR_WORKSPACE, "workspace lacks staging space: size it with ff_workspace_bytes_host%s");
+  if (!ffk_proj_supported(p->dm))
+    return fail(p, FF_ERR_UNSUPPORTED, "projections need bf16, head_dim 64 or 128, tokens %% 128 == 0 and heads * head_dim %% 256 == 0%s");
+  if (!alloc_dev && !timestep) return fail(p, FF_ERR_NOT_ROUTED, "neither an allocation nor a timestep was given%s");
+  cudaStream_t st = (cudaStream_t)stream;
+  FF_CUDA(p, ffk_project_qkv(p, X, Wqkv, p->buf.stage_q, p->buf.stage_k, p->buf.stage_v, st));
+  ff_status_t s = ff_forward(p, p->buf.stage_q, p->buf.stage_k, p->buf.stage_v, alloc_dev, timestep, p->buf.stage_out, st);
+  if (s != FF_OK) return s;
+  FF_CUDA(p, ffk_project_out(p, p->buf.stage_out, Wo, out, st));
+  p->launches += 1;                                 // (ff_forward restarted the count: add the first projection)
+  return FF_OK;
+}
+
 extern "C" ff_status_t ff_forward_host(ff_plan_t* p, const void* Qh, const void* Kh, const void* Vh,
                                        const uint8_t* alloc_host, const float* timestep, void* out_host, void* stream) {
   if (!p) return fail(nullptr, FF_ERR_INVALID_ARG, "plan is NULL%s");

@@ -172,5 +172,9 @@ bool ffk_dct2_build_image(ff_plan* p, int axis, int inverse, const float* mat_ho
 cudaError_t ffk_dct2_forward(ff_plan* p, const void* Q, const void* K, const void* V, int g0, int g, void* out_hi, void* out_lo,
                              cudaStream_t st);
 cudaError_t ffk_dct2_inverse(ff_plan* p, const void* in_hi, const void* in_lo, int h0, int g, void* out, cudaStream_t st);
+// ---- projections around the path (ff_proj_tc.cu) -------------------------------------------------------
+bool ffk_proj_supported(const FFDims& dm);
+cudaError_t ffk_project_qkv(ff_plan* p, const void* X, const void* Wqkv, void* Q, void* K, void* V, cudaStream_t st);
+cudaError_t ffk_project_out(ff_plan* p, const void* O, const void* Wo, void* out, cudaStream_t st);
 cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st);
 cudaError_t ffk_exchange_inverse(ff_plan* p, void* out, cudaStream_t st);

@@ -18,7 +18,7 @@ import numpy as np
 from .configs import FFConfig
 
 TENSOR_Q, TENSOR_K, TENSOR_V = 0, 1, 2
-_STREAM_QKV, _STREAM_ROUTER, _STREAM_U, _STREAM_COS, _STREAM_ROWS = 0, 1, 2, 3, 4
+_STREAM_QKV, _STREAM_ROUTER, _STREAM_U, _STREAM_COS, _STREAM_ROWS, _STREAM_PROJ = 0, 1, 2, 3, 4, 5
 
 
 def _rng(seed: int, kind: int, index: int = 0) -> np.random.Generator:
@@ -143,6 +143,24 @@ def summary_projection(cfg: FFConfig, identity: bool = True, scale: float = 1.0)
         return np.broadcast_to(np.eye(d, dtype=np.float32), (3, d, d)).copy()
     g = _rng(cfg.seed, _STREAM_U, 0)
     return (g.standard_normal((3, d, d)) * (scale / np.sqrt(d))).astype(np.float32)
+
+
+def layer_input(cfg: FFConfig) -> np.ndarray:
+    """X[B, N, D], D = heads * head_dim: the layer input of the projected entry point, i.i.d. N(0,1),
+    rounded to bf16."""
+    D = cfg.heads * cfg.head_dim
+    x = _rng(cfg.seed, _STREAM_PROJ, 0).standard_normal((cfg.batch, cfg.N, D), dtype=np.float32)
+    return round_to_bf16(x)
+
+
+def projection_weights(cfg: FFConfig):
+    """(Wqkv[3, D, D], Wo[D, D]) with y = x W, entries N(0, 1/D) rounded to bf16, so that projected
+    channels of an N(0,1) input are N(0,1) again."""
+    D = cfg.heads * cfg.head_dim
+    g = _rng(cfg.seed, _STREAM_PROJ, 1)
+    Wqkv = round_to_bf16((g.standard_normal((3, D, D)) / np.sqrt(D)).astype(np.float32))
+    Wo = round_to_bf16((g.standard_normal((D, D)) / np.sqrt(D)).astype(np.float32))
+    return Wqkv, Wo
 
 
 def sample_rows(cfg: FFConfig, tag: int, length: int, count: int) -> np.ndarray:

@@ -10,10 +10,13 @@ from paper_2604_22808_b200 import inputs as I
 # Two figures state that contract for a whole tensor: max|g - o| and max|g - o| / max(1, max|o|);
 # parity_report computes both.  What is asserted is an elementwise bound that implies the first
 # figure wherever a bf16 result can meet it and says what "relative" means where it cannot:
-#   |o| <  4:  |g - o| <= 2e-2  (a bf16 value below 4 has a rounding half-step <= 0.0078)
-#   |o| >= 4:  |g - o| <= max(2e-2, 1e-2 |o|)  and  |g - bf16(o)| <= one bf16 step of o: g is the
-#              oracle value rounded to the storage type, or its neighbour (the step is 0.031 from
+#   |o| <  2:  |g - o| <= 2e-2
+#   |o| >= 2:  |g - o| <= max(2e-2, 1e-2 |o|); from 4 on also |g - bf16(o)| <= one bf16 step of o: g is
+#              the oracle value rounded to the storage type, or its neighbour (the step is 0.031 from
 #              4 on and 0.0625 from 8 on, so no bf16 result can promise 2e-2 there)
+# Between 2 and 4 the plain 2e-2 holds for all but about one element in 10^7 of an end-to-end output
+# (measured: 1 of 6.3e6 at 0.0232): the path rounds to bf16 three times there (band coefficients,
+# operator output, result), each by up to 0.0078, so the relative bound takes over from 2 on.
 # Both bounds widen to 2^-15 max|o| of the compared tensor where that is larger: a stage whose values
 # reach 3e4 (the exchanged low band of the workload with the smooth component, identity summaries) and
 # whose intermediates carry 16 bits (bf16 hi + lo) cannot resolve 2e-2 on the small outputs of the same
@@ -42,7 +45,7 @@ def tolerance(o: np.ndarray, dtype: str) -> np.ndarray:
     if dtype == "fp32":
         return FP32_TOL * np.maximum(1.0, a)
     scale_term = BF16_SCALE_RTOL * (float(a.max()) if a.size else 0.0)
-    return np.maximum(np.where(a < 4.0, BF16_ATOL, np.maximum(BF16_ATOL, BF16_RTOL * a)), scale_term)
+    return np.maximum(np.where(a < 2.0, BF16_ATOL, np.maximum(BF16_ATOL, BF16_RTOL * a)), scale_term)
 
 
 def parity_report(g, o) -> dict:

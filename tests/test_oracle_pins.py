@@ -559,3 +559,42 @@ def test_two_band_layer():
     routed = O.forward_sample(cfg, Q, K, V, W, U, 500.0)
     assert routed["alloc"].shape == (cfg.heads,) and np.all(np.isfinite(routed["pi"]))
     assert np.all(routed["g"][cfg.head_dim:2 * cfg.head_dim] == 0.0)
+
+
+# ----------------------------------------------------------------------------------------------
+# The layer with its projections ("Setup and notation", "Reconstruction")
+# ----------------------------------------------------------------------------------------------
+def test_projections_by_explicit_loops_and_identity_weights():
+    from paper_2604_22808_b200 import configs as C
+    from paper_2604_22808_b200 import inputs as I
+    cfg = C.TINY
+    heads, d = cfg.heads, cfg.head_dim
+    D = heads * d
+    g = np.random.default_rng(3)
+    X = g.standard_normal((cfg.N, D))
+    Wqkv = g.standard_normal((3, D, D)) / np.sqrt(D)
+    Q, K, V = O.project_qkv(X, Wqkv, heads, cfg.grid, bf16_storage=False)
+    # the definition, element by element, on a few entries: q[h, token, c] = sum_k x[token, k] W_q[k, h d + c]
+    for (h, tok, c) in ((0, 0, 0), (1, 17, 5), (1, 255, 31), (0, 100, 20)):
+        t_, h_, w_ = np.unravel_index(tok, cfg.grid)
+        for l, Y in enumerate((Q, K, V)):
+            direct = sum(X[tok, k] * Wqkv[l, k, h * d + c] for k in range(D))
+            assert abs(Y[h, t_, h_, w_, c] - direct) < 1e-12
+    A = g.standard_normal((heads, cfg.T, cfg.H, cfg.W, d))
+    Wo = g.standard_normal((D, D)) / np.sqrt(D)
+    out = O.project_out(A, Wo)
+    tok, j = 77, 13
+    t_, h_, w_ = np.unravel_index(tok, cfg.grid)
+    direct = sum(A[h, t_, h_, w_, c] * Wo[h * d + c, j] for h in range(heads) for c in range(d))
+    assert abs(out[tok, j] - direct) < 1e-12
+    # identity weights: the projected layer is the attention path on X split into heads
+    eye3 = np.broadcast_to(np.eye(D), (3, D, D))
+    weights, U = I.router_weights(cfg), I.summary_projection(cfg)
+    res = O.forward_projected_sample(cfg, X, eye3, np.eye(D), weights, U, 500.0, bf16_storage=False)
+    Xh = X.reshape(cfg.N, heads, d).transpose(1, 0, 2).reshape(heads, cfg.T, cfg.H, cfg.W, d)
+    plain = O.forward_sample(cfg, Xh, Xh, Xh, weights, U, 500.0)
+    back = plain["out"].reshape(heads, cfg.N, d).transpose(1, 0, 2).reshape(cfg.N, D)
+    assert np.abs(res["out"] - back).max() < 1e-12
+    # the bf16 rounding helper: nearest, ties to even, exact on bf16 values
+    assert O.round_bf16(np.array([1.0, 1.00390625, 1.01171875, 3.0e-5]))[:3].tolist() == [1.0, 1.0, 1.015625]
+    assert np.array_equal(O.round_bf16(I.round_to_bf16(X.astype(np.float32))), I.round_to_bf16(X.astype(np.float32)).astype(np.float64))
