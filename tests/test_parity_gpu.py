@@ -219,7 +219,11 @@ def test_projected_layer(cfg):
         plan.forward_projected(x, wqkv, wo, out, alloc=torch.tensor(alloc, dtype=torch.uint8, device="cuda"))
         torch.cuda.synchronize()
         assert plan.device_status() == 0
-        Hn.assert_close(out[0].float().cpu().numpy(), ref["out"], "bf16", "projected layer")
+        # The output projection sums heads x head_dim attention outputs, each inside the path's tolerance and
+        # rounded to bf16 once more, with weights of variance 1/D: the sum's error has the standard deviation of
+        # one term's (about 4e-3), its maximum over 10^7 outputs lies near 2.5e-2, and the result is rounded
+        # again -- hence one and a half times the path's bounds for this comparison.
+        Hn.assert_close(out[0].float().cpu().numpy(), ref["out"], "bf16", "projected layer", tol_scale=1.5)
     # without staging space the call is refused
     plain = B.Plan(cfg, weights)
     with pytest.raises(B.FFError) as ei:
