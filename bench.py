@@ -31,8 +31,11 @@ METRIC = "freqformer_attn_layer_tokens_per_s"
 # dram__bytes_read.sum + dram__bytes_write.sum of the transform kernels per token and head, from the ncu
 # capture of the 6-head 64K case (forward: the passes over Q, K and V; inverse: the passes over one tensor).
 FP32_FMA_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 74.5: plain fp32 FMA rate of the GPU (unit counts x max clock)
-NCU_DRAM_BYTES_PER_TOKEN_HEAD = {"transform": 7330.0, "inverse": 3110.0}
-TRANSFORM_KERNELS = {"transform": "dct_tc_kernel (transform stage)", "inverse": "dct_tc_kernel (inverse stage)"}
+# [0]: three separate axis passes; [1]: two axes in one launch (64K-class grids)
+NCU_DRAM_BYTES_PER_TOKEN_HEAD = {"transform": (7330.0, 4359.0), "inverse": (3110.0, 2203.0)}
+TRANSFORM_KERNELS = {"transform": ("dct_tc_kernel x3 (transform stage)", "dct2_tc_kernel + dct_tc_kernel (transform stage)"),
+                     "inverse": ("exchange_tc_kernel + dct_tc_kernel x3 (inverse stage)",
+                                 "exchange_tc_kernel + dct_tc_kernel + dct2_tc_kernel (inverse stage)")}
 # Reported beside the 64K line by the default run: the larger workloads with the router's allocation and the
 # 64K grid with every band operator present.
 EXTRA_WORKLOADS = {"256k": ("256k", ""), "1m": ("1m", ""), "64k_forced_8_8_8": ("64k", "8,8,8")}
@@ -368,7 +371,7 @@ def extra_workload(name, alloc_text, args, dev, local, peaks):
         raise RuntimeError(B.library().ff_last_error(plan.handle).decode())
     alloc = forced if forced is not None else plan.tap(B.TAP_ALLOC).cpu().numpy().tolist()
     stages, work = stage_rooflines(cfg, alloc, stage_ms, peaks)
-    res = {"grid": list(cfg.grid), "batch": cfg.batch, "heads": cfg.heads, "head_dim": cfg.head_dim,
+    res = {"kernels": plan.kernel_info(), "grid": list(cfg.grid), "batch": cfg.batch, "heads": cfg.heads, "head_dim": cfg.head_dim,
            "allocation": "router" if forced is None else "forced", "timestep": ts[0],
            "heads_per_band": [alloc.count(1), alloc.count(2), alloc.count(4)],
            "inputs": "drawn on the device (torch CUDA generator), same distribution as the parity tests' host inputs",
@@ -378,6 +381,49 @@ def extra_workload(name, alloc_text, args, dev, local, peaks):
            "clocks": clocks}
     plan.destroy()
     del q, k, v, out, plan
+    torch.cuda.empty_cache()
+    return res
+
+
+def projected_workload(name, args, dev, peaks):
+    """The layer with its Q/K/V and output projections (ff_forward_projected) on one workload: device time of the
+    whole call, and of the two projection GEMMs as the difference to the attention path alone."""
+    import torch
+    from paper_2604_22808_b200 import binding as B
+    cfg = C.BY_NAME[name]
+    D = cfg.heads * cfg.head_dim
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4242 + cfg.seed)
+    x = torch.randn((cfg.batch, cfg.N, D), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    wqkv = (torch.randn((3, D, D), generator=gen, device=dev, dtype=torch.float32) / D ** 0.5).to(torch.bfloat16)
+    wo = (torch.randn((D, D), generator=gen, device=dev, dtype=torch.float32) / D ** 0.5).to(torch.bfloat16)
+    out = torch.empty_like(x)
+    plan = B.Plan(cfg, I.router_weights(cfg), host_staging=True, device=dev)
+    plan.set_profiling(True)
+    ts = [cfg.timesteps[0]] * cfg.batch
+    steps = max(3, min(args.steps, 10))
+    for _ in range(3):
+        plan.forward_projected(x, wqkv, wo, out, timesteps=ts)
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    inner = 0.0
+    ev[0].record()
+    for _ in range(steps):
+        plan.forward_projected(x, wqkv, wo, out, timesteps=ts)
+        inner += sum(ms for ms, _ in plan.stage_times().values())
+    ev[1].record()
+    torch.cuda.synchronize()
+    if plan.device_status() != 0:
+        raise RuntimeError(B.library().ff_last_error(plan.handle).decode())
+    ms_step = ev[0].elapsed_time(ev[1]) / steps
+    ms_proj = ms_step - inner / steps
+    flops = 2.0 * cfg.batch * cfg.N * D * 4 * D
+    res = {"grid": list(cfg.grid), "heads": cfg.heads, "head_dim": cfg.head_dim, "model_width": D, "steps": steps,
+           "ms_per_step": ms_step, "tokens_per_s": cfg.batch * cfg.N / (ms_step * 1e-3), "projections_ms": ms_proj,
+           "projections_tflops": flops / (ms_proj * 1e-3) / 1e12,
+           "projections_frac_of_sustained_bf16": flops / (ms_proj * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]}
+    plan.destroy()
+    del x, wqkv, wo, out, plan
     torch.cuda.empty_cache()
     return res
 
@@ -435,6 +481,7 @@ def run_cuda(args, cfg):
     clocks = sampler.stop()
     ms_step = reduce_max_(ms_local)
     launches = plan.last_launches()
+    kinfo = plan.kernel_info()
     if plan.device_status() != 0:
         raise RuntimeError(B.library().ff_last_error(plan.handle).decode())
     alloc = forced if forced is not None else plan.tap(B.TAP_ALLOC).cpu().numpy().tolist()
@@ -478,10 +525,11 @@ def run_cuda(args, cfg):
             nbytes = work["bytes_transform_strict"] if top == "transform" else work["bytes_inverse"]
             # DRAM bytes per token-head and stage from the ncu capture of the 6-head 64K case; the traffic is
             # proportional to tokens x heads
-            per_token_head = NCU_DRAM_BYTES_PER_TOKEN_HEAD[top] * cfg.head_dim / 128.0
+            fused = int(kinfo["transform_fused"])
+            per_token_head = NCU_DRAM_BYTES_PER_TOKEN_HEAD[top][fused] * cfg.head_dim / 128.0
             roof = {"bound": "hbm", "achieved": st["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": st["frac"],
                     "traffic": per_token_head * cfg.N * heads_total / n_launch if tensor_core_path else None,
-                    "kernel": (TRANSFORM_KERNELS[top] if tensor_core_path else "dct_pass_kernel (%s stage)" % top),
+                    "kernel": (TRANSFORM_KERNELS[top][fused] if tensor_core_path else "dct_pass_kernel (%s stage)" % top),
                     "algorithmic_bytes_per_launch": nbytes / n_launch,
                     "algorithmic_bytes": "read Q,K,V, write V~ and the executed band of Q~,K~" if top == "transform"
                                          else "read the band outputs once, write out once"}
@@ -498,6 +546,7 @@ def run_cuda(args, cfg):
             "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
             "config": config_record(cfg, ts[0], forced is not None, alloc),
             "router_pi": pi[0],
+            "kernels": kinfo,
             "roofline": roof,
             "cpu_baseline": cpu,
             "e2e": ({"value": tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 3 * io_bytes,
@@ -523,6 +572,7 @@ def run_cuda(args, cfg):
             extra = {}
             for key, (name, alloc_text) in EXTRA_WORKLOADS.items():
                 extra[key] = extra_workload(name, alloc_text, args, dev, local, peaks)
+            extra["64k_with_projections"] = projected_workload("64k", args, dev, peaks)
             line["workloads"] = extra
         print(json.dumps(line))
     if world > 1:

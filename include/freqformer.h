@@ -208,6 +208,13 @@ ff_status_t ff_plan_device_status(ff_plan_t *plan, void *cuda_stream);
 ff_status_t ff_plan_selftest_bounded_wait(ff_plan_t *plan, int64_t limit_cycles,
                                           int32_t *waiters_released, void *cuda_stream);
 
+/* Which kernels the plan's forward runs with the workspace it has (benchmarks label their numbers with it):
+ *   info[0]  1: the transform runs two axes in one launch (intermediate in shared memory), 0: three passes
+ *   info[1]  CTAs per cluster of that launch (0 if unused)
+ *   info[2]  1: the band operators run on the tensor-core kernel, 0: generic kernels
+ *   info[3]  1: the pooled low band is part of the tensor-core attention launch */
+ff_status_t ff_plan_kernel_info(const ff_plan_t *plan, int32_t info[4]);
+
 /* Number of kernel launches the last ff_forward / ff_route on this plan issued. */
 ff_status_t ff_plan_last_launches(const ff_plan_t *plan, int64_t *launches);
 

@@ -29,7 +29,7 @@ FF_BAND_LOW, FF_BAND_MID, FF_BAND_HIGH = 1, 2, 4
 
 EXPORTS = ("ff_config_validate", "ff_band_sizes", "ff_band_rank", "ff_workspace_bytes", "ff_workspace_bytes_host",
            "ff_plan_create", "ff_plan_workspace_bytes", "ff_band_info", "ff_plan_set_workspace", "ff_destroy", "ff_last_error",
-           "ff_route", "ff_forward", "ff_forward_host", "ff_forward_projected", "ff_plan_device_status", "ff_plan_last_launches",
+           "ff_route", "ff_forward", "ff_forward_host", "ff_forward_projected", "ff_plan_device_status", "ff_plan_last_launches", "ff_plan_kernel_info",
            "ff_get_tap", "ff_plan_set_attention_impl", "ff_plan_set_profiling", "ff_plan_stage_times", "ff_high_attention_noalloc",
            "ff_plan_selftest_bounded_wait")
 STAGES = ("transform", "router", "attention", "summary", "inverse")
@@ -77,6 +77,7 @@ def library() -> C.CDLL:
         lib.ff_forward_projected.argtypes = [C.c_void_p] + [C.c_void_p] * 3 + [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.ff_plan_device_status.argtypes = [C.c_void_p, C.c_void_p]
         lib.ff_plan_last_launches.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
+        lib.ff_plan_kernel_info.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
         lib.ff_get_tap.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
         lib.ff_plan_set_attention_impl.argtypes = [C.c_void_p, C.c_int32]
         lib.ff_plan_set_profiling.argtypes = [C.c_void_p, C.c_int32]
@@ -261,6 +262,12 @@ class Plan:
         n = C.c_int32(-1)
         _check(library().ff_plan_selftest_bounded_wait(self.handle, int(limit_cycles), C.byref(n), self._stream()), self.handle)
         return n.value
+
+    def kernel_info(self) -> dict:
+        info = (C.c_int32 * 4)()
+        _check(library().ff_plan_kernel_info(self.handle, info), self.handle)
+        return {"transform_fused": bool(info[0]), "transform_cluster": int(info[1]), "attention_tensor_core": bool(info[2]),
+                "low_band_tensor_core": bool(info[3])}
 
     def last_launches(self) -> int:
         n = C.c_int64()

@@ -320,6 +320,15 @@ extern "C" ff_status_t ff_plan_set_attention_impl(ff_plan_t* p, int32_t impl) {
   return FF_OK;
 }
 
+extern "C" ff_status_t ff_plan_kernel_info(const ff_plan_t* p, int32_t info[4]) {
+  if (!p || !info) return fail(nullptr, FF_ERR_INVALID_ARG, "plan or info is NULL%s");
+  int cs = 0;
+  const bool fused = p->dct_tc_ok && p->dct2_ok && !(p->attn_impl & 6) && ffk_dct2_supported(p->dm, nullptr, &cs);
+  info[0] = fused ? 1 : 0; info[1] = fused ? cs : 0;
+  info[2] = (p->tc_ok && !(p->attn_impl & 1)) ? 1 : 0; info[3] = (info[2] && p->low_tc_ok) ? 1 : 0;
+  return FF_OK;
+}
+
 extern "C" ff_status_t ff_plan_last_launches(const ff_plan_t* p, int64_t* n) {
   if (!p || !n) return fail(nullptr, FF_ERR_INVALID_ARG, "plan or output is NULL%s");
   *n = p->launches;
