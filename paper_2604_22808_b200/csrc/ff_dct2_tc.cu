@@ -77,9 +77,11 @@ __device__ unsigned long long g_d2_prof[32];
 
 struct D2Shared {
   uint64_t in_full[NSTG], in_empty[NSTG], acc1_full[NA1], acc1_empty[NA1], acc2_full[NA2], acc2_empty[NA2];
-  uint64_t buf_full;       // all rows of the item have landed in this CTA's buffer (arrivals from every CTA's warps)
-  uint64_t buf_free;       // every CTA of the cluster has finished reading its buffer (phase 2 of the item)
-  uint64_t mma2_done;      // this CTA's phase-2 instructions of the item have completed
+  // The plane buffer has one slot of 8 tiles or two of 4 (items alternate): phase 1 of the next item fills one
+  // slot while phase 2 of the current item reads the other.
+  uint64_t buf_full[2];    // all rows of the item have landed in this CTA's slot (arrivals from every CTA's warps)
+  uint64_t buf_free[2];    // every CTA of the cluster has finished reading the slot (phase 2 of the item)
+  uint64_t mma2_done[2];   // this CTA's phase-2 instructions of the item (by slot) have completed
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -220,6 +222,7 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   const int lkf2 = 31 - __clz(kf2);
   const int ltpc = 31 - __clz(tpc);
   const int total = P.group * P.n3 * P.nchunk;
+  const int nsl = tpc <= MAX_TPC / 2 ? 2 : 1;                      // slots of the plane buffer
   const int bt = tpc < 4 ? tpc : 4;                                // tiles per instruction batch (N = 32 bt columns): an
   const int nb = tpc / bt;                                         // instruction costs the same for any N up to 128
 
@@ -227,9 +230,8 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
     for (int i = 0; i < NSTG; ++i) { mbar_init(&sh.in_full[i], 1); mbar_init(&sh.in_empty[i], 1); }
     for (int i = 0; i < NA1; ++i) { mbar_init(&sh.acc1_full[i], 1); mbar_init(&sh.acc1_empty[i], 256); }
     for (int i = 0; i < NA2; ++i) { mbar_init(&sh.acc2_full[i], 1); mbar_init(&sh.acc2_empty[i], 256); }
-    mbar_init(&sh.buf_full, 8 * cs);
-    mbar_init(&sh.buf_free, cs);
-    mbar_init(&sh.mma2_done, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.buf_full[i], 8 * cs); mbar_init(&sh.buf_free[i], cs); }
+    mbar_init(&sh.mma2_done[0], 1); mbar_init(&sh.mma2_done[1], 1);
     sh.abort_flag = 0;
     fence_mbar_init();
   }
@@ -360,7 +362,8 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       for (int it = cid; it < total && ok; it += ncl, ++ni) {
         // the plane's rows have landed in this CTA's buffer
         PROF_T0(tm2);
-        ok = mbar_wait_cluster(&sh.buf_full, ni & 1, abort_flag);
+        const int sl = (int)(ni % nsl);                             // the item's slot of the plane buffer
+        ok = mbar_wait_cluster(&sh.buf_full[sl], (ni / nsl) & 1, abort_flag);
         PROF_ADD(9, tm2);
         if (!ok) break;
         fence_proxy_async_all();
@@ -371,7 +374,7 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           PROF_ADD(10, tm3);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t x0 = buf_base + (uint32_t)(bt * kb) * 2 * TILE_B;    // tiles bt kb ..: hi, lo of each in turn
+          const uint32_t x0 = buf_base + (uint32_t)(sl * tpc + bt * kb) * 2 * TILE_B;   // tiles bt kb ..: hi, lo of each in turn
           const uint64_t xh = smem_desc_sw64(x0, 2 * TILE_B, 512), xl = smem_desc_sw64(x0 + TILE_B, 2 * TILE_B, 512);
           const uint32_t d_tm = tm + COL_ACC2 + ab * 128;
 #pragma unroll
@@ -382,7 +385,7 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           }
           umma_commit(&sh.acc2_full[ab]);
         }
-        umma_commit(&sh.mma2_done);
+        umma_commit(&sh.mma2_done[sl]);
       }
     }
   } else if (warp == 2) {
@@ -391,9 +394,9 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       unsigned ni = 0;
       bool ok = true;
       for (int it = cid; it < total && ok; it += ncl, ++ni) {
-        ok = mbar_wait(&sh.mma2_done, ni & 1, abort_flag);
+        ok = mbar_wait(&sh.mma2_done[ni % nsl], (ni / nsl) & 1, abort_flag);
         if (!ok) break;
-        for (int rk = 0; rk < cs; ++rk) mbar_arrive_cluster(mapa(smem_u32(&sh.buf_free), (uint32_t)rk));
+        for (int rk = 0; rk < cs; ++rk) mbar_arrive_cluster(mapa(smem_u32(&sh.buf_free[ni % nsl]), (uint32_t)rk));
       }
     }
   } else if (warp >= 4 && warp < 12) {
@@ -418,8 +421,9 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
     bool ok = true;
     for (int it = cid; it < total && ok; it += ncl, ++ni) {
       PROF_T0(te0);
-      if (ni >= 1) {
-        ok = __all_sync(0xffffffffu, mbar_wait_cluster(&sh.buf_free, (ni - 1) & 1, abort_flag));
+      const int sl = (int)(ni % nsl);                         // the item's slot: free once phase 2 of item ni - nsl is done
+      if (ni >= (unsigned)nsl) {
+        ok = __all_sync(0xffffffffu, mbar_wait_cluster(&sh.buf_free[sl], ((ni / nsl) - 1) & 1, abort_flag));
         if (!ok) break;
       }
       if (threadIdx.x == 128) PROF_ADD(1, te0);
@@ -445,7 +449,7 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         const int u1 = (int)rank * tpc + bt * kb + tb;
         const int b = u1 * kf1 + l1;
         const int drow = (b << lkf2) | (a1 & (kf2 - 1));
-        const uint32_t laddr = buf_base + (uint32_t)u2l * 2 * TILE_B + (uint32_t)drow * STG_ROW;
+        const uint32_t laddr = buf_base + (uint32_t)(sl * tpc + u2l) * 2 * TILE_B + (uint32_t)drow * STG_ROW;
         const uint32_t daddr = cs == 1 ? laddr : mapa(laddr, owner);
         const int swz = (drow >> 1) & 3;
         // (debug build) the row lies inside a tile of the owner's buffer
@@ -487,11 +491,11 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       if (cs == 1) {
         fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.buf_full);
+        if (lane == 0) mbar_arrive(&sh.buf_full[sl]);
       } else {
         fence_proxy_async_all();
         __syncwarp();
-        if (lane < cs) mbar_arrive_cluster(mapa(smem_u32(&sh.buf_full), (uint32_t)lane));
+        if (lane < cs) mbar_arrive_cluster(mapa(smem_u32(&sh.buf_full[sl]), (uint32_t)lane));
       }
       if (threadIdx.x == 128) PROF_ADD(6, te4);
     }
