@@ -44,6 +44,11 @@ struct XParams {
   int h0, g;                  // heads [h0, h0+g)
   int nkeys;                  // 3m rounded up to a multiple of 16
   int ybufs;                  // token-tile buffers in shared memory (1 or 2)
+  // With one buffer (two CTAs with two buffers each no longer fit an SM: more than 64 summary keys) the tile is
+  // handed back to the producer as soon as the score MMAs have read it, and the store warps take the tokens for
+  // the residual add from global memory instead (they were just loaded: L2 hits), so that the next tile's load
+  // still overlaps this tile's softmax and stores.
+  const __nv_bfloat16* src[4];   // y_mid, v~_mid, y_high, v~_high: bases of the buffers the four maps cover
   int* status;
 };
 
@@ -102,7 +107,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
   const int it1 = it0 + chunk < total ? it0 + chunk : total;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; ++i) { mbar_init(&sh.y_full[i], 1); mbar_init(&sh.y_empty[i], 128); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.y_full[i], 1); mbar_init(&sh.y_empty[i], P.ybufs == 1 ? 1 : 128); }
     mbar_init(&sh.z_ready, 128); mbar_init(&sh.s_full, 1); mbar_init(&sh.p_full, 128);
     mbar_init(&sh.d_full, 1); mbar_init(&sh.d_empty, 128);
     sh.abort_flag = 0;
@@ -161,6 +166,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
           umma_ss(tmem, a, smem_desc_sw128(zlo + zo, 16, 1024), idesc1, 1u);
         }
         umma_commit(&sh.s_full);
+        if (YB == 1) umma_commit(&sh.y_empty[slot]);      // single buffer: free for the next load once the scores are done
         ok = mbar_wait(&sh.p_full, n & 1, abort_flag);
         if (ok && n >= 1) ok = mbar_wait(&sh.d_empty, (n - 1) & 1, abort_flag);
         if (!ok) break;
@@ -325,6 +331,10 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       for (int i = 0; i < 4; ++i) fpos[i] = __shfl_sync(0xffffffffu, f, 8 * i + (lane >> 2));
       const size_t obase = (size_t)(x.bh - P.h0) * dm.N * XD;
       const uint8_t* yrow = sY + slot * X_TILE_BYTES + row * 128;
+      // (single buffer) this token's row in global memory; rows past the band end are never stored
+      const bool exec_g = P.alloc[x.bh] & (1 << x.band);
+      const __nv_bfloat16* grow = P.src[(x.band == 1 ? 0 : 2) + (exec_g ? 0 : 1)] +
+                                  ((size_t)(exec_g ? x.bh : 2 * dm.BH + x.bh) * n_band + (valid ? p : 0)) * XD;
       const float dscale = NK32 >= 2 ? sh.inv[n & 1][row] : 1.f;    // (two-sweep variants: P was left unnormalised)
       uint8_t* st_hi = sh.stage[quarter][0];
       uint8_t* st_lo = sh.stage[quarter][1];
@@ -337,7 +347,8 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         for (int v4 = 0; v4 < 4; ++v4) {
           // channels 32q + 8v4 .. +7 of this token: one 16-byte chunk of the swizzled Y tile
           const int cch = q * 4 + v4;                    // 16-byte chunk index along the row, 0..15
-          const uint4 yv = *(const uint4*)(yrow + (cch >> 3) * X_HALF + (((cch & 7) ^ (row & 7)) << 4));
+          const uint4 yv = YB == 1 ? __ldg((const uint4*)(grow + cch * 8))
+                                   : *(const uint4*)(yrow + (cch >> 3) * X_HALF + (((cch & 7) ^ (row & 7)) << 4));
           const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
           uint32_t hi[4], lo[4];
 #pragma unroll
@@ -368,7 +379,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       }
       tc_fence_before();
       mbar_arrive(&sh.d_empty);
-      mbar_arrive(&sh.y_empty[slot]);
+      if (YB > 1) mbar_arrive(&sh.y_empty[slot]);
     }
   }
 
@@ -449,6 +460,8 @@ cudaError_t ffk_exchange_tc(ff_plan* p, int h0, int g, void* grid_hi, void* grid
   P.pos_mid = p->pos_table; P.pos_high = p->pos_table + dm.Nmid;
   P.grid_hi = (__nv_bfloat16*)grid_hi; P.grid_lo = (__nv_bfloat16*)grid_lo;
   P.h0 = h0; P.g = g; P.nkeys = (3 * dm.m + 15) / 16 * 16; P.status = p->buf.status;
+  P.src[0] = (const __nv_bfloat16*)p->buf.y_mid; P.src[1] = (const __nv_bfloat16*)p->buf.spec_mid;
+  P.src[2] = (const __nv_bfloat16*)p->buf.y_high; P.src[3] = (const __nv_bfloat16*)p->buf.spec_high;
   // Two CTAs per SM; the token tile is double-buffered if both still fit in shared memory
   const int per_sm = 2;
   P.ybufs = (2 * X_TILE_BYTES + 4 * P.nkeys * 128 + sizeof(XShared) + 2048) * per_sm <= 227 * 1024 ? 2 : 1;
