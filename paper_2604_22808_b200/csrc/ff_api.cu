@@ -177,7 +177,7 @@ extern "C" ff_status_t ff_destroy(ff_plan_t* p) {
     for (int i = 0; i <= 2 * FF_COPY_EVENTS; ++i) cudaEventDestroy(p->ev_copy[i]);
     cudaStreamDestroy(p->copy_stream);
   }
-  cudaFree(p->dct_images); cudaFree(p->dct2_images); cudaFree(p->pos_table);
+  cudaFree(p->dct2_images); cudaFree(p->pos_table);
   cudaFree(p->W1); cudaFree(p->b1); cudaFree(p->W2); cudaFree(p->b2); cudaFree(p->U);
   delete p;
   return FF_OK;
@@ -228,9 +228,6 @@ extern "C" ff_status_t ff_plan_create(const ff_config_t* c, const ff_weights_t* 
     s = upload(p, &p->basis[a], C.data(), C.size());
     if (s == FF_OK) s = upload(p, &p->basis_t[a], Ct.data(), Ct.size());
     if (s == FF_OK && ffk_dct_tc_supported(p->dm) &&
-        !(ffk_dct_tc_build_image(p, a, 0, C.data(), n[a]) && ffk_dct_tc_build_image(p, a, 1, Ct.data(), n[a])))
-      s = fail(p, FF_ERR_CUDA, "could not upload the transform matrix images%s");
-    if (s == FF_OK && ffk_dct2_supported(p->dm, nullptr, nullptr) &&
         !(ffk_dct2_build_image(p, a, 0, C.data(), n[a]) && ffk_dct2_build_image(p, a, 1, Ct.data(), n[a])))
       s = fail(p, FF_ERR_CUDA, "could not upload the transform matrix images%s");
   }
@@ -306,7 +303,7 @@ extern "C" ff_status_t ff_plan_set_workspace(ff_plan_t* p, void* ptr, size_t byt
   if (ffk_dct_tc_supported(p->dm)) {
     const size_t room = (size_t)((char*)base + o[14] - (char*)b.scratchA) + (size_t)p->lay.group * p->dm.N * p->dm.d * 4;
     const int G = p->lay.tc_group;
-    if (p->dct_images && ffk_dct_tc_scratch_bytes(p->dm, G) <= room) { p->dct_tc_ok = true; p->dct_group = G; }
+    if (p->dct2_images && ffk_dct_tc_scratch_bytes(p->dm, G) <= room) { p->dct_tc_ok = true; p->dct_group = G; }
   }
   return FF_OK;
 }

@@ -6,7 +6,7 @@
 // axis position for the h and t axes, so that the strided axes also read contiguous pieces).
 // One tile is one 128 x 128 x 128 contraction
 //     D[j][c] = sum_r A[j][r] * X[r][c],   A = Mat kron I (or I kron Mat) over the lines of the tile
-// with A the K-major operand built once per CTA in shared memory, X the TMA tile used in place as
+// with A held in tensor memory for the whole launch (loaded once per CTA), X the TMA tile used in place as
 // the MN-major B operand, and D in tensor memory with one output position per lane, so that an
 // epilogue thread owns a whole 256-byte output row and stores it with 16-byte accesses.
 //
@@ -16,8 +16,8 @@
 // values (low-frequency content, the constant offset the exchange adds to a whole band), so a
 // single bf16 rounding between passes would not meet the output tolerance.
 //
-//   warp 0      TMA producer (ring of 2-4 stages, as many as fit beside the matrix images)
-//   warp 1      tcgen05.mma issuer, 4 accumulator buffers of 128 TMEM columns
+//   warp 0      TMA producer (ring of 3-6 stages)
+//   warp 1      tcgen05.mma issuer (A from tensor memory), 3 accumulator buffers of 128 TMEM columns
 //   warps 2..9  epilogue: tcgen05.ld, convert to hi/lo bf16, store; a thread owns one output position
 // Output path (FIRST, MIDDLE, LAST): an epilogue warp's 32 rows are 32 grid positions that form a
 // box of the grid, so the warp writes 32 channels of them (64 bytes per row, 64-byte swizzle, no
@@ -48,14 +48,16 @@ constexpr int TILE_ROWS = 128;
 constexpr int TILE_BYTES = TILE_ROWS * CH_MAX * 2; // 32 KB: 128 rows of bf16
 constexpr int HALF_BYTES = TILE_BYTES / 2;
 constexpr int MAX_STAGE = 8;
-constexpr int NACC = 4;
+constexpr int NACC = 3;                     // accumulator buffers of 128 tensor-memory columns, behind the matrix (128 columns)
+constexpr int IMG_CELLS = 64;               // 32-bit tensor-memory cells per matrix row: two bf16 K elements each
+constexpr uint32_t COL_IMG_HI = 0, COL_IMG_LO = 64, COL_ACC = 128;
 constexpr int DCT_TC_THREADS = 320;        // TMA warp, MMA warp, 8 epilogue warps
 
 enum { MODE_FIRST = 0, MODE_MIDDLE = 1, MODE_SPLIT = 2, MODE_LAST = 3 };
 
 struct DctTcParams {
   FFDims dm;
-  const uint8_t* image;    // matrix images (hi then lo, 32 KB each) in their shared-memory layout
+  const uint32_t* image;   // matrix image as the tensor-memory A operand: hi [128][64] cells, then lo
   int n;                   // axis length
   int axis;                // 0 = t, 1 = h, 2 = w
   int mode;
@@ -72,7 +74,7 @@ struct DctTcParams {
 constexpr int STG_PITCH = 64;                       // bytes per staged row piece; the 16-byte chunks are rotated by row/2 against bank conflicts
 
 struct DctShared {
-  uint64_t full[MAX_STAGE], empty[MAX_STAGE], acc_full[NACC], acc_empty[NACC], img_full;
+  uint64_t full[MAX_STAGE], empty[MAX_STAGE], acc_full[NACC], acc_empty[NACC];
   uint32_t tmem_base;
   int abort_flag;
   // per epilogue warp: 32 rows x 64 bytes of hi and of lo, to turn one-row-per-thread registers
@@ -106,12 +108,6 @@ __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.comm
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(smem_u32(smem_dst)), "l"((uint64_t)gsrc), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
-
 // Three source maps (Q, K, V) in MODE_FIRST; otherwise map0 (= hi) and, for split input, map1 (= lo).
 // map_oh / map_ol: destination hi / lo grids with the box of one epilogue warp (32 positions x 32
 // channels), all modes but SPLIT; MODE_LAST has no lo grid.
@@ -133,9 +129,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
   constexpr int TB = TILE_ROWS * CH * 2;                  // bytes of one data tile (16 KB for 64 channels)
   const int STAGE_BYTES = P.in_split ? 2 * TB : TB;       // hi tile, then lo tile
   uint8_t* sData = smem;                                  // NSTAGE x STAGE_BYTES
-  uint8_t* sHi = smem + NSTAGE * STAGE_BYTES;             // matrix hi: [K half][128 rows][128 B], swizzled
-  uint8_t* sLo = sHi + TILE_BYTES;                        // matrix lo
-  DctShared& sh = *(DctShared*)(sLo + TILE_BYTES);
+  DctShared& sh = *(DctShared*)(smem + NSTAGE * STAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_per_th = (int)(dm.N / TILE_ROWS);
   const int total_tiles = P.group * tiles_per_th;
@@ -143,7 +137,6 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NSTAGE; ++i) { mbar_init(&sh.full[i], 1); mbar_init(&sh.empty[i], 1); }
     for (int i = 0; i < NACC; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 256); }
-    mbar_init(&sh.img_full, 1);
     sh.abort_flag = 0;
     fence_mbar_init();
   }
@@ -154,13 +147,34 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
   const uint32_t tm = sh.tmem_base;
   volatile int* abort_flag = &sh.abort_flag;
 
+  if (warp >= 2 && warp < 6) {
+    // The matrix (hi and lo bf16 parts) into tensor memory, where it is the A operand of every tile: a thread
+    // loads the row of its lane (prepared at plan creation as pairs of bf16 K elements per 32-bit cell).
+    const int quarter = warp & 3, row = quarter * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+#pragma unroll 1
+    for (int im = 0; im < 2; ++im) {
+      const uint32_t* src = P.image + (size_t)im * TILE_ROWS * IMG_CELLS + (size_t)row * IMG_CELLS;
+#pragma unroll
+      for (int c0 = 0; c0 < IMG_CELLS; c0 += 32) {
+        uint32_t r[32];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const uint4 v = *(const uint4*)(src + c0 + 4 * i);
+          r[4 * i] = v.x; r[4 * i + 1] = v.y; r[4 * i + 2] = v.z; r[4 * i + 3] = v.w;
+        }
+        tmem_st32(tm + lane_addr + im * 64 + c0, r);
+      }
+    }
+    tmem_wait_st();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+
   if (warp == 0) {
     if (lane == 0) {
       tma_prefetch_desc(&map0);
-      // the two matrix images (prepared at plan creation, already in the operand layout)
-      mbar_arrive_expect_tx(&sh.img_full, 2 * TILE_BYTES);
-      bulk_load(sHi, P.image, TILE_BYTES, &sh.img_full);
-      bulk_load(sLo, P.image + TILE_BYTES, TILE_BYTES, &sh.img_full);
       unsigned it = 0;
       bool ok = true;
       for (int s = blockIdx.x; s < total_tiles && ok; s += gridDim.x, ++it) {
@@ -190,9 +204,8 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16_f32(TILE_ROWS, CH, /*a_mn_major=*/false, /*b_mn_major=*/true);
-      const uint32_t hi_base = smem_u32(sHi), lo_base = smem_u32(sLo);
       unsigned it = 0;
-      bool ok = mbar_wait(&sh.img_full, 0, abort_flag);
+      bool ok = true;
       for (int s = blockIdx.x; s < total_tiles && ok; s += gridDim.x, ++it) {
         const int slot = it % NSTAGE, ab = it % NACC;
         ok = mbar_wait(&sh.full[slot], (it / NSTAGE) & 1, abort_flag);
@@ -200,15 +213,14 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
         if (!ok) break;
         tc_fence_after();
         const uint32_t dbase = smem_u32(sData + slot * STAGE_BYTES);
-        const uint32_t d_tm = tm + ab * 128;
+        const uint32_t d_tm = tm + COL_ACC + ab * 128;
+        const uint64_t xh0 = smem_desc_sw128(dbase, HALF_BYTES, 1024), xl0 = smem_desc_sw128(dbase + TB, HALF_BYTES, 1024);
 #pragma unroll
         for (int ks = 0; ks < TILE_ROWS / 16; ++ks) {
-          const uint32_t aoff = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-          const uint64_t ahi = smem_desc_sw128(hi_base + aoff, 16, 1024);
-          const uint64_t xhi = smem_desc_sw128(dbase + ks * 2048, HALF_BYTES, 1024);
-          umma_ss(d_tm, ahi, xhi, idesc, ks > 0 ? 1u : 0u);
-          umma_ss(d_tm, smem_desc_sw128(lo_base + aoff, 16, 1024), xhi, idesc, 1u);
-          if (P.in_split) umma_ss(d_tm, ahi, smem_desc_sw128(dbase + TB + ks * 2048, HALF_BYTES, 1024), idesc, 1u);
+          // (a descriptor advances by 2048 bytes = 128 in its address field per 16 rows of K)
+          umma_ts(d_tm, tm + COL_IMG_HI + ks * 8, xh0 + (uint64_t)(ks * 128), idesc, ks > 0 ? 1u : 0u);
+          umma_ts(d_tm, tm + COL_IMG_LO + ks * 8, xh0 + (uint64_t)(ks * 128), idesc, 1u);
+          if (P.in_split) umma_ts(d_tm, tm + COL_IMG_HI + ks * 8, xl0 + (uint64_t)(ks * 128), idesc, 1u);
         }
         umma_commit(&sh.empty[slot]);
         umma_commit(&sh.acc_full[ab]);
@@ -308,7 +320,7 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
       // both 32-channel chunks of the row at once; the accumulator buffer is free as soon as they are read
       uint32_t rr2[NQ][32];
 #pragma unroll
-      for (int qi = 0; qi < NQ; ++qi) tmem_ld32(tm + lane_addr + ab * 128 + (q_lo + qi) * 32, rr2[qi]);
+      for (int qi = 0; qi < NQ; ++qi) tmem_ld32(tm + lane_addr + COL_ACC + ab * 128 + (q_lo + qi) * 32, rr2[qi]);
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(&sh.acc_empty[ab]);
@@ -481,9 +493,8 @@ bool encode_store_map(CUtensorMap* map, const void* base, const FFDims& dm, int 
 
 cudaError_t launch_pass(ff_plan* p, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& m2,
                         const CUtensorMap& moh, const CUtensorMap& mol, DctTcParams& P, cudaStream_t st) {
-  const size_t img = TILE_BYTES;
   const size_t stage = (size_t)(P.in_split ? 2 : 1) * TILE_ROWS * P.dm.d * 2;
-  const size_t fixed = 2 * img + sizeof(DctShared) + 1024;
+  const size_t fixed = sizeof(DctShared) + 1024;
   int nstage = (int)((232448 - 256 - fixed) / stage);   // 227 KB of shared memory per CTA
   if (nstage > MAX_STAGE) nstage = MAX_STAGE;
   P.nstage = nstage;
@@ -514,33 +525,11 @@ bool ffk_dct_tc_supported(const FFDims& dm) {
   return dm.H % (TILE_ROWS / dm.W) == 0 && dm.W % (TILE_ROWS / dm.H) == 0 && dm.W % (TILE_ROWS / dm.T) == 0;
 }
 
-// Matrix images of one axis (0 = t, 1 = h, 2 = w) and direction, in the layout the kernel's A
-// operand has in shared memory: row j = output position of a tile, 64 input positions per 128-byte
-// row, 16-byte chunks XOR-swizzled with the row index (the 128-byte swizzle the MMA expects), the
-// bf16 hi part followed by the lo part.  Lines that follow one another (w axis): I kron Mat,
-// index = line*n + a.  Interleaved lines (h, t axes): Mat kron I, index = a*kf + line.
-// `mat` is the host matrix [n][n] with out[a] = sum_b mat[a][b] in[b].
-bool ffk_dct_tc_build_image(ff_plan* p, int axis, int inverse, const float* mat, int n) {
-  if (!p->dct_images && cudaMalloc((void**)&p->dct_images, (size_t)12 * TILE_BYTES) != cudaSuccess) return false;
-  const int kf = TILE_ROWS / n;
-  const bool seq = axis == 2;
-  std::vector<__nv_bfloat16> img((size_t)TILE_BYTES);          // hi and lo: 2 x 16384 elements
-  __nv_bfloat16* hi_img = img.data();
-  __nv_bfloat16* lo_img = img.data() + TILE_ROWS * TILE_ROWS;
-  for (int j = 0; j < TILE_ROWS; ++j)
-    for (int r = 0; r < TILE_ROWS; ++r) {
-      float v;
-      if (seq) v = (j / n == r / n) ? mat[(j % n) * n + (r % n)] : 0.f;
-      else v = (j % kf == r % kf) ? mat[(j / kf) * n + (r / kf)] : 0.f;
-      const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-      const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-      const int half = r >> 6, rk = r & 63;
-      const size_t off = (size_t)half * HALF_BYTES + (size_t)j * 128 + ((((rk >> 3) ^ (j & 7)) << 4) | ((rk & 7) << 1));
-      hi_img[off / 2] = hi;
-      lo_img[off / 2] = lo;
-    }
-  const int slot = (inverse ? 3 : 0) + axis;
-  return cudaMemcpy(p->dct_images + (size_t)2 * slot * TILE_BYTES, img.data(), 2 * TILE_BYTES, cudaMemcpyHostToDevice) == cudaSuccess;
+// The matrix of axis `axis` (0 = t, 1 = h, 2 = w), forward or inverse, as the tensor-memory operand image the
+// plan holds (built at plan creation by ffk_dct2_build_image: w lines follow one another, A = I kron Mat;
+// h and t lines interleave, A = Mat kron I).
+static const uint32_t* matrix_image(const ff_plan* p, int axis, int inverse) {
+  return p->dct2_images + (size_t)((inverse ? 3 : 0) + axis) * 2 * TILE_ROWS * IMG_CELLS;
 }
 
 // Scratch: two hi/lo pairs of bf16 grids for `group` tensor-heads.
@@ -600,19 +589,19 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
       e = ffk_dct2_forward(p, Q, K, V, g0, g, sc.a_hi, sc.a_lo, st);
       if (e != cudaSuccess) return e;
       P.in_split = 1;
-      P.mode = MODE_SPLIT; P.axis = last_axis; P.n = last_n; P.image = p->dct_images + (size_t)(2 * last_axis + 0) * TILE_BYTES;
+      P.mode = MODE_SPLIT; P.axis = last_axis; P.n = last_n; P.image = matrix_image(p, last_axis, 0);
       e = launch_pass(p, m3h, m3l, m3l, m3h, m3l, P, st);    // (no tensor stores in this mode)
       if (e != cudaSuccess) return e;
       continue;
     }
-    P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 2 + 0) * TILE_BYTES;
+    P.mode = MODE_FIRST; P.in_split = 0; P.axis = 2; P.n = dm.W; P.image = matrix_image(p, 2, 0);
     e = launch_pass(p, mq, mk, mv, o0h, o0l, P, st);
     if (e != cudaSuccess) return e;
-    P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 1 + 0) * TILE_BYTES;
+    P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = matrix_image(p, 1, 0);
     e = launch_pass(p, m1h, m1l, m1l, o1h, o1l, P, st);
     if (e != cudaSuccess) return e;
     P.in_split = 1;
-    P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.image = p->dct_images + (size_t)(2 * 0 + 0) * TILE_BYTES;
+    P.mode = MODE_SPLIT; P.axis = 0; P.n = dm.T; P.image = matrix_image(p, 0, 0);
     e = launch_pass(p, m2h, m2l, m2l, m2h, m2l, P, st);    // (no tensor stores in this mode)
     if (e != cudaSuccess) return e;
   }
@@ -646,13 +635,13 @@ cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaS
   DctTcParams P{};
   P.dm = dm; P.status = p->buf.status; P.group = g; P.group_start = h0;
   P.mode = MODE_MIDDLE; P.in_split = 1; P.axis = first_axis; P.n = first_n;
-  P.image = p->dct_images + (size_t)(2 * (3 + first_axis) + 0) * TILE_BYTES;
+  P.image = matrix_image(p, first_axis, 1);
   cudaError_t e = launch_pass(p, m_in, m_inl, m_inl, obh, obl, P, st);
   if (e != cudaSuccess) return e;
   if (fused) return ffk_dct2_inverse(p, sc.b_hi, sc.b_lo, h0, g, out, st);
-  P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = p->dct_images + (size_t)(2 * 4 + 0) * TILE_BYTES;
+  P.in_split = 1; P.axis = 1; P.n = dm.H; P.image = matrix_image(p, 1, 1);
   e = launch_pass(p, mbh, mbl, mbl, oah, oal, P, st);
   if (e != cudaSuccess) return e;
-  P.mode = MODE_LAST; P.axis = 2; P.n = dm.W; P.image = p->dct_images + (size_t)(2 * 5 + 0) * TILE_BYTES;
+  P.mode = MODE_LAST; P.axis = 2; P.n = dm.W; P.image = matrix_image(p, 2, 1);
   return launch_pass(p, mah, mal, mal, mout, mout, P, st);
 }

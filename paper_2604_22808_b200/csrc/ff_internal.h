@@ -115,8 +115,7 @@ struct ff_plan {
   bool xtc_ok;                                 // tensor-core exchange usable
   int* pos_table;                              // rank -> flat coefficient index of the mid, then the high band (plan-owned)
   alignas(64) unsigned char tmap_x[4][128];    // CUtensorMaps of the exchange kernel (Y / V~ of the mid and high bands)
-  uint8_t* dct_images;                         // 6 x (hi, lo) matrix images of the tensor-core transform (plan-owned)
-  uint32_t* dct2_images;                       // the same matrices as tensor-memory operands of the fused two-axis launch
+  uint32_t* dct2_images;                       // 6 x (hi, lo) transform matrices as tensor-memory operand images (plan-owned)
   bool dct2_ok;                                // the fused two-axis launch covers this configuration
   int dct2_axis2;                              // its second axis (1 = h, 0 = t); the remaining axis gets a pass of its own
   int dct2_clusters;                           // clusters of that launch the device runs at once (0 = not yet asked)
@@ -161,7 +160,6 @@ bool ffk_exchange_tc_prepare(ff_plan* p);
 cudaError_t ffk_exchange_tc(ff_plan* p, int h0, int g, void* grid_hi, void* grid_lo, cudaStream_t st);
 // ---- tensor-core transform (ff_dct_tc.cu) --------------------------------------------------------
 bool ffk_dct_tc_supported(const FFDims& dm);
-bool ffk_dct_tc_build_image(ff_plan* p, int axis, int inverse, const float* mat_host, int n);
 size_t ffk_dct_tc_scratch_bytes(const FFDims& dm, int group);
 cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, const void* V, bool want_energy,
                                      cudaStream_t st);
