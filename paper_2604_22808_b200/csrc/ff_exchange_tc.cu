@@ -52,6 +52,15 @@ struct XParams {
   int* status;
 };
 
+#ifdef FF_X_PROF
+__device__ unsigned long long g_x_prof[16];
+#define XPROF_T0(v) const long long v = clock64()
+#define XPROF_ADD(i, v) atomicAdd(&g_x_prof[i], (unsigned long long)(clock64() - (v)))
+#else
+#define XPROF_T0(v)
+#define XPROF_ADD(i, v)
+#endif
+
 constexpr int X_STG_PITCH = 64;         // bytes per staged row piece (32 channels)
 
 struct XShared {
@@ -132,7 +141,9 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         const CUtensorMap* map = x.band == 1 ? (exec ? &map_y_mid : &map_v_mid) : (exec ? &map_y_high : &map_v_high);
         const int slice = exec ? x.bh : 2 * dm.BH + x.bh;
         const int slot = n % YB;
+        XPROF_T0(x0);
         if (n >= YB) ok = mbar_wait(&sh.y_empty[slot], ((n / YB) - 1) & 1, abort_flag);
+        XPROF_ADD(0, x0);
         if (!ok) break;
         mbar_arrive_expect_tx(&sh.y_full[slot], XT * XD * 2);
         tma_load_3d(sY + slot * X_TILE_BYTES, map, &sh.y_full[slot], 0, x.tile * XT, slice);
@@ -150,11 +161,15 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       for (int it = it0; it < it1 && ok; ++it, ++n) {
         const XItem x = x_decode(dm, P.h0, it, tm_tiles, th_tiles);
         if (x.bh != prev_bh) {                            // the softmax warps re-staged Z for this head
+          XPROF_T0(x4);
           ok = mbar_wait(&sh.z_ready, zc & 1, abort_flag); ++zc; prev_bh = x.bh;
+          XPROF_ADD(4, x4);
           if (!ok) break;
         }
         const int slot = n % YB;
+        XPROF_T0(x1);
         ok = mbar_wait(&sh.y_full[slot], (n / YB) & 1, abort_flag);
+        XPROF_ADD(1, x1);
         if (!ok) break;
         tc_fence_after();
         const uint32_t ybase = smem_u32(sY + slot * X_TILE_BYTES);
@@ -167,8 +182,12 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         }
         umma_commit(&sh.s_full);
         if (YB == 1) umma_commit(&sh.y_empty[slot]);      // single buffer: free for the next load once the scores are done
+        XPROF_T0(x2);
         ok = mbar_wait(&sh.p_full, n & 1, abort_flag);
+        XPROF_ADD(2, x2);
+        XPROF_T0(x3);
         if (ok && n >= 1) ok = mbar_wait(&sh.d_empty, (n - 1) & 1, abort_flag);
+        XPROF_ADD(3, x3);
         if (!ok) break;
         tc_fence_after();
         for (int k = 0; k < nk / 16; ++k) {               // D = (Phi + Plo) (Zhi + Zlo) without lo*lo, K = keys
@@ -188,6 +207,20 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
     const int tid = row;                                  // 0..127 among the softmax threads
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const float sl2 = rsqrtf((float)XD) * 1.4426950408889634f;
+    // Keys a token attends to, as bit masks per 32-key chunk and band: the 3m summaries without the token's own
+    // band's and without those of an empty mid band.
+    uint32_t keys_mid[NK32], keys_high[NK32];
+#pragma unroll
+    for (int c3 = 0; c3 < NK32; ++c3) {
+      uint32_t a = 0, b = 0;
+      for (int i = 0; i < 32; ++i) {
+        const int j = c3 * 32 + i;
+        const bool live = j < 3 * m && !(dm.Nmid == 0 && j >= m && j < 2 * m);
+        if (live && (j < m || j >= 2 * m)) a |= 1u << i;
+        if (live && j < 2 * m) b |= 1u << i;
+      }
+      keys_mid[c3] = a; keys_high[c3] = b;
+    }
     bool ok = true;
     int n = 0, prev_bh = -1;
     for (int it = it0; it < it1 && ok; ++it, ++n) {
@@ -197,10 +230,13 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         // 64 channels per 128-byte row, 16-byte chunks XOR-swizzled with the row.  Rows >= 3m are zero.
         // The MMAs of the previous tile, which read the old images, must have completed.
         prev_bh = x.bh;
+        XPROF_T0(x8);
         if (n >= 1) {
           ok = __all_sync(0xffffffffu, mbar_wait(&sh.d_full, (n - 1) & 1, abort_flag));
           if (!ok) break;
         }
+        if (tid == 0) XPROF_ADD(8, x8);
+        XPROF_T0(x5);
         const float* S = P.summary + (size_t)x.bh * 3 * m * XD;
         for (int idx = tid; idx < nk * XD; idx += 128) {
           const int j = idx / XD, c = idx % XD;
@@ -214,13 +250,18 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         }
         fence_proxy_async();
         mbar_arrive(&sh.z_ready);
+        if (tid == 0) XPROF_ADD(5, x5);
       }
       // ---- softmax over the 2m summaries of the other bands
+      XPROF_T0(x6);
       ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full, n & 1, abort_flag));
+      if (tid == 0) XPROF_ADD(6, x6);
       if (!ok) break;
+      XPROF_T0(x7);
       tc_fence_after();
-      const int own0 = x.band * m, own1 = own0 + m;       // this band's own summaries are not attended
-      const int emp0 = dm.Nmid == 0 ? m : -1, emp1 = dm.Nmid == 0 ? 2 * m : -1;   // nor are those of an empty mid band
+      uint32_t keys[NK32];
+#pragma unroll
+      for (int c3 = 0; c3 < NK32; ++c3) keys[c3] = x.band == 1 ? keys_mid[c3] : keys_high[c3];
       if (NK32 >= 2) {
         // first sweep: the row maximum
         float mx = -INFINITY;
@@ -231,8 +272,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
           tmem_wait_ld();
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            const int j = c3 * 32 + i;
-            if (j < 3 * m && (j < own0 || j >= own1) && (j < emp0 || j >= emp1)) mx = fmaxf(mx, __uint_as_float(r[i]));
+            if (keys[c3] & (1u << i)) mx = fmaxf(mx, __uint_as_float(r[i]));
           }
         }
         const float mb = mx * sl2;
@@ -246,10 +286,9 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
           uint32_t ph[16], pl[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const int j = c3 * 32 + 2 * i;
             float p0 = 0.f, p1 = 0.f;
-            if (j < 3 * m && (j < own0 || j >= own1) && (j < emp0 || j >= emp1)) p0 = ex2f_approx(fmaf(__uint_as_float(r[2 * i]), sl2, -mb));
-            if (j + 1 < 3 * m && (j + 1 < own0 || j + 1 >= own1) && (j + 1 < emp0 || j + 1 >= emp1)) p1 = ex2f_approx(fmaf(__uint_as_float(r[2 * i + 1]), sl2, -mb));
+            if (keys[c3] & (1u << (2 * i))) p0 = ex2f_approx(fmaf(__uint_as_float(r[2 * i]), sl2, -mb));
+            if (keys[c3] & (2u << (2 * i))) p1 = ex2f_approx(fmaf(__uint_as_float(r[2 * i + 1]), sl2, -mb));
             den0 += p0; den1 += p1;
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
             ph[i] = *(const uint32_t*)&h2;
@@ -274,13 +313,13 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int j = 0; j < NK32 * 32; ++j)
-          if (j < 3 * m && (j < own0 || j >= own1) && (j < emp0 || j >= emp1)) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(sc[j]));
+          if (keys[j >> 5] & (1u << (j & 31))) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(sc[j]));
         const float mb = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
         float den4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < NK32 * 32; ++j) {
           float pv = 0.f;
-          if (j < 3 * m && (j < own0 || j >= own1) && (j < emp0 || j >= emp1)) pv = ex2f_approx(fmaf(__uint_as_float(sc[j]), sl2, -mb));
+          if (keys[j >> 5] & (1u << (j & 31))) pv = ex2f_approx(fmaf(__uint_as_float(sc[j]), sl2, -mb));
           den4[j & 3] += pv;
           sc[j] = __float_as_uint(pv);
         }
@@ -305,6 +344,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&sh.p_full);
+      if (tid == 0) XPROF_ADD(7, x7);
     }
   } else {
     // ------------------------------------------------------------------ store warps
@@ -319,10 +359,14 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       const long long n_band = x.band == 1 ? dm.Nmid : dm.Nhigh;
       const long long p = (long long)x.tile * XT + row;
       // ---- residual add and store
+      XPROF_T0(x9);
       ok = __all_sync(0xffffffffu, mbar_wait(&sh.d_full, n & 1, abort_flag));
+      if (row == 0) XPROF_ADD(9, x9);
       if (!ok) break;
+      XPROF_T0(x10);
       tc_fence_after();
       const bool valid = p < n_band;
+      XPROF_T0(x14);
       int f = valid ? (x.band == 1 ? P.pos_mid[p] : P.pos_high[p]) : -1;
       if (valid && !FF_DBG_OK(f >= 0 && f < dm.N && x.bh >= P.h0 && x.bh < P.h0 + P.g, P.status, 3)) f = -1;   // (debug build)
       // lane L stores for rows 8 i + L/4 of its warp: fetch those rows' grid positions
@@ -338,11 +382,15 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       const float dscale = NK32 >= 2 ? sh.inv[n & 1][row] : 1.f;    // (two-sweep variants: P was left unnormalised)
       uint8_t* st_hi = sh.stage[quarter][0];
       uint8_t* st_lo = sh.stage[quarter][1];
+      if (row == 0) XPROF_ADD(14, x14);
 #pragma unroll
       for (int q = 0; q < XD / 32; ++q) {
         uint32_t r[32];
+        XPROF_T0(x11);
         tmem_ld32(tmem + lane_addr + 128 + q * 32, r);
         tmem_wait_ld();
+        if (row == 0) XPROF_ADD(11, x11);
+        XPROF_T0(x12);
 #pragma unroll
         for (int v4 = 0; v4 < 4; ++v4) {
           // channels 32q + 8v4 .. +7 of this token: one 16-byte chunk of the swizzled Y tile
@@ -365,6 +413,8 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
           *(uint4*)(st_lo + so) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         }
         __syncwarp();
+        if (row == 0) XPROF_ADD(12, x12);
+        XPROF_T0(x13);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int rr = 8 * i + (lane >> 2), piece = lane & 3;      // row of the warp, 16-byte piece of its 64 bytes
@@ -376,10 +426,12 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
           }
         }
         __syncwarp();
+        if (row == 0) XPROF_ADD(13, x13);
       }
       tc_fence_before();
       mbar_arrive(&sh.d_empty);
       if (YB > 1) mbar_arrive(&sh.y_empty[slot]);
+      if (row == 0) XPROF_ADD(10, x10);
     }
   }
 
@@ -417,6 +469,14 @@ bool encode_rows_map(CUtensorMap* map, void* base, long long rows, int slices, i
 }
 
 }  // namespace
+
+#ifdef FF_X_PROF
+extern "C" void ff_debug_x_prof(unsigned long long* out16, int reset) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(out16, g_x_prof, sizeof(unsigned long long) * 16);
+  if (reset) { unsigned long long z[16] = {}; cudaMemcpyToSymbol(g_x_prof, z, sizeof(z)); }
+}
+#endif
 
 bool ffk_exchange_tc_supported(const FFDims& dm) {
   return !dm.fp32 && (dm.d == 128 || dm.d == 64) && dm.m >= 1 && dm.m <= 32 && dm.N < (1LL << 31);

@@ -88,6 +88,7 @@ struct FFLayout {
   size_t total;
   int group;         // G: tensor-heads processed per generic transform launch
   int tc_group;      // tensor-heads per tensor-core transform launch
+  int tc_group_pipe; // ... when the launches are pipelined with host copies (host-buffer entry point)
 };
 
 constexpr int FF_COPY_EVENTS = 64;

@@ -143,7 +143,7 @@ def test_paper_reference_1m_full():
 
 def test_host_buffer_entry_point_64k_matches_device_path():
     """Bench configuration of the end-to-end number: three copy groups in, one out; the result equals
-    the device-resident call's up to the last bits of the atomically accumulated summaries."""
+    the device-resident call's up to the last bits of the atomically accumulated summaries (one bf16 step of an output)."""
     import torch
     from paper_2604_22808_b200 import binding as B
     cfg = C.G64K
@@ -160,6 +160,9 @@ def test_host_buffer_entry_point_64k_matches_device_path():
         oh.zero_()
         plan.forward_host(qh, kh, vh, oh, timesteps=ts)
         assert plan.device_status() == 0
-        diff = (oh.float() - out.cpu().float()).abs()
-        assert diff.max().item() <= 2e-2 and diff.mean().item() <= 1e-4
+        ref = out.cpu().float()
+        diff = (oh.float() - ref).abs()
+        # (two runs of either entry point differ the same way: a last-bit change of a summary moves a few outputs
+        # to the neighbouring bf16 value, one step = at most 2^-7 of the value)
+        assert bool((diff <= torch.clamp(ref.abs() * 2.0 ** -7, min=2e-2)).all()) and diff.mean().item() <= 1e-4
     plan.destroy()
