@@ -755,7 +755,7 @@ cudaError_t ffk_forward_transform_tc(ff_plan* p, const void* Q, const void* K, c
   return cudaSuccess;
 }
 
-// Inverse transform of `g` recombined grids (bf16 hi/lo pair in the first scratch pair, written by the
+// Inverse transform of `g` recombined grids (three-byte form in the first scratch pair, written by the
 // exchange) into out[h0 .. h0+g).
 cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaStream_t st) {
   const FFDims& dm = p->dm;
@@ -764,12 +764,12 @@ cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaS
   const bool fused = p->dct2_ok && !(p->attn_impl & 4);
   const int first_axis = fused ? (p->dct2_axis2 == 1 ? 0 : 1) : 0;       // the axis the fused launch leaves out
   const int first_n = first_axis == 0 ? dm.T : dm.H;
-  // The first pass reads the exchange's bf16 pair.  With three passes the pairs between them have the three-byte
-  // form; the fused launch takes a bf16 pair.
+  // The first pass reads the exchange's output, which has the three-byte form.  With three passes the pairs
+  // between them have it too; the fused launch takes a bf16 pair.
   const bool b8 = !fused;
   const bool inv8 = true;
   CUtensorMap m_in, m_inl, mbh, mbl, mah, mal, obh, obl, oah, oal, mout;
-  if (!encode_grid_map(&m_in, sc.a_hi, dm, G, first_axis) || !encode_grid_map(&m_inl, sc.a_lo, dm, G, first_axis) ||
+  if (!encode_grid_map(&m_in, sc.a_hi, dm, G, first_axis) || !encode_grid_map(&m_inl, sc.a_lo, dm, G, first_axis, true) ||
       !encode_grid_map(&mbh, sc.b_hi, dm, G, 1) ||
       !encode_grid_map(&mbl, sc.b_lo, dm, G, 1, true) || !encode_grid_map(&mah, sc.a_hi, dm, G, 2) ||
       !encode_grid_map(&mal, sc.a_lo, dm, G, 2, inv8) || !encode_store_map(&obh, sc.b_hi, dm, G, first_axis) ||
@@ -780,7 +780,7 @@ cudaError_t ffk_inverse_transform_tc(ff_plan* p, int h0, int g, void* out, cudaS
   P.dm = dm; P.status = p->buf.status; P.group = g; P.group_start = h0;
   P.mode = MODE_MIDDLE; P.in_split = 1; P.out_lo8 = b8 ? 1 : 0; P.reverse = 1; P.axis = first_axis; P.n = first_n;
   P.image = matrix_image(p, first_axis, 1);
-  cudaError_t e = launch_pass(p, m_in, m_inl, m_inl, obh, obl, P, false, st);
+  cudaError_t e = launch_pass(p, m_in, m_inl, m_inl, obh, obl, P, true, st);
   if (e != cudaSuccess) return e;
   if (fused) return ffk_dct2_inverse(p, sc.b_hi, sc.b_lo, h0, g, out, st);
   P.in_split = 1; P.out_lo8 = inv8 ? 1 : 0; P.reverse = 0; P.axis = 1; P.n = dm.H; P.image = matrix_image(p, 1, 1);

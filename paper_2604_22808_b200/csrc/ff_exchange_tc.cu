@@ -13,8 +13,9 @@
 //   softmax one token per thread (row = TMEM lane); P written back to TMEM as bf16 hi + lo (normalised
 //           for up to 32 keys, otherwise unnormalised with the row sum handed to the store warps)
 //   MMA 2   D[128 x 128] = P Z  (A = P from tensor memory, B = the same Z image read MN-major)
-//   store   Y + D as a bf16 hi/lo pair; a thread owns a token, the warp stages 32 channels of its 32
-//           tokens in shared memory and four lanes then write a token's 64 contiguous bytes
+//   store   Y + D in the three-byte form the inverse passes read (the value rounded to 24 bits: a grid of its
+//           upper 16 bits and a grid of the next byte); a thread owns a token, the warp stages 32 channels of
+//           its 32 tokens in shared memory and four lanes then write a token's 64 + 32 contiguous bytes
 // Z and P are split into bf16 hi + lo parts (Y is exact bf16), so the logits and the update carry
 // about 16 bits: the summary logits of a band with large low-frequency content reach O(100).
 // The low band (fp32, a few hundred tokens) is handled by the generic kernel.
@@ -39,8 +40,8 @@ struct XParams {
   const float* summary;       // [BH][3][m][d]
   const int* pos_mid;         // [N_mid]  flat coefficient index of each band rank
   const int* pos_high;        // [N_high]
-  __nv_bfloat16* grid_hi;     // [g][N][d]
-  __nv_bfloat16* grid_lo;
+  __nv_bfloat16* grid_hi;     // [g][N][d]: upper 16 bits of the value rounded to 24 bits
+  uint8_t* grid_lo;           // [g][N][d]: the next 8 bits (the three-byte form the inverse passes read)
   int h0, g;                  // heads [h0, h0+g)
   int nkeys;                  // 3m rounded up to a multiple of 16
   int ybufs;                  // token-tile buffers in shared memory (1 or 2)
@@ -358,13 +359,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       const int slot = n % YB;
       const long long n_band = x.band == 1 ? dm.Nmid : dm.Nhigh;
       const long long p = (long long)x.tile * XT + row;
-      // ---- residual add and store
-      XPROF_T0(x9);
-      ok = __all_sync(0xffffffffu, mbar_wait(&sh.d_full, n & 1, abort_flag));
-      if (row == 0) XPROF_ADD(9, x9);
-      if (!ok) break;
-      XPROF_T0(x10);
-      tc_fence_after();
+      // ---- residual add and store (where the rows go does not depend on the data: looked up before the wait)
       const bool valid = p < n_band;
       XPROF_T0(x14);
       int f = valid ? (x.band == 1 ? P.pos_mid[p] : P.pos_high[p]) : -1;
@@ -379,10 +374,16 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
       const bool exec_g = P.alloc[x.bh] & (1 << x.band);
       const __nv_bfloat16* grow = P.src[(x.band == 1 ? 0 : 2) + (exec_g ? 0 : 1)] +
                                   ((size_t)(exec_g ? x.bh : 2 * dm.BH + x.bh) * n_band + (valid ? p : 0)) * XD;
-      const float dscale = NK32 >= 2 ? sh.inv[n & 1][row] : 1.f;    // (two-sweep variants: P was left unnormalised)
       uint8_t* st_hi = sh.stage[quarter][0];
       uint8_t* st_lo = sh.stage[quarter][1];
       if (row == 0) XPROF_ADD(14, x14);
+      XPROF_T0(x9);
+      ok = __all_sync(0xffffffffu, mbar_wait(&sh.d_full, n & 1, abort_flag));
+      if (row == 0) XPROF_ADD(9, x9);
+      if (!ok) break;
+      XPROF_T0(x10);
+      tc_fence_after();
+      const float dscale = NK32 >= 2 ? sh.inv[n & 1][row] : 1.f;    // (two-sweep variants: P was left unnormalised)
 #pragma unroll
       for (int q = 0; q < XD / 32; ++q) {
         uint32_t r[32];
@@ -398,19 +399,19 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
           const uint4 yv = YB == 1 ? __ldg((const uint4*)(grow + cch * 8))
                                    : *(const uint4*)(yrow + (cch >> 3) * X_HALF + (((cch & 7) ^ (row & 7)) << 4));
           const uint32_t yw[4] = {yv.x, yv.y, yv.z, yv.w};
-          uint32_t hi[4], lo[4];
+          // three-byte form: the value rounded to 24 bits; hi = its upper 16 bits, lo = the next byte
+          uint32_t hi[4], u[8];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const float v0 = fmaf(__uint_as_float(r[v4 * 8 + 2 * i]), dscale, __uint_as_float(yw[i] << 16));
-            const float v1 = fmaf(__uint_as_float(r[v4 * 8 + 2 * i + 1]), dscale, __uint_as_float(yw[i] & 0xffff0000u));
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
-            hi[i] = *(const uint32_t*)&h2;
-            const __nv_bfloat162 l2 = __floats2bfloat162_rn(v0 - __uint_as_float(hi[i] << 16), v1 - __uint_as_float(hi[i] & 0xffff0000u));
-            lo[i] = *(const uint32_t*)&l2;
+            u[2 * i] = __float_as_uint(fmaf(__uint_as_float(r[v4 * 8 + 2 * i]), dscale, __uint_as_float(yw[i] << 16))) + 0x80u;
+            u[2 * i + 1] = __float_as_uint(fmaf(__uint_as_float(r[v4 * 8 + 2 * i + 1]), dscale, __uint_as_float(yw[i] & 0xffff0000u))) + 0x80u;
+            hi[i] = __byte_perm(u[2 * i], u[2 * i + 1], 0x7632);
           }
-          const int so = lane * X_STG_PITCH + ((v4 ^ ((lane >> 1) & 3)) << 4);
-          *(uint4*)(st_hi + so) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *(uint4*)(st_lo + so) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          const uint32_t lo0 = __byte_perm(__byte_perm(u[0], u[1], 0x0051), __byte_perm(u[2], u[3], 0x0051), 0x5410);
+          const uint32_t lo1 = __byte_perm(__byte_perm(u[4], u[5], 0x0051), __byte_perm(u[6], u[7], 0x0051), 0x5410);
+          *(uint4*)(st_hi + lane * X_STG_PITCH + ((v4 ^ ((lane >> 1) & 3)) << 4)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          // (lo: 32 bytes per row, 8-byte pieces XOR-swizzled with row / 4)
+          *(uint2*)(st_lo + lane * 32 + ((v4 ^ ((lane >> 2) & 3)) << 3)) = make_uint2(lo0, lo1);
         }
         __syncwarp();
         if (row == 0) XPROF_ADD(12, x12);
@@ -422,7 +423,7 @@ exchange_tc_kernel(const __grid_constant__ CUtensorMap map_y_mid, const __grid_c
             const size_t o = obase + (size_t)fpos[i] * XD + q * 32 + piece * 8;
             const int so = rr * X_STG_PITCH + ((piece ^ ((rr >> 1) & 3)) << 4);
             *(uint4*)(P.grid_hi + o) = *(const uint4*)(st_hi + so);
-            *(uint4*)(P.grid_lo + o) = *(const uint4*)(st_lo + so);
+            *(uint2*)(P.grid_lo + o) = *(const uint2*)(st_lo + rr * 32 + ((piece ^ ((rr >> 2) & 3)) << 3));
           }
         }
         __syncwarp();
@@ -518,7 +519,7 @@ cudaError_t ffk_exchange_tc(ff_plan* p, int h0, int g, void* grid_hi, void* grid
   XParams P;
   P.dm = dm; P.alloc = p->buf.alloc; P.summary = p->buf.summary;
   P.pos_mid = p->pos_table; P.pos_high = p->pos_table + dm.Nmid;
-  P.grid_hi = (__nv_bfloat16*)grid_hi; P.grid_lo = (__nv_bfloat16*)grid_lo;
+  P.grid_hi = (__nv_bfloat16*)grid_hi; P.grid_lo = (uint8_t*)grid_lo;
   P.h0 = h0; P.g = g; P.nkeys = (3 * dm.m + 15) / 16 * 16; P.status = p->buf.status;
   P.src[0] = (const __nv_bfloat16*)p->buf.y_mid; P.src[1] = (const __nv_bfloat16*)p->buf.spec_mid;
   P.src[2] = (const __nv_bfloat16*)p->buf.y_high; P.src[3] = (const __nv_bfloat16*)p->buf.spec_high;

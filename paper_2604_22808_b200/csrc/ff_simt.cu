@@ -487,7 +487,7 @@ static int exc_rounds(long long tokens, int g, int sm_count) {
 
 template <typename ST, int DPL, typename OT>
 __global__ void __launch_bounds__(EXC_WARPS * 32) exchange_recombine_kernel(FFBuffers buf, FFDims dm, int bh0,
-                                                                             OT* grid_out, OT* grid_lo, int low_only, int rounds) {
+                                                                             OT* grid_out, void* grid_lo, int low_only, int rounds) {
   extern __shared__ float S[];   // [3][m][d]
   const int gi = blockIdx.y, bh = bh0 + gi;
   const int d = dm.d, m = dm.m;
@@ -539,15 +539,21 @@ __global__ void __launch_bounds__(EXC_WARPS * 32) exchange_recombine_kernel(FFBu
 #pragma unroll
     for (int j = 0; j < DPL; ++j) acc[j] /= den;
   }
-  // With a second grid the value is stored as a hi/lo pair (hi = rounded value, lo = rounded
-  // remainder): a band's tokens share almost the same exchange offset, so a single rounding would
-  // bias whole bands coherently and the inverse transform would focus that bias on a few tokens.
+  // With a second grid (bf16 output) the value is stored in three bytes, rounded to 24 bits: its upper 16 bits
+  // in grid_out, the next 8 bits in the byte grid.  A band's tokens share almost the same exchange offset, so a
+  // single bf16 rounding would bias whole bands coherently and the inverse transform would focus that bias on a
+  // few tokens.
   OT* dst = grid_out + ((size_t)gi * dm.N + f) * d;
 #pragma unroll
   for (int j = 0; j < DPL; ++j) {
     const float v = y[j] + acc[j];
-    stf<OT>(dst + lane + 32 * j, v);
-    if (grid_lo) stf<OT>(grid_lo + ((size_t)gi * dm.N + f) * d + lane + 32 * j, v - ldf<OT>(dst + lane + 32 * j));
+    if (grid_lo) {
+      const uint32_t u = __float_as_uint(v) + 0x80u;
+      ((uint16_t*)dst)[lane + 32 * j] = (uint16_t)(u >> 16);
+      ((uint8_t*)grid_lo)[((size_t)gi * dm.N + f) * d + lane + 32 * j] = (uint8_t)(u >> 8);
+    } else {
+      stf<OT>(dst + lane + 32 * j, v);
+    }
   }
   }
 }
