@@ -32,7 +32,7 @@ METRIC = "freqformer_attn_layer_tokens_per_s"
 # capture of the 6-head 64K case (forward: the passes over Q, K and V; inverse: the passes over one tensor).
 FP32_FMA_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 74.5: plain fp32 FMA rate of the GPU (unit counts x max clock)
 # [0]: three separate axis passes; [1]: two axes in one launch (64K-class grids)
-NCU_DRAM_BYTES_PER_TOKEN_HEAD = {"transform": (7330.0, 4359.0), "inverse": (3110.0, 2203.0)}
+NCU_DRAM_BYTES_PER_TOKEN_HEAD = {"transform": (6554.0, 4380.0), "inverse": (2345.0, 1985.0)}
 TRANSFORM_KERNELS = {"transform": ("dct_tc_kernel x3 (transform stage)", "dct2_tc_kernel + dct_tc_kernel (transform stage)"),
                      "inverse": ("exchange_tc_kernel + dct_tc_kernel x3 (inverse stage)",
                                  "exchange_tc_kernel + dct_tc_kernel + dct2_tc_kernel (inverse stage)")}
