@@ -676,6 +676,97 @@ cudaError_t ffk_summaries(ff_plan* p, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+__device__ __forceinline__ float exp2f_fast(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Low band of the tensor-core inverse ("Cross-band residual exchange", "Reconstruction"): exchange + recombination
+// of the low band's coefficients into the three-byte grids.  One warp per SOURCE row: a head that executes the
+// low band has one pooled output row for every r consecutive coefficient ranks, so its update is computed once
+// and written r times; other heads carry V~ low, one row per rank.  The scores of eight summaries at a time
+// are reduced side by side (independent shuffle trees) and merged into the running softmax as a group
+// (exponentials by ex2.approx on scores scaled to log2 units, like the tensor-core kernel's).  DPL = d / 32.
+template <int DPL>
+__global__ void __launch_bounds__(EXC_WARPS * 32) exchange_low_kernel(FFBuffers buf, FFDims dm, int bh0, __nv_bfloat16* grid_hi,
+                                                                       uint8_t* grid_lo, int rounds) {
+  extern __shared__ float S[];   // [3][m][d]
+  const int gi = blockIdx.y, bh = bh0 + gi;
+  const int d = dm.d, m = dm.m;
+  for (int i = threadIdx.x; i < 3 * m * d; i += blockDim.x) S[i] = buf.summary[(size_t)bh * 3 * m * d + i];
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  const bool exec = buf.alloc[bh] & FF_BAND_LOW;
+  const float* src = exec ? buf.y_low + (size_t)bh * dm.Nbar * d : buf.spec_low + ((size_t)2 * dm.BH + bh) * dm.Nlow * d;
+  const long long rows = exec ? dm.Nbar : dm.Nlow;
+  const int rep = exec ? dm.r : 1;
+  // the summaries of the other bands: the mid band's (none if it is empty), then the high band's
+  const int k_first = dm.Nmid == 0 ? 2 * m : m, nkeys = 3 * m - k_first;
+  const float scale = rsqrtf((float)d) * 1.4426950408889634f;      // scores in units of log2: exponentials by ex2
+  for (int round = 0; round < rounds; ++round) {
+    const long long row = ((long long)blockIdx.x * rounds + round) * EXC_WARPS + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    float y[DPL], acc[DPL];
+#pragma unroll
+    for (int j = 0; j < DPL; ++j) { y[j] = src[(size_t)row * d + lane + 32 * j]; acc[j] = 0.f; }
+    if (nkeys > 0) {
+      float mx = -INFINITY, den = 0.f;
+      for (int k0 = 0; k0 < nkeys; k0 += 8) {
+        float sc[8];
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const float* z = S + (size_t)(k_first + (k0 + kk < nkeys ? k0 + kk : 0)) * d;
+          float part = 0.f;
+#pragma unroll
+          for (int j = 0; j < DPL; ++j) part = fmaf(y[j], z[lane + 32 * j], part);
+          sc[kk] = part;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) sc[kk] += __shfl_xor_sync(0xffffffffu, sc[kk], o);
+        float nm = mx;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          sc[kk] = k0 + kk < nkeys ? sc[kk] * scale : -INFINITY;
+          nm = fmaxf(nm, sc[kk]);
+        }
+        const float corr = exp2f_fast(mx - nm);
+        den *= corr;
+#pragma unroll
+        for (int j = 0; j < DPL; ++j) acc[j] *= corr;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const float pr = exp2f_fast(sc[kk] - nm);         // (0 for the keys past the end)
+          const float* z = S + (size_t)(k_first + (k0 + kk < nkeys ? k0 + kk : 0)) * d;
+          den += pr;
+#pragma unroll
+          for (int j = 0; j < DPL; ++j) acc[j] = fmaf(pr, z[lane + 32 * j], acc[j]);
+        }
+        mx = nm;
+      }
+#pragma unroll
+      for (int j = 0; j < DPL; ++j) acc[j] /= den;
+    }
+    // the value in three bytes (rounded to 24 bits: upper 16 bits and the next 8), at every rank the row stands for
+    uint32_t u[DPL];
+#pragma unroll
+    for (int j = 0; j < DPL; ++j) u[j] = __float_as_uint(y[j] + acc[j]) + 0x80u;
+    for (int i = 0; i < rep; ++i) {
+      const long long p = row * rep + i;
+      if (p >= dm.Nlow) break;
+      const int kw = (int)(p % dm.L[2]), kh = (int)((p / dm.L[2]) % dm.L[1]), kt = (int)(p / ((long long)dm.L[2] * dm.L[1]));
+      const size_t o = ((size_t)gi * dm.N + ((size_t)kt * dm.H + kh) * dm.W + kw) * d;
+#pragma unroll
+      for (int j = 0; j < DPL; ++j) {
+        ((uint16_t*)grid_hi)[o + lane + 32 * j] = (uint16_t)(u[j] >> 16);
+        grid_lo[o + lane + 32 * j] = (uint8_t)(u[j] >> 8);
+      }
+    }
+  }
+}
+
 // Generic exchange + recombination into the hi/lo bf16 grids of the tensor-core inverse; DPL = d / 32.
 template <int DPL>
 static cudaError_t exchange_to_grids(ff_plan* p, long long tokens, int g, size_t smem, int h0, __nv_bfloat16* ghi,
@@ -702,8 +793,20 @@ static cudaError_t exchange_inverse_tc(ff_plan* p, void* out, cudaStream_t st) {
     __nv_bfloat16* ghi = (__nv_bfloat16*)p->buf.scratchA;
     __nv_bfloat16* glo = (__nv_bfloat16*)((char*)p->buf.scratchA + grid_bytes);
     if (p->xtc_ok) {
-      // mid and high bands on the tensor cores, the (small, fp32) low band with the generic kernel
-      e = dm.d == 128 ? exchange_to_grids<4>(p, dm.Nlow, g, smem, h0, ghi, glo, 1, st) : exchange_to_grids<2>(p, dm.Nlow, g, smem, h0, ghi, glo, 1, st);
+      // mid and high bands on the tensor cores, the fp32 low band with its own kernel (one warp per source row)
+      {
+        const int rounds = exc_rounds(dm.Nlow, g, p->sm_count);
+        const long long per_block = (long long)EXC_WARPS * rounds;
+        dim3 grid((unsigned)((dm.Nlow + per_block - 1) / per_block), (unsigned)g);
+        if (dm.d == 128) {
+          e = cudaFuncSetAttribute(exchange_low_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+          if (e == cudaSuccess) exchange_low_kernel<4><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, dm, h0, ghi, (uint8_t*)glo, rounds);
+        } else {
+          e = cudaFuncSetAttribute(exchange_low_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+          if (e == cudaSuccess) exchange_low_kernel<2><<<grid, EXC_WARPS * 32, smem, st>>>(p->buf, dm, h0, ghi, (uint8_t*)glo, rounds);
+        }
+        if (e == cudaSuccess) e = cudaGetLastError();
+      }
       if (e == cudaSuccess) e = ffk_exchange_tc(p, h0, g, ghi, glo, st);
     } else {
       e = dm.d == 128 ? exchange_to_grids<4>(p, dm.N, g, smem, h0, ghi, glo, 0, st) : exchange_to_grids<2>(p, dm.N, g, smem, h0, ghi, glo, 0, st);
