@@ -110,8 +110,8 @@ void ff_compute_layout(const FFDims& dm, bool with_staging, FFLayout* lay) {
   if (G > 3 * BH) G = 3 * BH;
   lay->group = (int)G;
   // Tensor-core transform: as many tensor-heads per launch as fit ~8 GiB of scratch (at least 3): every launch
-  // pays a ramp-up and a tail, and fewer, longer launches measured faster (64K tokens: one group of 48 against
-  // 32 + 16 tensor-heads, 1.58 against 1.66 ms for the forward transform).  The host-buffer entry point
+  // pays a ramp-up and a tail, and fewer, longer launches measured faster (64K tokens, 72 tensor-heads: one group against
+  // 32 + 32 + 8, 1.58 against 1.66 ms for the forward transform).  The host-buffer entry point
   // works in groups of a quarter of that, so that the transform of one group overlaps the copy of the next.
   size_t Gt = ((size_t)8 << 30) / (4 * (size_t)dm.N * d * 2);
   if (Gt < 3) Gt = 3;

@@ -80,6 +80,7 @@ struct D2Shared {
   // The plane buffer has one slot of 8 tiles or two of 4 (items alternate): phase 1 of the next item fills one
   // slot while phase 2 of the current item reads the other.
   uint64_t buf_full[2];    // all rows of the item have landed in this CTA's slot (arrivals from every CTA's warps)
+  uint64_t buf_half[2];    // (one CTA per plane) the rows of the first half of the second axis have landed
   uint64_t buf_free[2];    // every CTA of the cluster has finished reading the slot (phase 2 of the item)
   uint64_t mma2_done[2];   // this CTA's phase-2 instructions of the item (by slot) have completed
   uint32_t tmem_base;
@@ -225,12 +226,16 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   const int nsl = tpc <= MAX_TPC / 2 ? 2 : 1;                      // slots of the plane buffer
   const int bt = tpc < 4 ? tpc : 4;                                // tiles per instruction batch (N = 32 bt columns): an
   const int nb = tpc / bt;                                         // instruction costs the same for any N up to 128
+  // One CTA per plane and an even number of batches: the first half of the phase-1 batches holds the first half
+  // of the second axis, i.e. rows 0..63 of every phase-2 tile = its k-steps 0..3.  Phase 2 of the item's first
+  // batch starts on those while phase 1 still works on the second half.
+  const bool half_start = cs == 1 && nb >= 2 && (nb & 1) == 0;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NSTG; ++i) { mbar_init(&sh.in_full[i], 1); mbar_init(&sh.in_empty[i], 1); }
     for (int i = 0; i < NA1; ++i) { mbar_init(&sh.acc1_full[i], 1); mbar_init(&sh.acc1_empty[i], 256); }
     for (int i = 0; i < NA2; ++i) { mbar_init(&sh.acc2_full[i], 1); mbar_init(&sh.acc2_empty[i], 256); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sh.buf_full[i], 8 * cs); mbar_init(&sh.buf_free[i], cs); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.buf_full[i], 8 * cs); mbar_init(&sh.buf_free[i], cs); mbar_init(&sh.buf_half[i], 8); }
     mbar_init(&sh.mma2_done[0], 1); mbar_init(&sh.mma2_done[1], 1);
     sh.abort_flag = 0;
     fence_mbar_init();
@@ -363,7 +368,8 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         // the plane's rows have landed in this CTA's buffer
         PROF_T0(tm2);
         const int sl = (int)(ni % nsl);                             // the item's slot of the plane buffer
-        ok = mbar_wait_cluster(&sh.buf_full[sl], (ni / nsl) & 1, abort_flag);
+        ok = half_start ? mbar_wait(&sh.buf_half[sl], (ni / nsl) & 1, abort_flag)
+                        : mbar_wait_cluster(&sh.buf_full[sl], (ni / nsl) & 1, abort_flag);
         PROF_ADD(9, tm2);
         if (!ok) break;
         fence_proxy_async_all();
@@ -379,10 +385,19 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           const uint32_t d_tm = tm + COL_ACC2 + ab * 128;
 #pragma unroll
           for (int ks = 0; ks < ROWS / 16; ++ks) {
+            if (ks == ROWS / 32 && kb == 0 && half_start) {          // the second half of the rows
+              PROF_T0(tm4);
+              ok = mbar_wait_cluster(&sh.buf_full[sl], (ni / nsl) & 1, abort_flag);
+              PROF_ADD(11, tm4);
+              if (!ok) break;
+              fence_proxy_async_all();
+              tc_fence_after();
+            }
             umma_ts(d_tm, tm + COL_A2H + ks * 8, xh + (uint64_t)(ks * 64), idesc, ks > 0 ? 1u : 0u);
             umma_ts(d_tm, tm + COL_A2L + ks * 8, xh + (uint64_t)(ks * 64), idesc, 1u);
             umma_ts(d_tm, tm + COL_A2H + ks * 8, xl + (uint64_t)(ks * 64), idesc, 1u);
           }
+          if (!ok) break;
           umma_commit(&sh.acc2_full[ab]);
         }
         umma_commit(&sh.mma2_done[sl]);
@@ -484,6 +499,11 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         }
         }
         if (threadIdx.x == 128) PROF_ADD(2, te2);
+        if (half_start && kb == nb / 2 - 1) {               // this warp's rows of the first half are written
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh.buf_half[sl]);
+        }
       }
       if (!ok) break;
       // this warp's rows of the item are written: tell every CTA of the cluster

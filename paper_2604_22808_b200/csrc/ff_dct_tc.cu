@@ -496,15 +496,26 @@ dct_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ 
               // Router statistics: channel energies of the staged (bf16) coefficients, summed down the
               // columns of the warp's 32 x 32 block; a lane reads one channel pair of every other row.
               const int par = lane >> 4, cp = lane & 15;
-              const unsigned nl = nonlow_rows >> par, md = mid_rows >> par;
               float a0 = 0.f, a1 = 0.f, m0 = 0.f, m1 = 0.f;
+              if (nonlow_rows == 0xffffffffu && (mid_rows == 0u || mid_rows == 0xffffffffu)) {
+                // (almost every block: its 32 rows lie in one band, mid or high)
 #pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const uint32_t wd = *(const uint32_t*)(st_hi + (2 * i + par) * STG_PITCH + (((cp >> 2) ^ (i & 3)) << 4) + (cp & 3) * 4);
-                const float v0 = __uint_as_float(wd << 16), v1 = __uint_as_float(wd & 0xffff0000u);
-                const float s0 = v0 * v0, s1 = v1 * v1;
-                if ((nl >> (2 * i)) & 1) { a0 += s0; a1 += s1; }
-                if ((md >> (2 * i)) & 1) { m0 += s0; m1 += s1; }
+                for (int i = 0; i < 16; ++i) {
+                  const uint32_t wd = *(const uint32_t*)(st_hi + (2 * i + par) * STG_PITCH + (((cp >> 2) ^ (i & 3)) << 4) + (cp & 3) * 4);
+                  const float v0 = __uint_as_float(wd << 16), v1 = __uint_as_float(wd & 0xffff0000u);
+                  a0 = fmaf(v0, v0, a0); a1 = fmaf(v1, v1, a1);
+                }
+                if (mid_rows) { m0 = a0; m1 = a1; }
+              } else {
+                const unsigned nl = nonlow_rows >> par, md = mid_rows >> par;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                  const uint32_t wd = *(const uint32_t*)(st_hi + (2 * i + par) * STG_PITCH + (((cp >> 2) ^ (i & 3)) << 4) + (cp & 3) * 4);
+                  const float v0 = __uint_as_float(wd << 16), v1 = __uint_as_float(wd & 0xffff0000u);
+                  const float s0 = v0 * v0, s1 = v1 * v1;
+                  if ((nl >> (2 * i)) & 1) { a0 += s0; a1 += s1; }
+                  if ((md >> (2 * i)) & 1) { m0 += s0; m1 += s1; }
+                }
               }
               ea[qi][0] += a0; ea[qi][1] += a1; em[qi][0] += m0; em[qi][1] += m1;
             }

@@ -36,18 +36,34 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The same with a suspend-time hint: the thread may sleep in hardware for up to `ns` nanoseconds, or until the
+// phase completes, before the instruction returns, instead of coming back to the issue slots to poll.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
 
 // Bounded wait.  `abort_flag` (shared memory) is raised by the first waiter whose limit runs out;
 // every later wait in the CTA then returns at once, so all roles reach the common teardown.
 // Returns false when the wait was abandoned.
 constexpr long long kWaitLimitCycles = 4000000000LL;   // about two seconds of SM clock
+#ifndef FF_WAIT_HINT_NS
+#define FF_WAIT_HINT_NS 20000u                        // a waiting thread sleeps up to 20 us at a time (the abort flag is looked at in between)
+#endif
 
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                           long long limit_cycles = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait_hint(bar, parity, FF_WAIT_HINT_NS)) return true;
     if (*abort_flag) return false;
     if (clock64() - t0 > limit_cycles) {
       *abort_flag = 1;

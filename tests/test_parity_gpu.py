@@ -249,6 +249,7 @@ def test_replica_simt_attention_matches_too():
 def test_replica_separate_axis_passes_match_too():
     _run(C.R64K, alloc=[2, 4, 1, 7, 4, 2], impl=4)
     _run(C.R1M, alloc=[7, 2, 4, 1], impl=4)
+    _run(C.R_PAPER_REF, alloc=[1, 2, 4, 7], impl=4)      # head_dim 64: the byte-form intermediates' 64-channel layout
 
 
 def test_replica_generic_transform_matches_too():
