@@ -244,6 +244,12 @@ __device__ __forceinline__ bool row_exchange(unsigned long long* slots, int part
   return true;
 }
 
+// max of three (one instruction on sm_100)
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -479,6 +485,15 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
             chi = hi < TILE - 1 ? (int)(hi < -1 ? -1 : hi) : TILE - 1;
           }
         }
+        // (edge tiles) the valid columns of this thread's 32-column chunks as bit masks
+        uint32_t vmask[SCOLS / 32];
+#pragma unroll
+        for (int c = 0; c < SCOLS / 32; ++c) {
+          const int a = clo - (col0 + c * 32), b = chi - (col0 + c * 32);      // valid bits [a, b] of the chunk
+          const uint32_t lo_m = a <= 0 ? 0xffffffffu : (a >= 32 ? 0u : 0xffffffffu << a);
+          const uint32_t hi_m = b >= 31 ? 0xffffffffu : (b < 0 ? 0u : 0xffffffffu >> (31 - b));
+          vmask[c] = lo_m & hi_m;
+        }
         ok = __all_sync(0xffffffffu, mbar_wait(&sh.s_full[sx], cs & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
@@ -491,11 +506,11 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
           tmem_wait_ld();
           if (full) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, __uint_as_float(r[i]));
+            for (int i = 0; i < 32; i += 2) tmax = max3f(tmax, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
           } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (col0 + c * 32 + i >= clo && col0 + c * 32 + i <= chi) tmax = fmaxf(tmax, __uint_as_float(r[i]));
+              if (vmask[c] & (1u << i)) tmax = fmaxf(tmax, __uint_as_float(r[i]));
           }
         }
         // row maximum over the row's threads (slots alternate with the tile parity, so a partner's
@@ -542,12 +557,11 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const int col = col0 + c * 32 + 2 * i;
             float p0 = ex2(fmaf(__uint_as_float(r[2 * i]), sl2, -mb));
             float p1 = ex2(fmaf(__uint_as_float(r[2 * i + 1]), sl2, -mb));
             if (!full) {
-              if (col < clo || col > chi) p0 = 0.f;
-              if (col + 1 < clo || col + 1 > chi) p1 = 0.f;
+              if (!(vmask[c] & (1u << (2 * i)))) p0 = 0.f;
+              if (!(vmask[c] & (2u << (2 * i)))) p1 = 0.f;
             }
             sum += p0 + p1;
             const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
