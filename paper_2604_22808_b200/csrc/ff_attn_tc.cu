@@ -546,7 +546,8 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         if (need) { l *= alpha; m_ref = m_new; }
         // P = 2^(s*scale*log2e - m) as bf16 over the scores, partial row sum
         const float mb = m_ref * sl2;
-        float sum = 0.f;
+        float2 sum2 = make_float2(0.f, 0.f);              // (two scores per FMA / add: packed fp32 instructions)
+        const float2 sl22 = make_float2(sl2, sl2), nmb2 = make_float2(-mb, -mb);
 #pragma unroll
         for (int c = 0; c < SCOLS / 32; ++c) {
           // second sweep: the scores again (tensor-memory reads are cheap; keeping them in registers
@@ -557,19 +558,20 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            float p0 = ex2(fmaf(__uint_as_float(r[2 * i]), sl2, -mb));
-            float p1 = ex2(fmaf(__uint_as_float(r[2 * i + 1]), sl2, -mb));
+            const float2 arg = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sl22, nmb2);
+            float p0 = ex2(arg.x);
+            float p1 = ex2(arg.y);
             if (!full) {
               if (!(vmask[c] & (1u << (2 * i)))) p0 = 0.f;
               if (!(vmask[c] & (2u << (2 * i)))) p1 = 0.f;
             }
-            sum += p0 + p1;
+            sum2 = __fadd2_rn(sum2, make_float2(p0, p1));
             const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
             pk[i] = *(const uint32_t*)&v;
           }
           tmem_st16(s_addr + col0 + c * 16, pk);      // inside this thread's own score columns
         }
-        l += sum;
+        l += sum2.x + sum2.y;
         tmem_wait_st();
         if (!first && !waited_prev) {
           ok = __all_sync(0xffffffffu, mbar_wait(&sh.o_full[sx], co & 1, abort_flag));
