@@ -463,9 +463,9 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         bool full;
         if (x.band == 1) {
           const long long u0 = (long long)j * TILE;
-          // ranks grow with the class-local position, so the valid keys are a prefix
-          const long long last = mid_rank(dm, x.c, u0 + TILE - 1);
-          full = last < dm.Nmid;
+          // ranks grow with the class-local position, so the valid keys are a prefix; a class is a whole number
+          // of blocks and blocks tile the 128 rows, so only its last tile can hold keys past the band end
+          full = j + 1 < x.nk || mid_rank(dm, x.c, u0 + TILE - 1) < dm.Nmid;
           if (!full) {
             chi = -1;
             for (int cc = TILE - 1; cc >= 0; --cc)
