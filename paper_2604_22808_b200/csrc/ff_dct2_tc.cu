@@ -81,6 +81,7 @@ struct D2Shared {
   // slot while phase 2 of the current item reads the other.
   uint64_t buf_full[2];    // all rows of the item have landed in this CTA's slot (arrivals from every CTA's warps)
   uint64_t buf_half[2];    // (one CTA per plane) the rows of the first half of the second axis have landed
+  uint64_t half_free[2];   // (one CTA per plane) phase 2 has finished reading those rows (its k-steps 0..3 of every batch)
   uint64_t buf_free[2];    // every CTA of the cluster has finished reading the slot (phase 2 of the item)
   uint64_t mma2_done[2];   // this CTA's phase-2 instructions of the item (by slot) have completed
   uint32_t tmem_base;
@@ -230,6 +231,9 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   // of the second axis, i.e. rows 0..63 of every phase-2 tile = its k-steps 0..3.  Phase 2 of the item's first
   // batch starts on those while phase 1 still works on the second half.
   const bool half_start = cs == 1 && nb >= 2 && (nb & 1) == 0;
+  // ... and phase 1 of the next item may overwrite those rows as soon as phase 2 has read them (forward launch:
+  // measured slower for the inverse, whose phase 1 issues half as many instructions again)
+  const bool half_release = half_start && !P.in_split;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NSTG; ++i) { mbar_init(&sh.in_full[i], 1); mbar_init(&sh.in_empty[i], 1); }
@@ -237,6 +241,7 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
     for (int i = 0; i < NA2; ++i) { mbar_init(&sh.acc2_full[i], 1); mbar_init(&sh.acc2_empty[i], 256); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.buf_full[i], 8 * cs); mbar_init(&sh.buf_free[i], cs); mbar_init(&sh.buf_half[i], 8); }
     mbar_init(&sh.mma2_done[0], 1); mbar_init(&sh.mma2_done[1], 1);
+    mbar_init(&sh.half_free[0], 1); mbar_init(&sh.half_free[1], 1);
     sh.abort_flag = 0;
     fence_mbar_init();
   }
@@ -396,6 +401,9 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
             umma_ts(d_tm, tm + COL_A2H + ks * 8, xh + (uint64_t)(ks * 64), idesc, ks > 0 ? 1u : 0u);
             umma_ts(d_tm, tm + COL_A2L + ks * 8, xh + (uint64_t)(ks * 64), idesc, 1u);
             umma_ts(d_tm, tm + COL_A2H + ks * 8, xl + (uint64_t)(ks * 64), idesc, 1u);
+            // rows 0..63 of every tile have been read once the last batch's k-step 3 is done: phase 1 of the next
+            // item may overwrite them
+            if (ks == ROWS / 32 - 1 && kb == nb - 1 && half_release) umma_commit(&sh.half_free[sl]);
           }
           if (!ok) break;
           umma_commit(&sh.acc2_full[ab]);
@@ -438,11 +446,17 @@ dct2_tc_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       PROF_T0(te0);
       const int sl = (int)(ni % nsl);                         // the item's slot: free once phase 2 of item ni - nsl is done
       if (ni >= (unsigned)nsl) {
-        ok = __all_sync(0xffffffffu, mbar_wait_cluster(&sh.buf_free[sl], ((ni / nsl) - 1) & 1, abort_flag));
+        // (half_release: the first half of the batches writes rows phase 2 releases earlier; the rest waits below)
+        ok = half_release ? __all_sync(0xffffffffu, mbar_wait(&sh.half_free[sl], ((ni / nsl) - 1) & 1, abort_flag))
+                        : __all_sync(0xffffffffu, mbar_wait_cluster(&sh.buf_free[sl], ((ni / nsl) - 1) & 1, abort_flag));
         if (!ok) break;
       }
       if (threadIdx.x == 128) PROF_ADD(1, te0);
       for (int kb = 0; kb < nb && ok; ++kb, ++n1b) {
+        if (half_release && kb == nb / 2 && ni >= (unsigned)nsl) {
+          ok = __all_sync(0xffffffffu, mbar_wait_cluster(&sh.buf_free[sl], ((ni / nsl) - 1) & 1, abort_flag));
+          if (!ok) break;
+        }
         const int ab = n1b % NA1;
         PROF_T0(te1);
         ok = __all_sync(0xffffffffu, mbar_wait(&sh.acc1_full[ab], (n1b / NA1) & 1, abort_flag));
