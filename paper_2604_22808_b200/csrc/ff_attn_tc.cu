@@ -556,18 +556,27 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
           tmem_ld32(s_addr + col0 + c * 32, r);
           tmem_wait_ld();
           uint32_t pk[16];
+          if (full) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float2 arg = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sl22, nmb2);
-            float p0 = ex2(arg.x);
-            float p1 = ex2(arg.y);
-            if (!full) {
+            for (int i = 0; i < 16; ++i) {
+              const float2 arg = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sl22, nmb2);
+              const float2 pp = make_float2(ex2(arg.x), ex2(arg.y));
+              sum2 = __fadd2_rn(sum2, pp);
+              const __nv_bfloat162 v = __floats2bfloat162_rn(pp.x, pp.y);
+              pk[i] = *(const uint32_t*)&v;
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float2 arg = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sl22, nmb2);
+              float p0 = ex2(arg.x);
+              float p1 = ex2(arg.y);
               if (!(vmask[c] & (1u << (2 * i)))) p0 = 0.f;
               if (!(vmask[c] & (2u << (2 * i)))) p1 = 0.f;
+              sum2 = __fadd2_rn(sum2, make_float2(p0, p1));
+              const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
+              pk[i] = *(const uint32_t*)&v;
             }
-            sum2 = __fadd2_rn(sum2, make_float2(p0, p1));
-            const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
-            pk[i] = *(const uint32_t*)&v;
           }
           tmem_st16(s_addr + col0 + c * 16, pk);      // inside this thread's own score columns
         }
