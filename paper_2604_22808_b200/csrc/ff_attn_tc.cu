@@ -499,18 +499,27 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_a, cons
         tc_fence_after();
         // first sweep over this thread's raw scores: the row maximum of its columns
         float tmax = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < SCOLS / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(s_addr + col0 + c * 32, r);
+        {
+          // (both 32-column chunks are requested before the first is used: one tensor-memory latency instead of two)
+          static_assert(SCOLS == 64, "the first sweep reads two chunks");
+          uint32_t r0[32], r1[32];
+          tmem_ld32(s_addr + col0, r0);
+          tmem_ld32(s_addr + col0 + 32, r1);
           tmem_wait_ld();
           if (full) {
+            float t1 = -INFINITY;                          // two chains
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) tmax = max3f(tmax, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+            for (int i = 0; i < 32; i += 2) {
+              tmax = max3f(tmax, __uint_as_float(r0[i]), __uint_as_float(r0[i + 1]));
+              t1 = max3f(t1, __uint_as_float(r1[i]), __uint_as_float(r1[i + 1]));
+            }
+            tmax = fmaxf(tmax, t1);
           } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (vmask[c] & (1u << i)) tmax = fmaxf(tmax, __uint_as_float(r[i]));
+            for (int i = 0; i < 32; ++i) {
+              if (vmask[0] & (1u << i)) tmax = fmaxf(tmax, __uint_as_float(r0[i]));
+              if (vmask[1] & (1u << i)) tmax = fmaxf(tmax, __uint_as_float(r1[i]));
+            }
           }
         }
         // row maximum over the row's threads (slots alternate with the tile parity, so a partner's
